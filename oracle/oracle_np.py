@@ -1,0 +1,182 @@
+"""NumPy statement of the codec -- TEST INFRASTRUCTURE, not product code.
+
+A second, independently written CPU statement of the method of "Towards Low-bit
+Communication for Tensor Parallel LLM Inference" (arXiv 2411.07942), used to
+cross-check the scalar C oracle bit for bit and as the readable form of the
+algorithm.  It shares nothing with the CUDA library and must never be imported
+by it.
+
+BF16 tensors are ``np.uint16`` bit patterns.  Every calibration / parameter /
+quantiser operation is one ``np.float32`` operation (NumPy never fuses a
+multiply with an add); the reduction reference is ``np.float64``.
+
+Paper passages followed:
+  Section 3 "Calibration", Eq. (1)-(2)             -> col_minmax, calibrate
+  Section 3, R = 2 max(-m, M); R-bar = sum_i R^(i)  -> ranges
+  Section 3 "Selecting High Precision Features"    -> select, default_k (Section 4)
+  Section 3 symmetric Int4                          -> params, quantize_codes
+  Figure 2, Section 4 bit count                     -> pack, payload_bytes
+  Figure 2 caption, Section 5                       -> dequant_reduce
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F32 = np.float32
+LEVELS_MINUS_ONE = F32(15.0)          # 2**4 - 1 steps across the range R
+S_FLOOR = F32(2.0 ** -23)             # floor for a degenerate (zero) range
+Q_MIN, Q_MAX = F32(-8.0), F32(7.0)    # signed Int4 codes
+
+
+# ------------------------------------------------------------------ BF16 <-> f32
+def widen(bits: np.ndarray) -> np.ndarray:
+    """BF16 bit patterns -> float32, exactly."""
+    return (np.asarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)).view(F32)
+
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """float32 -> BF16 bit patterns, round to nearest even."""
+    u = np.asarray(x, dtype=F32).view(np.uint32)
+    nan = (u & np.uint32(0x7FFFFFFF)) > np.uint32(0x7F800000)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    r = np.where(nan, (u >> np.uint32(16)) | np.uint32(0x40), r)
+    return r.astype(np.uint16)
+
+
+def _order_key(bits: np.ndarray) -> np.ndarray:
+    """Monotone integer key of non-NaN BF16 patterns with -0 below +0."""
+    b = np.asarray(bits, dtype=np.uint16).astype(np.int32)
+    mag = b & 0x7FFF
+    return np.where(b & 0x8000, -mag - 1, mag)
+
+
+# ------------------------------------------------------------------ calibration
+def col_minmax(y_bits: np.ndarray):
+    """Eq. (1)-(2): min and max of every feature column over one sequence [S, E]."""
+    key = _order_key(y_bits)
+    lo = np.take_along_axis(y_bits, key.argmin(axis=0)[None, :], axis=0)[0]
+    hi = np.take_along_axis(y_bits, key.argmax(axis=0)[None, :], axis=0)[0]
+    return widen(lo), widen(hi)
+
+
+def calibrate(m, M, count: int, y_bits: np.ndarray, gamma):
+    """Fold sequences [n_seq, S, E] of one device into its (m, M), Eq. (1)-(2).
+
+    The first sequence a device sees initialises (m, M); afterwards
+    m <- (1-gamma) m + gamma min, literally left to right in float32."""
+    gamma = F32(gamma)
+    c = F32(F32(1.0) - gamma)
+    for seq in y_bits:
+        mn, mx = col_minmax(seq)
+        if count == 0:
+            m, M = mn.copy(), mx.copy()
+        else:
+            m = (c * m).astype(F32) + (gamma * mn).astype(F32)
+            M = (c * M).astype(F32) + (gamma * mx).astype(F32)
+        count += 1
+    return m.astype(F32), M.astype(F32), count
+
+
+def ranges(m: np.ndarray, M: np.ndarray):
+    """R^(i)_j = 2 max(-m, M) and R-bar_j = sum over devices (ascending, float32)."""
+    m = np.asarray(m, dtype=F32)
+    M = np.asarray(M, dtype=F32)
+    R = (F32(2.0) * np.maximum(-m, M)).astype(F32)
+    Rbar = R[0].copy()
+    for i in range(1, R.shape[0]):
+        Rbar = (Rbar + R[i]).astype(F32)
+    return R, Rbar
+
+
+def default_k(E: int) -> int:
+    """Section 4: k = floor(E / 64)."""
+    return E // 64
+
+
+def select(Rbar: np.ndarray, k: int) -> np.ndarray:
+    """Top-k features by R-bar; ties to the lower index; returned ascending."""
+    E = Rbar.shape[0]
+    order = sorted(range(E), key=lambda j: (-float(Rbar[j]), j))
+    return np.array(sorted(order[:k]), dtype=np.int32)
+
+
+def params(R: np.ndarray):
+    """Step s = R/15 floored at 2^-23, and the reciprocal the quantiser uses."""
+    s = (np.asarray(R, dtype=F32) / LEVELS_MINUS_ONE).astype(F32)
+    s = np.where(s >= S_FLOOR, s, S_FLOOR).astype(F32)
+    inv_s = (F32(1.0) / s).astype(F32)
+    return s, inv_s
+
+
+# ------------------------------------------------------------------ compression
+def lp_index(E: int, hp_idx: np.ndarray) -> np.ndarray:
+    keep = np.ones(E, dtype=bool)
+    keep[np.asarray(hp_idx, dtype=np.int64)] = False
+    return np.nonzero(keep)[0].astype(np.int32)
+
+
+def quantize_codes(y_bits: np.ndarray, inv_s: np.ndarray) -> np.ndarray:
+    """Symmetric Int4 codes in [-8, 7]: product rounded to float32, clamped,
+    then rounded half-to-even (np.rint)."""
+    with np.errstate(over="ignore"):
+        u = (widen(y_bits) * np.asarray(inv_s, dtype=F32)).astype(F32)
+    u = np.minimum(np.maximum(u, Q_MIN), Q_MAX)
+    return np.rint(u).astype(np.int8)
+
+
+def lp_bytes(T: int, E: int, k: int) -> int:
+    nib = T * (E - k)
+    return ((nib + 1) // 2 + 15) // 16 * 16
+
+
+def payload_bytes(T: int, E: int, k: int) -> int:
+    return lp_bytes(T, E, k) + 2 * T * k
+
+
+def bits_per_value(T: int, E: int, k: int) -> float:
+    return 8.0 * payload_bytes(T, E, k) / (T * E)
+
+
+def quantize_pack(y_bits: np.ndarray, hp_idx: np.ndarray, inv_s: np.ndarray) -> np.ndarray:
+    """One device's [T, E] BF16 partial sums -> payload bytes."""
+    T, E = y_bits.shape
+    k = len(hp_idx)
+    lp = lp_index(E, hp_idx)
+    codes = quantize_codes(y_bits[:, lp], inv_s[lp])            # [T, E-k]
+    nib = (codes.astype(np.int16) & 0xF).astype(np.uint8).reshape(-1)
+    if nib.size % 2:
+        nib = np.concatenate([nib, np.zeros(1, np.uint8)])
+    packed = nib[0::2] | (nib[1::2] << 4)
+    out = np.zeros(payload_bytes(T, E, k), dtype=np.uint8)
+    out[: packed.size] = packed
+    hp = np.ascontiguousarray(y_bits[:, np.asarray(hp_idx, dtype=np.int64)])
+    out[lp_bytes(T, E, k):] = hp.view(np.uint8).reshape(-1)
+    return out
+
+
+def unpack(payload: np.ndarray, T: int, E: int, k: int):
+    """Payload -> (codes [T, E-k] int8, hp [T, k] BF16 bits)."""
+    L = E - k
+    nb = lp_bytes(T, E, k)
+    b = payload[:nb]
+    nib = np.empty(nb * 2, dtype=np.uint8)
+    nib[0::2] = b & 0xF
+    nib[1::2] = b >> 4
+    nib = nib[: T * L].astype(np.int8)
+    codes = np.where(nib >= 8, nib - 16, nib).astype(np.int8).reshape(T, L)
+    hp = payload[nb:].view(np.uint16).reshape(T, k) if k else np.zeros((T, 0), np.uint16)
+    return codes, hp
+
+
+# ------------------------------------------------------------------ decompression + sum
+def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray):
+    """Sum over devices of the dequantised payloads, in float64, original feature order."""
+    k = len(hp_idx)
+    lp = lp_index(E, hp_idx)
+    out = np.zeros((T, E), dtype=np.float64)
+    for i, p in enumerate(payloads):
+        codes, hp = unpack(np.asarray(p, dtype=np.uint8), T, E, k)
+        out[:, lp] += codes.astype(np.float64) * s[i, lp].astype(np.float64)[None, :]
+        if k:
+            out[:, np.asarray(hp_idx, dtype=np.int64)] += widen(hp).astype(np.float64)
+    return out
