@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the low-bit tensor-parallel synchronisation hot path on B200.
+
+One "step" = one synchronisation of the Llama-2-13B-shaped prefill workload
+(BASELINE config 2): N = 4 simulated tensor-parallel shards, 2048 tokens x 5120
+features of BF16 partial sums each; tpq_quantize_pack once per shard, then one
+tpq_dequant_reduce (BF16 output) over the 4 payloads.  The static parameters
+(calibration + feature selection) are computed once before the timed region,
+as in the method (they never change at inference time); their throughput is
+reported separately under "extra".
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Metric: GB/s of BF16 input processed (N*T*E*2 bytes per step), whole job.
+N > 1 GPUs (torchrun): every rank runs the same workload on its own batch, no
+data-path collective (replicas of the single-GPU simulation): weak scaling.
+
+--impl reference times the CPU oracle (oracle/, scalar C + OpenMP) on the host
+cores on the same workload; there is no other reference implementation.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "quantize_pack + dequant_reduce GB/s (BF16 input)"
+UNIT = "GB/s"
+WORKLOAD = "llama13b_prefill"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the current kernel).
+NCU_TRAFFIC_BYTES = {"quantize_tiled": None, "dequant_tiled": None}
+
+
+# ------------------------------------------------------------------ helpers
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def payload_bytes(T, E, k):
+    nib = T * (E - k)
+    return ((nib + 1) // 2 + 15) // 16 * 16 + 2 * T * k
+
+
+def algorithmic_bytes(N, T, E, k):
+    """Bytes the method itself must move per launch (tables are O(N*E) and cache resident)."""
+    P = payload_bytes(T, E, k)
+    return {"quantize_pack": 2 * T * E + P, "dequant_reduce": N * P + 2 * T * E}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [r for ts, r in self.rows if t0 - 0.05 <= ts <= t1 + 0.15] or [r for _, r in self.rows]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def aggregate_over_ranks(local_ms: float, local_units: float, dist=None):
+    """max over ranks of the step time, sum over ranks of the units one step processes."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms, local_units
+    import torch
+
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([local_ms], dtype=torch.float64, device=dev)
+    u = torch.tensor([local_units], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+# ------------------------------------------------------------------ the CPU oracle leg
+def oracle_leg(w, steps: int, warmup: int):
+    """Times the oracle as it stands on one full-size step; returns (GB/s, ms_per_step, cores, sample)."""
+    import oracle
+    from paper_2411_07942_b200 import synth
+
+    orc = oracle.c()
+    N, T, E = w.n_shards, w.tokens, w.features
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, n_seq=2, tokens=256, scale=scale) for i in range(N)]
+    ms, Ms = [], []
+    for i in range(N):
+        m, M, _ = orc.calibrate(None, None, 0, cal[i], 0.01)
+        ms.append(m)
+        Ms.append(M)
+    R, Rbar = orc.ranges(np.stack(ms), np.stack(Ms))
+    hp = orc.select(Rbar, orc.default_k(E))
+    s, inv = orc.params(R)
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+
+    def step():
+        pl = [orc.quantize_pack(ys[i], hp, inv[i]) for i in range(N)]
+        orc.dequant_reduce(pl, T, E, hp, s, want_chain32=True)
+
+    for _ in range(warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    gbs = N * T * E * 2 / dt / 1e9
+    sample = f"{steps} full steps of {w.name} (N={N}, {T}x{E} BF16 per shard), scalar C oracle, OpenMP over rows"
+    return gbs, dt * 1e3, orc.num_threads(), sample
+
+
+# ------------------------------------------------------------------ main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="tpq", choices=["tpq", "reference"])
+    ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank, local_rank, world = dist_env()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    from paper_2411_07942_b200 import synth
+
+    w = synth.WORKLOADS[WORKLOAD]
+    N, T, E, k = w.n_shards, w.tokens, w.features, w.k
+    in_bytes = N * T * E * 2
+    config = {"workload": f"{WORKLOAD}: N={N} shards x {T} tokens x {E} features BF16, k={k} BF16 features, "
+                          f"BF16 output", "n_shards": N, "tokens": T, "features": E, "k": k}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return 0
+        steps = max(1, min(args.steps, 10))
+        gbs, ms, cores, sample = oracle_leg(w, steps, min(args.warmup, 1))
+        line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": 0, "steps": steps,
+                "warmup": min(args.warmup, 1), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+                "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return 0
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2411_07942_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    peak, peak_kind = measured_peak()
+    scale = synth.column_scales(w)
+    stream = torch.cuda.current_stream()
+    sh = stream.cuda_stream
+
+    # ---- static parameters: calibration (timed separately) + selection
+    t = binding.Tpq(N, E)
+    cal_seqs, cal_S = 8, w.calib_tokens
+    cal_bufs = [synth.activations_torch(w, i, cal_seqs * cal_S, dev, stream=1, scale=scale) for i in range(N)]
+    for i in range(N):
+        t.calibrate_ranges(i, cal_bufs[i].data_ptr(), cal_seqs, cal_S, stream=sh)
+    torch.cuda.synchronize()
+    # calibration throughput (not part of the step): a second context folds the same set a few times
+    tc = binding.Tpq(N, E)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(N):
+        tc.calibrate_ranges(i, cal_bufs[i].data_ptr(), cal_seqs, cal_S, stream=sh)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    cal_reps = 3
+    for _ in range(cal_reps):
+        for i in range(N):
+            tc.calibrate_ranges(i, cal_bufs[i].data_ptr(), cal_seqs, cal_S, stream=sh)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    cal_ms = e0.elapsed_time(e1) / cal_reps
+    cal_bytes = N * cal_seqs * cal_S * E * 2
+    tc.close()
+    ts0 = time.perf_counter()
+    hp = t.select_features(-1)
+    select_ms = (time.perf_counter() - ts0) * 1e3
+    assert len(hp) == k
+    del cal_bufs
+    P = t.payload_bytes(T)
+    comm = t.comm_bytes(T)
+    alg = algorithmic_bytes(N, T, E, k)
+
+    # ---- rotating buffer sets (inputs resident in HBM; working set > L2)
+    sets = []
+    for b in range(args.sets):
+        ys = [synth.activations_torch(w, i, T, dev, stream=2 + b, scale=scale) for i in range(N)]
+        pls = [torch.empty(P, dtype=torch.uint8, device=dev) for _ in range(N)]
+        out = torch.empty((T, E), dtype=torch.bfloat16, device=dev)
+        sets.append((ys, pls, out))
+    set_bytes = in_bytes + N * P + 2 * T * E
+    config["l2"] = (f"rotating {args.sets} buffer sets, {args.sets * set_bytes / 1e6:.0f} MB touched between "
+                    f"reuses (> 126 MB L2)")
+
+    def step(b):
+        ys, pls, out = sets[b % args.sets]
+        for i in range(N):
+            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
+        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for b in range(args.warmup):
+        step(b)
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = t.launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    wall0 = time.time()
+    ev0.record(stream)
+    for b in range(args.steps):
+        step(b)
+    ev1.record(stream)
+    barrier()
+    wall1 = time.time()
+    local_ms = ev0.elapsed_time(ev1) / args.steps
+    gpu_launches = t.launch_count() - launches0
+
+    # ---- per-kernel durations, same buffers and rotation, CUDA events on the launching stream
+    def time_loop(fn, reps):
+        for b in range(3):
+            fn(b)
+        torch.cuda.synchronize()
+        a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for b in range(reps):
+            fn(b)
+        z.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / reps
+
+    def q_only(b):
+        ys, pls, _ = sets[b % args.sets]
+        for i in range(N):
+            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
+
+    def d_only(b):
+        _, pls, out = sets[b % args.sets]
+        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+
+    reps = max(20, min(args.steps, 200))
+    q_ms = time_loop(q_only, reps) / N          # per launch
+    d_ms = time_loop(d_only, reps)
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+
+    # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
+    ys0, pls0, out0 = sets[0]
+    host_in = [torch.empty((T, E), dtype=torch.bfloat16).pin_memory() for _ in range(N)]
+    for i in range(N):
+        host_in[i].copy_(ys0[i])
+    host_out = torch.empty((T, E), dtype=torch.bfloat16).pin_memory()
+
+    def e2e_step(b):
+        ys, pls, out = sets[b % args.sets]
+        for i in range(N):
+            ys[i].copy_(host_in[i], non_blocking=True)
+            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
+        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+        host_out.copy_(out, non_blocking=True)
+
+    e2e_reps = max(5, min(args.steps, 30))
+    for b in range(3):
+        e2e_step(b)
+    barrier()
+    a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for b in range(e2e_reps):
+        e2e_step(b)
+    z.record(stream)
+    barrier()
+    e2e_local_ms = a.elapsed_time(z) / e2e_reps
+    assert t.device_status() == 0
+
+    ms, units = aggregate_over_ranks(local_ms, float(in_bytes), dist if world > 1 else None)
+    e2e_ms, _ = aggregate_over_ranks(e2e_local_ms, float(in_bytes), dist if world > 1 else None)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    value = units / (ms * 1e-3) / 1e9
+    dom = "quantize_pack" if N * q_ms >= d_ms else "dequant_reduce"
+    dom_ms = q_ms if dom == "quantize_pack" else d_ms
+    achieved = alg[dom] / (dom_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": alg[dom], "launch_ms": dom_ms,
+                "traffic": NCU_TRAFFIC_BYTES["quantize_tiled" if dom == "quantize_pack" else "dequant_tiled"]}
+    extra = {
+        "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
+        "payload_bytes_per_shard": int(comm.payload_bytes),
+        "comm_bytes_per_rank": {"quantized_allgather": int(comm.quantized_allgather_send),
+                                "bf16_allgather": int(comm.bf16_allgather_send),
+                                "bf16_ring_allreduce": int(comm.bf16_ring_allreduce_send)},
+        "quantize_pack": {"ms_per_launch": q_ms, "hbm_GBps": alg["quantize_pack"] / q_ms / 1e6,
+                          "frac_of_measured": alg["quantize_pack"] / q_ms / 1e6 / peak,
+                          "frac_of_8000": alg["quantize_pack"] / q_ms / 1e6 / NOMINAL_HBM_GBS,
+                          "input_GBps": 2 * T * E / q_ms / 1e6},
+        "dequant_reduce": {"ms_per_launch": d_ms, "hbm_GBps": alg["dequant_reduce"] / d_ms / 1e6,
+                           "frac_of_measured": alg["dequant_reduce"] / d_ms / 1e6 / peak,
+                           "frac_of_8000": alg["dequant_reduce"] / d_ms / 1e6 / NOMINAL_HBM_GBS,
+                           "input_GBps": in_bytes / d_ms / 1e6},
+        "calibrate_ranges": {"ms": cal_ms, "bytes": cal_bytes, "hbm_GBps": cal_bytes / cal_ms / 1e6,
+                             "frac_of_measured": cal_bytes / cal_ms / 1e6 / peak,
+                             "shape": f"{N} shards x {cal_seqs} sequences x {cal_S} tokens x {E}"},
+        "select_features_ms_incl_sync": select_ms,
+    }
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": config, "clocks": clocks, "gpu_launches": int(gpu_launches),
+            "e2e": {"value": world * in_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": 2 * T * E, "ms_per_step": e2e_ms},
+            "roofline": roofline, "extra": extra}
+    if world == 1 and not args.no_cpu_baseline:
+        gbs, cms, cores, sample = oracle_leg(w, 5, 1)
+        line["cpu_baseline"] = {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                                "ms_per_step": cms}
+    print(json.dumps(line))
+    t.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

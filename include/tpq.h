@@ -1,0 +1,202 @@
+/*
+ * tpq.h -- C ABI of libtpq: low-bit synchronisation of tensor-parallel partial
+ * sums on NVIDIA B200 (sm_100a), after "Towards Low-bit Communication for
+ * Tensor Parallel LLM Inference" (arXiv 2411.07942).
+ *
+ * Setting (paper Section 2): N devices each hold a partial sum
+ * f^(i)(x^(i)) in R^E per token; the synchronised value is their sum.  The
+ * library provides the per-device compression C^(i) (tpq_quantize_pack), the
+ * decompress-and-sum  sum_i D^(i)  (tpq_dequant_reduce), and the calibration
+ * that fixes their static parameters (tpq_calibrate_ranges,
+ * tpq_select_features), paper Section 3.
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are host memory.
+ *   - BF16 tensors are 16-bit patterns, row-major, row stride given in ELEMENTS
+ *     (any stride >= E; the tiled kernels need E, k and the strides to be
+ *     multiples of 8, other shapes run on slower shape-generic kernels).
+ *   - The caller owns every data buffer.  The library owns only the context
+ *     and its small device tables (O(N*E) floats), released by tpq_destroy.
+ *   - Calls that take a `cuda_stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) only ENQUEUE work on it and never synchronise.  Calls
+ *     that return host data synchronise the device.
+ *   - Arguments are validated before anything is launched; a non-zero status
+ *     means nothing was enqueued.  No entry point throws, aborts or traps.
+ *   - A context is bound to the CUDA device that was current at tpq_create and
+ *     may be used from one host thread at a time.
+ *   - One context serves all N simulated devices: the static parameters and
+ *     the selected feature set are identical on every device by construction
+ *     (Section 3: "fixed across all sequences and devices").
+ */
+#ifndef TPQ_H
+#define TPQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tpq_ctx tpq_ctx; /* opaque */
+
+typedef enum {
+    TPQ_OK = 0,
+    TPQ_ERR_INVALID_ARG = 1, /* null pointer, negative size, shard out of range, unsorted index set ... */
+    TPQ_ERR_BAD_STATE = 2,   /* e.g. quantize before a feature set exists, select before calibration */
+    TPQ_ERR_SIZE = 3,        /* a caller buffer is too small */
+    TPQ_ERR_ALIGN = 4,       /* a device pointer is not 16-byte aligned */
+    TPQ_ERR_CUDA = 5,        /* a CUDA call failed; text in tpq_last_error */
+    TPQ_ERR_NOMEM = 6,       /* host or device allocation failed */
+    TPQ_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (see tpq_device_status) */
+} tpq_status;
+
+typedef enum { TPQ_OUT_BF16 = 0, TPQ_OUT_FP32 = 1 } tpq_out_dtype;
+
+/* Options for tpq_set_option. */
+typedef enum {
+    TPQ_OPT_KERNEL_PATH = 0 /* 0 = automatic (default); 1 = always the shape-generic kernels;
+                               2 = the tiled kernels, TPQ_ERR_INVALID_ARG from the call if the
+                               shape does not admit them (E, k and strides multiples of 8) */
+} tpq_option;
+
+/* Bytes a real exchange would move per synchronisation and per device
+ * (paper Section 5: all-reduce executed as all-gather + local reduction). */
+typedef struct tpq_comm_report {
+    int64_t payload_bytes;             /* P: one device's payload for T tokens                         */
+    int64_t quantized_allgather_send;  /* (N-1) * P, unicast all-gather of payloads (the method)        */
+    int64_t bf16_allgather_send;       /* (N-1) * 2*T*E, all-gather of the raw BF16 partial sums         */
+    int64_t bf16_ring_allreduce_send;  /* 2*(N-1)/N * 2*T*E, bandwidth-optimal BF16 all-reduce           */
+    double bits_per_value;             /* 8*P / (T*E); equals 4 + 12k/E up to the 16-byte pad (Sec. 4)   */
+    double bits_per_value_formula;     /* 4 + 12k/E                                                      */
+} tpq_comm_report;
+
+/* ---------------------------------------------------------------- context */
+
+/* Create a context for n_shards (N >= 1) devices and n_features (E >= 1)
+ * features on the current CUDA device.  bits must be 4 (the paper's Int4,
+ * Section 3); gamma is the moving-average constant of Eq. (1)-(2) (the paper
+ * uses 0.01), 0 <= gamma <= 1.  Errors: INVALID_ARG, NOMEM, CUDA. */
+tpq_status tpq_create(tpq_ctx **ctx, int n_shards, int n_features, int bits, float gamma);
+tpq_status tpq_destroy(tpq_ctx *ctx); /* NULL is accepted */
+tpq_status tpq_set_option(tpq_ctx *ctx, tpq_option opt, int value);
+
+/* ------------------------------------------------------------ calibration */
+
+/* Section 3 "Calibration", Eq. (1)-(2): fold n_seq sequences of device `shard`
+ * into its running (m_j, M_j), in index order.  For every sequence the
+ * column-wise minimum and maximum over its S tokens are taken; the first
+ * sequence a device ever sees initialises (m, M), later ones update
+ *   m <- (1-gamma) m + gamma min,  M <- (1-gamma) M + gamma max
+ * in binary32, evaluated left to right.
+ *   y_bf16_dev : [n_seq][S][E] BF16, row stride row_stride_elems (>= E), the
+ *                sequences back to back (sequence q starts at row q*S).
+ * Enqueues on cuda_stream.  May grow a context-owned scratch buffer
+ * (cudaMalloc) when n_seq*S exceeds every earlier call.
+ * n_seq == 0 is a no-op.  Errors: INVALID_ARG, ALIGN, NOMEM, CUDA. */
+tpq_status tpq_calibrate_ranges(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t n_seq, int64_t S,
+                                int64_t row_stride_elems, void *cuda_stream);
+
+/* Section 3 "Selecting High Precision Features": R^(i)_j = 2 max(-m, M),
+ * aggregated range Rbar_j = sum_i R^(i)_j (binary32, devices ascending), the
+ * k features with the largest Rbar_j (ties: lower index) become the BF16 set;
+ * every other feature gets its static Int4 step s = R/15 (floored at 2^-23)
+ * and reciprocal.  k < 0 selects the paper's k = floor(E/64) (Section 4).
+ * Every device must have been calibrated with at least one sequence
+ * (else BAD_STATE).  Writes the k indices, ascending, to hp_idx_out_host
+ * (capacity >= k int32; may be NULL) and k to k_out (may be NULL).
+ * Synchronises the device. */
+tpq_status tpq_select_features(tpq_ctx *ctx, int k, int32_t *hp_idx_out_host, int *k_out);
+
+/* Install an arbitrary feature set (strictly ascending indices in [0, E),
+ * 0 <= k <= E) instead of the top-k one: the paper's "Int4" (k = 0) and
+ * "Int4 + Random BF16" baselines (Section 4), or a restored set.  Steps are
+ * derived from the calibrated ranges as in tpq_select_features.  Synchronises. */
+tpq_status tpq_set_features(tpq_ctx *ctx, const int32_t *hp_idx_host, int k);
+
+/* Install calibration state directly: m and M are [N][E] binary32 (host),
+ * counts[N] the number of sequences each device has folded.  Used to resume
+ * calibration or to skip it.  Synchronises. */
+tpq_status tpq_set_ranges(tpq_ctx *ctx, const float *m_host, const float *M_host, const int64_t *counts_host);
+
+/* Read back state (host outputs, any may be NULL; synchronises):
+ * m, M, R are [N][E]; Rbar is [E].  R and Rbar are valid after a feature set exists. */
+tpq_status tpq_get_ranges(tpq_ctx *ctx, float *m_host, float *M_host, float *R_host, float *Rbar_host);
+/* s and inv_s are [N][E] (entries at selected features are defined but unused). BAD_STATE before a feature set. */
+tpq_status tpq_get_scales(tpq_ctx *ctx, float *s_host, float *inv_s_host);
+/* Number of selected features, or -1 before a feature set exists. */
+int tpq_num_selected(const tpq_ctx *ctx);
+/* The selected indices, ascending (capacity >= k).  BAD_STATE before a feature set. */
+tpq_status tpq_get_features(tpq_ctx *ctx, int32_t *hp_idx_out_host);
+
+/* ------------------------------------------------------------- the payload */
+
+/* Payload size in bytes for T tokens with the current feature set:
+ *   roundup16(ceil(T*(E-k)/2)) + 2*T*k
+ * (Section 4 counts (E-k) 4-bit codes and k BF16 values per token).
+ * Layout: one flat stream of 4-bit two's-complement codes in (token, feature
+ * with the selected ones removed) order, low nibble first, zero padded to a
+ * multiple of 16 bytes; then T*k BF16 values, token-major, selected features
+ * ascending.  No header; the static steps are never transmitted.
+ * Returns 0 before a feature set exists or for T <= 0. */
+size_t tpq_payload_bytes(const tpq_ctx *ctx, int64_t T);
+/* The same closed form without a context. */
+size_t tpq_payload_bytes_for(int64_t T, int64_t E, int64_t k);
+
+/* Section 5 / Section 4: bytes per synchronisation and bits per value. */
+tpq_status tpq_comm_bytes(const tpq_ctx *ctx, int64_t T, tpq_comm_report *out);
+
+/* --------------------------------------------------------- the hot path */
+
+/* C^(i) (Sections 2-3, Figure 2): one device's [T][E] BF16 partial sums ->
+ * payload.  Low-precision feature: u = fl(x * inv_s); u clamped to [-8, 7];
+ * code = round-half-to-even(u) (two binary32 roundings, never fused).
+ * Selected feature: the BF16 pattern is copied unchanged.
+ *   y_bf16_dev  : [T][E] BF16, row stride row_stride_elems (>= E)
+ *   payload_dev : >= tpq_payload_bytes(ctx, T) bytes, 16-byte aligned; every
+ *                 byte of the payload (padding included) is written.
+ * Enqueues on cuda_stream; T == 0 is a no-op.
+ * Errors: BAD_STATE (no feature set), INVALID_ARG, ALIGN, SIZE, CUDA. */
+tpq_status tpq_quantize_pack(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t T, int64_t row_stride_elems,
+                             void *payload_dev, size_t payload_capacity, void *cuda_stream);
+
+/* sum_i D^(i) (Figure 2 caption; Section 5 "local reduction"): N payloads ->
+ * the synchronised [T][E] output in the original feature order.
+ * Low-precision feature: sum_i code_i * s^(i)_j; selected feature: sum_i of
+ * the BF16 values.  Accumulation is binary32 in ascending device order with
+ * one final rounding for BF16 output.
+ *   payloads_dev_host : HOST array of n_payloads DEVICE pointers, device order;
+ *                       n_payloads must equal N; each 16-byte aligned
+ *   out_dev           : [T][E] of dt, row stride out_row_stride_elems (>= E)
+ * Enqueues on cuda_stream; T == 0 is a no-op.
+ * Errors: BAD_STATE, INVALID_ARG, ALIGN, CUDA. */
+tpq_status tpq_dequant_reduce(tpq_ctx *ctx, const void *const *payloads_dev_host, int n_payloads, int64_t T,
+                              void *out_dev, tpq_out_dtype dt, int64_t out_row_stride_elems, void *cuda_stream);
+
+/* ------------------------------------------------- checkpoint and status */
+
+/* Serialise / restore the whole static state (N, E, bits, gamma, counts, m, M,
+ * feature set) as a flat little-endian blob.  tpq_get_state with blob == NULL
+ * writes the required size to *bytes; otherwise *bytes is the capacity on
+ * entry and the size written on return.  tpq_set_state requires a context of
+ * the same N, E and bits.  Both synchronise. */
+tpq_status tpq_get_state(tpq_ctx *ctx, void *blob_host, size_t *bytes);
+tpq_status tpq_set_state(tpq_ctx *ctx, const void *blob_host, size_t bytes);
+
+/* Synchronise and read the device-side status word: TPQ_OK, or
+ * TPQ_ERR_TIMEOUT if a kernel's bounded wait on an asynchronous copy gave up
+ * (the kernel then returned early and its output is incomplete).  The word is
+ * cleared by the call. */
+tpq_status tpq_device_status(tpq_ctx *ctx);
+
+/* Kernels launched by this context since creation (for launch accounting). */
+int64_t tpq_launch_count(const tpq_ctx *ctx);
+
+const char *tpq_status_string(tpq_status st);
+const char *tpq_last_error(const tpq_ctx *ctx); /* "" if none; valid until the next call on ctx */
+const char *tpq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TPQ_H */

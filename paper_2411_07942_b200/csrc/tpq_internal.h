@@ -1,0 +1,76 @@
+// Internal declarations shared by the translation units of libtpq (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tpq.h"
+
+#define TPQ_MAX_SHARDS 64
+
+// Device tables of one context.  All in the ORIGINAL feature order unless noted.
+struct tpq_tables {
+    float *m, *M;        // [N][E] running minimum / maximum, Eq. (1)-(2)
+    float *R;            // [N][E] symmetric range 2 max(-m, M)
+    float *Rbar;         // [E]    aggregated range
+    float *s, *inv_s;    // [N][E] Int4 step and its reciprocal
+    float *s_k;          // [N][E] step with 0 at selected features (dequantiser's copy)
+    uint8_t *flag;       // [E]    1 = selected (kept in BF16)
+    int32_t *hpre;       // [E]    number of selected features before j
+    int32_t *pos;        // [E]    >= 0: slot in the compacted code stream; < 0: -(h+1), h = rank among selected
+    int32_t *hp_idx;     // [E]    first k entries: selected features, ascending
+    int32_t *lp_idx;     // [E]    first E-k entries: the others, ascending
+    uint32_t *grp;       // [ceil(E/8)] per group of 8 features: (selected before the group << 8) | 8-bit mask
+    int *status;         // device status word (0 = ok)
+};
+
+struct tpq_ctx {
+    int N, E, bits;
+    float gamma;
+    int k;              // -1 until a feature set exists
+    int device;
+    int sm_count;
+    int smem_optin;     // max dynamic shared memory per block
+    int kernel_path;    // TPQ_OPT_KERNEL_PATH
+    int64_t counts[TPQ_MAX_SHARDS];
+    tpq_tables t;
+    void *scratch;      // calibration partial extremes
+    size_t scratch_bytes;
+    int64_t launches;
+    char err[512];
+};
+
+// Payload geometry (Section 4 bit count; layout documented in tpq.h).
+static inline int64_t tpq_lp_bytes_i(int64_t T, int64_t E, int64_t k)
+{
+    int64_t nib = T * (E - k);
+    int64_t b = (nib + 1) / 2;
+    return (b + 15) / 16 * 16;
+}
+
+// ---- launchers (each returns the launch error, enqueues on `st`, adds to *launches)
+
+// Eq. (1)-(2): column extremes of n_seq sequences, then the moving-average fold.
+size_t tpq_calib_scratch_bytes(int64_t n_seq, int64_t S, int E, int sm_count, int *n_split_out);
+cudaError_t tpq_launch_calibrate(const uint16_t *y, int64_t n_seq, int64_t S, int64_t stride, int E, float *m,
+                                 float *M, int64_t count0, float gamma, void *scratch, int n_split, cudaStream_t st,
+                                 int64_t *launches);
+
+// Section 3: ranges, aggregate, steps; top-k flags (or flags given); index tables.
+cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_topk_flags(const tpq_tables &t, int E, int k, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
+
+// C^(i): quantise + pack.
+bool tpq_quantize_tiled_ok(const tpq_ctx *c, int64_t T, int64_t stride);
+cudaError_t tpq_launch_quantize_generic(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
+                                        uint8_t *payload, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
+                                      uint8_t *payload, cudaStream_t st, int64_t *launches);
+
+// sum_i D^(i): dequantise + reduce.
+bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int fp32_out);
+cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,
+                                       int fp32_out, int64_t out_stride, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,
+                                     int fp32_out, int64_t out_stride, cudaStream_t st, int64_t *launches);

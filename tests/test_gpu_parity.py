@@ -1,0 +1,336 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.  Integer / byte / index results bit-exact; reduction
+outputs within 1e-5 relative (FP32) or 1 BF16 ulp (BF16) of the oracle's FP64 sum."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+import oracle  # noqa: E402
+from paper_2411_07942_b200 import binding, synth  # noqa: E402
+
+import gpu_util as gu  # noqa: E402
+from util import bf16_bits, finite_bf16_patterns  # noqa: E402
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    gu.ensure_lib()
+
+
+def _workload(N, T, E, seed, n_out=3, calib=(3, 8)):
+    return synth.Workload("t", N, T, E, 0.6, n_out, 20.0, 200.0, calib[0], calib[1], seed)
+
+
+def _full_pipeline(w, k, path, stride_pad=0, chunks=None):
+    orc = oracle.c()
+    t = binding.Tpq(w.n_shards, w.features)
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, scale=scale) for i in range(w.n_shards)]
+    m, M = gu.calibrate_both(t, cal, chunks=chunks)
+    gm, gM = t.get_ranges(with_R=False)
+    assert gu.bits_equal(gm, m) and gu.bits_equal(gM, M), "calibration state differs"
+    hp = t.select_features(k)
+    R, Rbar = orc.ranges(m, M)
+    kk = orc.default_k(w.features) if k < 0 else k
+    assert hp.tolist() == orc.select(Rbar, kk).tolist()
+    _, _, gR, gRbar = t.get_ranges()
+    assert gu.bits_equal(gR, R) and gu.bits_equal(gRbar, Rbar)
+    s, inv = orc.params(R)
+    gs, ginv = t.get_scales()
+    assert gu.bits_equal(gs, s) and gu.bits_equal(ginv, inv)
+    ys = [synth.activations_np(w, i, w.tokens, scale=scale) for i in range(w.n_shards)]
+    gu.run_sync(t, ys, k_expect=kk, path=path, stride_pad=stride_pad)
+    t.close()
+
+
+def test_tiny_config_end_to_end():
+    """BASELINE config 1: N=2, 16 tokens x 256 features, 64 calibration tokens, seed 0."""
+    w = synth.WORKLOADS["tiny"]
+    _full_pipeline(w, -1, binding.PATH_AUTO)          # k = 4: not a multiple of 8 -> shape-generic kernels
+    _full_pipeline(w, 8, binding.PATH_TILED)          # same data with k = 8 through the tiled kernels
+
+
+@pytest.mark.parametrize("N,T,E,k", [(2, 3, 65, 1), (3, 17, 130, 2), (2, 5, 253, 9), (1, 1, 64, 0), (2, 4, 40, 40),
+                                     (4, 9, 24, 0), (2, 1, 8, 3), (5, 33, 100, -1)])
+def test_generic_path_odd_shapes(N, T, E, k):
+    _full_pipeline(_workload(N, T, E, 100 + E + T), k, binding.PATH_AUTO)
+
+
+@pytest.mark.parametrize("N,T,E,k,pad", [(2, 67, 512, 8, 0), (4, 301, 1024, 16, 0), (4, 37, 5120, 80, 64),
+                                         (8, 64, 4608, 72, 0), (16, 33, 2048, 32, 8), (3, 1, 256, 8, 0),
+                                         (2, 150, 8192, 128, 0), (2, 600, 64, 8, 0), (2, 19, 16, 8, 0),
+                                         (2, 7, 10240, 160, 0), (4, 12, 256, 0, 0), (2, 11, 256, 248, 0)])
+def test_tiled_path_shapes(N, T, E, k, pad):
+    """Several tiles, ragged tails, strided input, every group-of-8 hole pattern."""
+    _full_pipeline(_workload(N, T, E, 7 * E + T), k, binding.PATH_TILED, stride_pad=pad)
+
+
+def test_tiled_equals_generic_on_clustered_feature_sets():
+    """Arbitrary feature sets (the paper's random-selection baseline and worse):
+    runs of adjacent selected features, whole groups of 8, first and last feature."""
+    N, T, E = 3, 29, 512
+    w = _workload(N, T, E, 77)
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, scale=scale) for i in range(N)]
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+    rng = np.random.default_rng(1)
+    sets = [
+        list(range(0, 8)),                                   # a whole group
+        list(range(0, 15)) + [511],
+        [0, 1, 2, 3, 4, 5, 6, 500, 501, 502, 503, 504, 505, 506, 507, 511],
+        list(range(3, 3 + 24)),                              # straddles groups
+        sorted(rng.permutation(E)[:64].tolist()),            # random baseline, k = E/8
+        sorted(rng.permutation(E)[:8].tolist()),
+        list(range(E - 8, E)),
+        list(range(8, E)),                                   # only the first group is quantised
+    ]
+    for hp in sets:
+        assert len(hp) % 8 == 0
+        t = binding.Tpq(N, E)
+        gu.calibrate_both(t, cal)
+        t.set_features(hp)
+        assert t.get_features().tolist() == hp
+        a = gu.run_sync(t, ys, path=binding.PATH_GENERIC)
+        b = gu.run_sync(t, ys, path=binding.PATH_TILED)
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+        t.close()
+
+
+@pytest.mark.parametrize("path", [binding.PATH_GENERIC, binding.PATH_TILED])
+def test_quantiser_all_bf16_patterns_and_ties(path):
+    """Every non-NaN BF16 pattern through the GPU quantiser at several steps, among them
+    s = 1 (exact ties) -- bit-exact against the oracle."""
+    orc = oracle.c()
+    pats = finite_bf16_patterns()
+    E = 256
+    T = (pats.size + E - 1) // E
+    y = np.zeros(T * E, np.uint16)
+    y[: pats.size] = pats
+    y = y.reshape(T, E)
+    steps = np.array([1.0, 0.37, 3.0e-3, 17.25, 2.0 ** -10, 1.0 / 3.0, 123.456, 2.0 ** -23], np.float32)
+    N = len(steps)
+    t = binding.Tpq(N, E)
+    half_range = (steps * np.float32(7.5)).astype(np.float32)          # R = 2 * 7.5 s = 15 s
+    M = np.repeat(half_range[:, None], E, axis=1)
+    t.set_ranges(-M, M, np.ones(N, np.int64))
+    t.set_features([])
+    s, inv = t.get_scales()
+    os_, oinv = orc.params((2 * M).astype(np.float32))
+    assert gu.bits_equal(s, os_) and gu.bits_equal(inv, oinv)
+    t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+    d = gu.dev_bf16(y)
+    P = t.payload_bytes(T)
+    for i in range(N):
+        whole, view = gu.guarded(P)
+        t.quantize_pack(i, d.data_ptr(), T, view.data_ptr(), P)
+        torch.cuda.synchronize()
+        assert np.array_equal(view.cpu().numpy(), orc.quantize_pack(y, np.zeros(0, np.int32), inv[i])), i
+        assert gu.guards_intact(whole, P)
+    t.close()
+
+
+@pytest.mark.parametrize("path", [binding.PATH_GENERIC, binding.PATH_TILED])
+def test_quantiser_product_is_rounded_before_the_integer_rounding(path):
+    """Searched (x, 1/s) pairs whose float32 product is an exact tie although the exact
+    product is not: a fused multiply-add in the kernel would give a different code."""
+    orc = oracle.c()
+    rng = np.random.default_rng(11)
+    E = 256
+    xs, invs = [], []
+    pats = finite_bf16_patterns()
+    from util import bf16_value
+    vals = bf16_value(pats)
+    cand = pats[(vals > 0.9) & (vals < 1.2)]
+    while len(xs) < E:
+        xb = int(cand[rng.integers(len(cand))])
+        x = float(bf16_value(np.array([xb], np.uint16))[0])
+        half = rng.integers(0, 7) + 0.5
+        i0 = np.float32(half / x)
+        for c in (np.nextafter(i0, np.float32(0)), i0, np.nextafter(i0, np.float32(10))):
+            exact = np.float64(x) * np.float64(c)
+            if float(np.float32(exact)) == half and exact != half:
+                xs.append(xb)
+                invs.append(np.float32(c))
+                break
+    xs = np.array(xs[:E], np.uint16)
+    invs = np.array(invs[:E], np.float32)
+    # ranges that reproduce these reciprocals exactly are not guaranteed; install steps s with fl(1/s) == inv
+    s = (np.float32(1.0) / invs).astype(np.float32)
+    keep = (np.float32(1.0) / s).astype(np.float32) == invs
+    assert keep.sum() > E // 4
+    R = (s * np.float32(15.0)).astype(np.float32)
+    ok = (R / np.float32(15.0)).astype(np.float32) == s
+    keep &= ok
+    assert keep.sum() > E // 8
+    M = np.where(keep, R / 2, 1.0).astype(np.float32)[None, :]
+    t = binding.Tpq(1, E)
+    t.set_ranges(-M, M, np.ones(1, np.int64))
+    t.set_features([])
+    gs, ginv = t.get_scales()
+    assert np.array_equal(ginv[0][keep], invs[keep])
+    t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+    y = np.tile(xs[None, :], (4, 1))
+    d = gu.dev_bf16(y)
+    P = t.payload_bytes(4)
+    whole, view = gu.guarded(P)
+    t.quantize_pack(0, d.data_ptr(), 4, view.data_ptr(), P)
+    torch.cuda.synchronize()
+    want = orc.quantize_pack(y, np.zeros(0, np.int32), ginv[0])
+    assert np.array_equal(view.cpu().numpy(), want)
+    # and those codes are the tie-to-even ones, not the fused ones
+    codes, _ = oracle.oracle_np.unpack(want, 4, E, 0)
+    assert np.all(codes[0][keep] % 2 == 0)
+    t.close()
+
+
+def test_selected_features_pass_every_pattern_through():
+    """All 65 536 BF16 patterns (NaNs, signed zeros, subnormals) in selected columns arrive unchanged."""
+    E, T = 64, 1024
+    pats = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    y = np.zeros((T, E), np.uint16)
+    hp = list(range(8, 16)) + list(range(40, 48))
+    y[:, 8:16] = pats[: T * 8].reshape(T, 8)
+    y[:, 40:48] = pats[:: -1][: T * 8].reshape(T, 8)
+    for off in (0, 8192 * 4):
+        yy = y.copy()
+        yy[:, 8:16] = np.roll(pats, -off)[: T * 8].reshape(T, 8)
+        t = binding.Tpq(1, E)
+        M = np.ones((1, E), np.float32)
+        t.set_ranges(-M, M, np.ones(1, np.int64))
+        t.set_features(hp)
+        for path in (binding.PATH_GENERIC, binding.PATH_TILED):
+            t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+            d = gu.dev_bf16(yy)
+            P = t.payload_bytes(T)
+            whole, view = gu.guarded(P)
+            t.quantize_pack(0, d.data_ptr(), T, view.data_ptr(), P)
+            torch.cuda.synchronize()
+            got = view.cpu().numpy()
+            lpb = oracle.c().lp_bytes(T, E, 16)
+            assert np.array_equal(got[lpb:].view(np.uint16).reshape(T, 16), yy[:, hp])
+        t.close()
+
+
+def test_calibration_batching_and_resume():
+    """One call with n sequences == n calls; state survives get_state / set_state bit for bit."""
+    w = _workload(2, 8, 256, 5, calib=(6, 40))
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, scale=scale) for i in range(2)]
+    a = binding.Tpq(2, 256)
+    m, M = gu.calibrate_both(a, cal)
+    b = binding.Tpq(2, 256)
+    gu.calibrate_both(b, cal, chunks=[1, 2, 3])
+    assert all(gu.bits_equal(x, y) for x, y in zip(a.get_ranges(with_R=False), b.get_ranges(with_R=False)))
+    assert gu.bits_equal(a.get_ranges(with_R=False)[0], m)
+    # resume: first 2 sequences, checkpoint, restore in a fresh context, fold the other 4
+    c = binding.Tpq(2, 256)
+    gu.calibrate_both(c, [x[:2] for x in cal])
+    blob = c.get_state()
+    d = binding.Tpq(2, 256)
+    d.set_state(blob)
+    for i in range(2):
+        dd = gu.dev_bf16(cal[i][2:])
+        d.calibrate_ranges(i, dd.data_ptr(), 4, 40)
+    torch.cuda.synchronize()
+    assert all(gu.bits_equal(x, y) for x, y in zip(a.get_ranges(with_R=False), d.get_ranges(with_R=False)))
+    # a state with a feature set restores the set and the steps
+    hp = a.select_features(-1)
+    e = binding.Tpq(2, 256)
+    e.set_state(a.get_state())
+    assert e.get_features().tolist() == hp.tolist()
+    assert all(gu.bits_equal(x, y) for x, y in zip(a.get_scales(), e.get_scales()))
+    for t in (a, b, c, d, e):
+        t.close()
+
+
+def test_calibration_prefill_sized_sequences():
+    """Several row splits and feature chunks of the tiled extremes kernel, and the generic one."""
+    orc = oracle.c()
+    for (n_seq, S, E) in [(3, 2048, 4608), (2, 517, 520), (2, 300, 1001)]:
+        w = synth.Workload("c", 1, 1, E, 0.7, 5, 20.0, 200.0, n_seq, S, 4000 + E)
+        cal = synth.calibration_np(w, 0)
+        t = binding.Tpq(1, E)
+        m, M = gu.calibrate_both(t, [cal])
+        gm, gM = t.get_ranges(with_R=False)
+        assert gu.bits_equal(gm, m) and gu.bits_equal(gM, M)
+        t.close()
+
+
+def test_signed_zero_and_infinity_extremes():
+    t = binding.Tpq(1, 8)
+    y = np.zeros((1, 4, 8), np.uint16)
+    y[0, :, 0] = [0x0000, 0x8000, 0x0000, 0x8000]          # +0 and -0: min -0, max +0
+    y[0, :, 1] = [0x7F80, 0x3F80, 0xFF80, 0x0000]          # +inf, 1, -inf, 0
+    y[0, :, 2] = [0x0001, 0x8001, 0x0000, 0x8000]          # subnormals
+    m, M = gu.calibrate_both(t, [y])
+    gm, gM = t.get_ranges(with_R=False)
+    assert gu.bits_equal(gm, m) and gu.bits_equal(gM, M)
+    assert gm.view(np.uint32)[0, 0] == 0x80000000 and gM.view(np.uint32)[0, 0] == 0
+    t.close()
+
+
+def test_llama_prefill_full_size():
+    """BASELINE config 2 at full size (N=4, 2048 x 5120), the launch configuration the benchmark times."""
+    w = synth.WORKLOADS["llama13b_prefill"]
+    wc = synth.Workload(w.name, w.n_shards, w.tokens, w.features, w.sd, w.n_outliers, w.outlier_lo, w.outlier_hi,
+                        3, 256, w.seed)
+    _full_pipeline(wc, -1, binding.PATH_AUTO)
+
+
+def test_large_config_sampled_rows():
+    """BASELINE config 5 shape (E = 8192, k = 128) at N = 16 and T = 2048 (the full 8192 rows need
+    2 GB per shard set; rows are independent, so fewer rows exercise the same launch shape).
+    Payload rows and output rows are compared with the oracle on sampled rows."""
+    orc = oracle.c()
+    w = synth.WORKLOADS["large"]
+    N, E, T = w.n_shards, w.features, 2048
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E)
+    cal = [synth.calibration_np(w, i, n_seq=2, tokens=64, scale=scale) for i in range(N)]
+    gu.calibrate_both(t, cal)
+    hp = t.select_features(-1)
+    k = len(hp)
+    assert k == 128
+    s, inv = t.get_scales()
+    P = t.payload_bytes(T)
+    L = E - k
+    lpb = orc.lp_bytes(T, E, k)
+    ys = [synth.activations_torch(w, i, T, "cuda", scale=scale) for i in range(N)]
+    bufs = []
+    for i in range(N):
+        whole, view = gu.guarded(P)
+        t.quantize_pack(i, ys[i].data_ptr(), T, view.data_ptr(), P)
+        bufs.append((whole, view))
+    out = torch.empty((T, E), dtype=torch.float32, device="cuda")
+    t.dequant_reduce([v.data_ptr() for _, v in bufs], T, out.data_ptr(), binding.TPQ_OUT_FP32)
+    outb = torch.empty((T, E), dtype=torch.bfloat16, device="cuda")
+    t.dequant_reduce([v.data_ptr() for _, v in bufs], T, outb.data_ptr(), binding.TPQ_OUT_BF16)
+    torch.cuda.synchronize()
+    assert t.device_status() == 0
+    rows = sorted(set([0, 1, T - 1, T - 2] + np.random.default_rng(0).integers(0, T, 28).tolist()))
+    host = [v.cpu().numpy() for _, v in bufs]
+    for whole, _ in bufs:
+        assert gu.guards_intact(whole, P)
+    for r in rows:
+        row_payloads = []
+        for i in range(N):
+            y_row = ys[i][r: r + 1].view(torch.int16).cpu().numpy().view(np.uint16)
+            want = orc.quantize_pack(y_row, hp, inv[i])                  # T = 1 payload of this row
+            got_lp = host[i][r * L // 2: (r + 1) * L // 2]
+            got_hp = host[i][lpb + r * k * 2: lpb + (r + 1) * k * 2]
+            assert np.array_equal(got_lp, want[: L // 2]), (r, i)
+            assert np.array_equal(got_hp, want[orc.lp_bytes(1, E, k):]), (r, i)
+            row_payloads.append(want)
+        ref, chain = orc.dequant_reduce(row_payloads, 1, E, hp, s)
+        abs_sum = gu.term_abs_sum(row_payloads, 1, E, hp, s)
+        o32 = out[r: r + 1].cpu().numpy()
+        ok, _ = gu.check_fp32(o32, ref, abs_sum, N)
+        assert ok, r
+        assert gu.bits_equal(o32, chain)
+        ob = outb[r: r + 1].view(torch.int16).cpu().numpy().view(np.uint16)
+        ok, _ = gu.check_bf16(ob, ref, abs_sum, N)
+        assert ok, r
+    t.close()
