@@ -57,6 +57,7 @@ class COracle:
         L.tpqo_lp_bytes.restype = i64
         L.tpqo_payload_bytes.argtypes = [i64, i64, i64]
         L.tpqo_payload_bytes.restype = i64
+        L.tpqo_slot_order.argtypes = [i64, i32p, i64, i32p]
         L.tpqo_quantize_one.argtypes = [ctypes.c_uint16, f32]
         L.tpqo_quantize_one.restype = ctypes.c_int
         L.tpqo_quantize_pack.argtypes = [u16p, i64, i64, i64, i32p, i64, f32p, u8p]
@@ -120,6 +121,15 @@ class COracle:
 
     def payload_bytes(self, T: int, E: int, k: int) -> int:
         return int(self.lib.tpqo_payload_bytes(T, E, k))
+
+    def lp_index(self, E: int, hp_idx) -> np.ndarray:
+        """Feature held by each code slot (the payload's slot order)."""
+        hp = np.ascontiguousarray(hp_idx, dtype=np.int32)
+        k = hp.shape[0]
+        out = np.empty(max(E - k, 1), np.int32)
+        hp_arg = hp if k else np.zeros(1, np.int32)
+        self.lib.tpqo_slot_order(E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(out, ctypes.c_int32))
+        return out[: E - k].copy()
 
     def quantize_one(self, x_bits: int, inv_s: float) -> int:
         return int(self.lib.tpqo_quantize_one(ctypes.c_uint16(int(x_bits)), ctypes.c_float(inv_s)))

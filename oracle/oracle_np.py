@@ -110,9 +110,19 @@ def params(R: np.ndarray):
 
 # ------------------------------------------------------------------ compression
 def lp_index(E: int, hp_idx: np.ndarray) -> np.ndarray:
-    keep = np.ones(E, dtype=bool)
-    keep[np.asarray(hp_idx, dtype=np.int64)] = False
-    return np.nonzero(keep)[0].astype(np.int32)
+    """Feature held by each of the L = E-k code slots of a token ("hole filling"):
+    slot c holds feature c unless c is selected; the selected features below L are
+    filled, in ascending order, with the unselected features at or above L."""
+    hp = np.asarray(hp_idx, dtype=np.int64)
+    L = E - len(hp)
+    sel = np.zeros(E, dtype=bool)
+    sel[hp] = True
+    order = np.arange(L, dtype=np.int32)
+    holes = np.nonzero(sel[:L])[0]
+    fillers = L + np.nonzero(~sel[L:])[0]
+    assert len(holes) == len(fillers)
+    order[holes] = fillers
+    return order
 
 
 def quantize_codes(y_bits: np.ndarray, inv_s: np.ndarray) -> np.ndarray:

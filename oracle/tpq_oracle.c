@@ -201,8 +201,32 @@ void tpqo_params(const float *R, int64_t n, float *s, float *inv_s)
 
 /* Section 4 counts (E-k) 4-bit codes and k BF16 values per token.
  * Layout (ours; the paper gives only the count): one flat stream of 4-bit
- * codes for all T tokens in (token, compacted feature) order, low nibble
- * first, zero padded to a multiple of 16 bytes; then T x k BF16 values. */
+ * codes for all T tokens in (token, slot) order, low nibble first, zero padded
+ * to a multiple of 16 bytes; then T x k BF16 values (selected features
+ * ascending).
+ *
+ * Slot order of the L = E-k codes of a token ("hole filling"): slot c holds
+ * feature c, unless feature c is a selected one; the selected features below L
+ * ("holes", ascending) are filled, in order, with the unselected features
+ * at or above L (ascending).  There are equally many of both, so every slot is
+ * used and most features keep their own index as slot. */
+void tpqo_slot_order(int64_t E, const int32_t *hp_idx, int64_t k, int32_t *slot_feature /* [E-k] */)
+{
+    int64_t L = E - k;
+    unsigned char *sel = (unsigned char *)calloc((size_t)(E > 0 ? E : 1), 1);
+    for (int64_t h = 0; h < k; ++h) sel[hp_idx[h]] = 1;
+    int64_t next_filler = L;          /* next candidate feature at or above L */
+    for (int64_t c = 0; c < L; ++c) {
+        if (!sel[c]) {
+            slot_feature[c] = (int32_t)c;
+        } else {
+            while (sel[next_filler]) ++next_filler;
+            slot_feature[c] = (int32_t)next_filler++;
+        }
+    }
+    free(sel);
+}
+
 int64_t tpqo_lp_bytes(int64_t T, int64_t E, int64_t k)
 {
     int64_t nib = T * (E - k);
@@ -243,12 +267,7 @@ void tpqo_quantize_pack(const uint16_t *y, int64_t T, int64_t E, int64_t stride,
     int64_t L = E - k;
     int64_t lp_bytes = tpqo_lp_bytes(T, E, k);
     int32_t *lp_idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L > 0 ? L : 1));
-    {
-        int64_t h = 0, c = 0;
-        for (int64_t j = 0; j < E; ++j) {
-            if (h < k && hp_idx[h] == j) ++h; else lp_idx[c++] = (int32_t)j;
-        }
-    }
+    tpqo_slot_order(E, hp_idx, k, lp_idx);      /* lp_idx[c] = feature held by slot c */
     memset(payload, 0, (size_t)lp_bytes);
     uint16_t *hp = (uint16_t *)(payload + lp_bytes);
     /* rows are independent; codes of two rows can share a byte only when L is
@@ -291,11 +310,11 @@ void tpqo_dequant_reduce(const uint8_t *const *payloads, int64_t N, int64_t T,
     int64_t lp_bytes = tpqo_lp_bytes(T, E, k);
     int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)E); /* >=0: code slot c; <0: -(h+1) */
     {
-        int64_t h = 0, c = 0;
-        for (int64_t j = 0; j < E; ++j) {
-            if (h < k && hp_idx[h] == j) { pos[j] = -(int32_t)(h + 1); ++h; }
-            else pos[j] = (int32_t)c++;
-        }
+        int32_t *slot_feature = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L > 0 ? L : 1));
+        tpqo_slot_order(E, hp_idx, k, slot_feature);
+        for (int64_t c = 0; c < L; ++c) pos[slot_feature[c]] = (int32_t)c;
+        for (int64_t h = 0; h < k; ++h) pos[hp_idx[h]] = -(int32_t)(h + 1);
+        free(slot_feature);
     }
 #pragma omp parallel for schedule(static)
     for (int64_t t = 0; t < T; ++t) {

@@ -135,17 +135,24 @@ __global__ void __launch_bounds__(128) dequant_tiled(const DQParams p)
                     }
                 }
             }
-            uint32_t lo[R][NC], hi[R][NC];
+            uint32_t lo[R][NC], hi[R][NC], hv[R][NC];
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
                 for (int i = 0; i < NC; ++i) {
                     lo[r][i] = 0u;
                     hi[r][i] = 0u;
+                    hv[r][i] = 0u;
                     if (t0 + r < p.T && i0 + i < p.N) {
                         const uint32_t *w = reinterpret_cast<const uint32_t *>(p.pl[i0 + i]) + (t0 + r) * L8 + wbase;
                         if (need_lo) lo[r][i] = __ldcs(w);
                         if (need_hi) hi[r][i] = __ldcs(w + 1);
+                        if (mask) {  // the first two selected features' values travel with the codes
+                            const uint16_t *hp = reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + p.lp_bytes) +
+                                                 (t0 + r) * p.k + hb;
+                            hv[r][i] = __ldcs(hp);
+                            if (n_lp < 7) hv[r][i] |= (uint32_t)__ldcs(hp + 1) << 16;
+                        }
                     }
                 }
 #pragma unroll
@@ -169,8 +176,13 @@ __global__ void __launch_bounds__(128) dequant_tiled(const DQParams p)
                             int h = 0;
 #pragma unroll
                             for (int n = 0; n < 8; ++n)
-                                if (mask & (1u << n))
-                                    acc[r][n] = __fadd_rn(acc[r][n], __uint_as_float((uint32_t)__ldcs(hp + h++) << 16));
+                                if (mask & (1u << n)) {
+                                    const uint32_t bits = (h == 0)   ? (hv[r][i] << 16)
+                                                          : (h == 1) ? (hv[r][i] & 0xFFFF0000u)
+                                                                     : ((uint32_t)__ldcs(hp + h) << 16);
+                                    acc[r][n] = __fadd_rn(acc[r][n], __uint_as_float(bits));
+                                    ++h;
+                                }
                         }
                     }
                 }
@@ -193,6 +205,278 @@ __global__ void __launch_bounds__(128) dequant_tiled(const DQParams p)
                     __stcs(o, make_uint4(w[0], w[1], w[2], w[3]));
                 }
             }
+        }
+    }
+}
+
+
+// ----------------------------------------------------------------------------------------------
+// Row kernel for N <= 8 devices (E, k, output stride multiples of 8; E/8 <= MAXT consumer threads).
+//
+// One persistent block per SM; a producer warp streams groups of G rows of all N payloads (code rows
+// and BF16 rows) into a ring of shared-memory stages with 1-D bulk asynchronous copies, completion on
+// "full" mbarriers; consumer warps release a stage through an "empty" mbarrier, so there is no
+// block-wide barrier in the loop.  Thread <-> 8 adjacent output features for every row: the N x 8
+// steps live in registers for the life of the block, pre-scaled by the power of 16 of the position at
+// which the code is decoded (see decode8), so each code costs one logic op, one subtract, one FMA.
+// G is a multiple of 4/gcd(4, (E-k)/8) so that every stage starts 16-byte aligned in the code stream.
+// ----------------------------------------------------------------------------------------------
+constexpr int DR_WAIT_LIMIT = 1 << 22;
+
+struct DRLayout {
+    size_t lp_stage, hp_stage, stage, bars, total;
+};
+__host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int nstage)
+{
+    DRLayout l;
+    l.lp_stage = (((size_t)G * (E - k) / 2) + 4 + 15) & ~(size_t)15;  // + one spare word: w[1] is read unconditionally
+    l.hp_stage = (size_t)G * k * 2;
+    l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
+    l.bars = (size_t)nstage * l.stage;
+    l.total = l.bars + (size_t)nstage * 16;
+    return l;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int i = 0; i < DR_WAIT_LIMIT; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// 8 two's-complement codes of `raw` times their steps, accumulated.  The codes are decoded in place:
+// (x & 0xF << 4n) | 0x4B000000 is the float 2^23 + (code+8) 16^n; subtracting 2^23 + 8*16^n leaves
+// code * 16^n exactly, and the step was pre-divided by 16^n (an exact scaling), so
+// fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 5..7 use raw >> 20.
+// Subtractions and FMAs run two at a time (f32x2), one binary32 rounding per element as before.
+__device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
+
+__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4])
+{
+    const uint32_t xa = raw ^ 0x88888888u;
+    const uint32_t xb = xa >> 20;
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const int n0 = 2 * h, n1 = 2 * h + 1;
+        const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
+        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | 0x4B000000u);
+        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | 0x4B000000u);
+        const float c0 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n0))));
+        const float c1 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n1))));
+        const float2 d = __fadd2_rn(make_float2(f0, f1), make_float2(c0, c1));
+        acc[h] = __ffma2_rn(d, sc[h], acc[h]);
+    }
+}
+
+struct DRParams {
+    DQParams q;
+    const int32_t *hp_idx;
+    int G, nstage;
+    int64_t ngroups;
+    int *status;
+};
+
+template <bool FP32OUT>
+__device__ __forceinline__ void store_one(void *out, int64_t off, float v)
+{
+    if (FP32OUT)
+        static_cast<float *>(out)[off] = v;
+    else
+        static_cast<__nv_bfloat16 *>(out)[off] = __float2bfloat16_rn(v);
+}
+
+template <int NMAX, int MAXT, bool FP32OUT>
+__global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    const DQParams &p = pp.q;
+    const int tid = threadIdx.x;
+    const int NT = blockDim.x - 32;  // consumer threads
+    const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;
+    const int E8 = E >> 3, L8 = (E - k) >> 3;
+    const DRLayout lay = dr_layout(N, E, k, G, nstage);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
+    uint64_t *empty = full + nstage;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), NT / 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (tid >= NT) {
+        // ---------------- producer warp: one lane streams the row groups
+        if (tid == NT) {
+            int st = 0;
+            uint32_t parity = 1;  // parity of the "empty" phase to wait for: ((it / nstage) - 1) & 1
+            for (int it = 0;; ++it) {
+                const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+                if (gi >= pp.ngroups) break;
+                if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
+                    atomicExch(pp.status, (int)TPQ_ERR_TIMEOUT);
+                    break;
+                }
+                const int64_t t0 = gi * G;
+                const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+                const uint32_t lp_bytes = (uint32_t)((((size_t)rows * (E - k) / 2) + 15) & ~(size_t)15);
+                const uint32_t hp_bytes = (uint32_t)rows * k * 2u;
+                const uint32_t bar = smem_u32(&full[st]);
+                uint8_t *stage = smem + (size_t)st * lay.stage;
+                mbar_expect_tx(bar, (uint32_t)N * (lp_bytes + hp_bytes));
+                for (int i = 0; i < N; ++i) {
+                    bulk_g2s(smem_u32(stage + (size_t)i * lay.lp_stage), p.pl[i] + t0 * ((E - k) / 2), lp_bytes, bar);
+                    if (hp_bytes)
+                        bulk_g2s(smem_u32(stage + (size_t)N * lay.lp_stage + (size_t)i * lay.hp_stage),
+                                 p.pl[i] + p.lp_bytes + t0 * k * 2, hp_bytes, bar);
+                }
+                if (++st == nstage) {
+                    st = 0;
+                    parity ^= 1u;
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers
+    // Thread <-> output features 8g .. 8g+7.  Its n_lp quantised ones are adjacent in the code stream
+    // (slots c0 ..); slot c belongs to feature 8g + ofs(c).  The codes are NOT moved to their feature
+    // positions: the step of slot c is the step of feature 8g + ofs(c), and the row store puts slot c
+    // where it belongs.  Selected features are summed and stored by the threads h < k below.
+    const int g = tid;
+    const bool live = g < E8;
+    uint32_t mask = 0;
+    int hb = 0;
+    if (live) {
+        const uint32_t gd = __ldg(p.grp + g);
+        mask = gd & 0xFFu;
+        hb = (int)(gd >> 8);
+    }
+    const int c0 = 8 * g - hb;
+    const int n_lp = 8 - __popc(mask);
+    const int sh = (c0 & 7) * 4;
+    const int wbase = c0 >> 3;
+    uint32_t ofs_pack = 0;
+    {
+        int c = 0;
+#pragma unroll
+        for (int n = 0; n < 8; ++n)
+            if (!(mask & (1u << n))) ofs_pack |= (uint32_t)n << (3 * c++);
+    }
+
+    float2 sc[NMAX][4];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) {
+        float v[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            v[c] = 0.0f;
+            if (live && i < N && c < n_lp)
+                v[c] = __ldg(p.s_k + (size_t)i * E + 8 * g + ((ofs_pack >> (3 * c)) & 7)) *
+                       (1.0f / (float)(1 << (4 * dq_pos(c))));
+        }
+#pragma unroll
+        for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(v[2 * h], v[2 * h + 1]);
+    }
+    const int my_hp = (tid < k) ? __ldg(pp.hp_idx + tid) : 0;
+
+    int st = 0;
+    uint32_t parity = 0;  // (it / nstage) & 1
+    for (int it = 0;; ++it) {
+        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+        if (gi >= pp.ngroups) break;
+        if (!mbar_wait(smem_u32(&full[st]), parity)) {
+            atomicExch(pp.status, (int)TPQ_ERR_TIMEOUT);
+            break;
+        }
+        const int64_t t0 = gi * G;
+        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+        const uint8_t *stage = smem + (size_t)st * lay.stage;
+        if (live) {
+            for (int r = 0; r < rows; ++r) {
+                float2 acc[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
+#pragma unroll
+                for (int i = 0; i < NMAX; ++i) {
+                    if (i < N) {
+                        const uint32_t *w =
+                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage) + r * L8 + wbase;
+                        decode8(__funnelshift_r(w[0], w[1], sh), sc[i], acc);
+                    }
+                }
+                const int64_t o = (t0 + r) * p.out_stride + 8 * g;
+                if (mask == 0) {
+                    if (FP32OUT) {
+                        float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.out) + o);
+                        __stcs(dst, make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
+                        __stcs(dst + 1, make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y));
+                    } else {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) {
+                            __nv_bfloat162 b = __floats2bfloat162_rn(acc[h].x, acc[h].y);
+                            w[h] = *reinterpret_cast<uint32_t *>(&b);
+                        }
+                        __stcs(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.out) + o),
+                               make_uint4(w[0], w[1], w[2], w[3]));
+                    }
+                } else {
+                    const float a8[8] = {acc[0].x, acc[0].y, acc[1].x, acc[1].y, acc[2].x, acc[2].y, acc[3].x, acc[3].y};
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        if (c < n_lp) store_one<FP32OUT>(p.out, o + ((ofs_pack >> (3 * c)) & 7), a8[c]);
+                }
+            }
+        }
+        // selected features: sum of the BF16 values, devices ascending
+        for (int h = tid; h < k; h += NT) {
+            const int j = (h == tid) ? my_hp : __ldg(pp.hp_idx + h);
+            const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
+            for (int r = 0; r < rows; ++r) {
+                float acc = 0.0f;
+                for (int i = 0; i < N; ++i)
+                    acc = __fadd_rn(acc, __uint_as_float((uint32_t)hp[(size_t)i * (lay.hp_stage / 2) + r * k + h] << 16));
+                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + j, acc);
+            }
+        }
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
+        if (++st == nstage) {
+            st = 0;
+            parity ^= 1u;
         }
     }
 }
@@ -230,11 +514,68 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
     return cudaGetLastError();
 }
 
+namespace {
+
+template <int NMAX, int MAXT>
+cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads, size_t smem, cudaStream_t st)
+{
+    cudaError_t e;
+    if (fp32_out) {
+        e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) dequant_rows<NMAX, MAXT, true><<<grid, threads, smem, st>>>(pp);
+    } else {
+        e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e == cudaSuccess) dequant_rows<NMAX, MAXT, false><<<grid, threads, smem, st>>>(pp);
+    }
+    return e;
+}
+
+// Row kernel geometry; returns false if the shape does not admit it.
+bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *ngroups_out, int *grid_out)
+{
+    const int N = c->N, E = c->E, k = c->k;
+    const int E8 = E / 8, L8 = (E - k) / 8;
+    if (N > 8 || E - k < 8) return false;
+    if (E8 > (N <= 4 ? 768 : 576)) return false;
+    int g0 = 4;
+    if (L8 % 4 == 0) g0 = 1;
+    else if (L8 % 2 == 0) g0 = 2;
+    int G = g0;
+    while (G < 2) G += g0;
+    if (dr_layout(N, E, k, G, 2).total > (size_t)c->smem_optin) return false;
+    const int64_t ngroups = (T + G - 1) / G;
+    const int grid = (int)(ngroups < c->sm_count ? ngroups : c->sm_count);
+    const int64_t per_block = (ngroups + grid - 1) / grid;
+    int nstage = (int)(per_block < 8 ? per_block : 8);
+    if (nstage < 2) nstage = 2;
+    while (nstage > 2 && dr_layout(N, E, k, G, nstage).total > (size_t)c->smem_optin) --nstage;
+    *G_out = G; *nstage_out = nstage; *ngroups_out = ngroups; *grid_out = grid;
+    return true;
+}
+
+}  // namespace
+
 cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out, int fp32_out,
                                      int64_t out_stride, cudaStream_t st, int64_t *launches)
 {
     DQParams p;
     fill_params(p, c, payloads, T, out, out_stride);
+    {
+        DRParams pp;
+        int grid = 0;
+        if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.ngroups, &grid)) {
+            pp.q = p;
+            pp.hp_idx = c->t.hp_idx;
+            pp.status = c->t.status;
+            const size_t smem = dr_layout(c->N, c->E, c->k, pp.G, pp.nstage).total;
+            const int threads = ((c->E / 8 + 31) / 32) * 32 + 32;
+            cudaError_t e = (c->N <= 4) ? launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st)
+                                        : launch_rows<8, 576>(pp, fp32_out, grid, threads, smem, st);
+            if (e != cudaSuccess) return e;
+            ++*launches;
+            return cudaGetLastError();
+        }
+    }
     const int E8 = c->E / 8;
     const int strips = (E8 + 127) / 128;
     constexpr int R = 4;

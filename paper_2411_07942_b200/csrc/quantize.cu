@@ -82,10 +82,14 @@ struct QPParams {
     const float *inv_s;    // this device's [E]
     const uint32_t *grp;   // [E/8]
     const int32_t *lp_idx; // [E-k]
+    const int32_t *hp_idx; // [k]
     uint32_t *lp_out;
     int64_t lp_words;      // words of the code section, padding included
     uint32_t *hp_out;      // as 32-bit words (k even)
     int *status;
+#ifdef TPQ_TRACE
+    long long *trace;
+#endif
 };
 
 // Dynamic shared memory layout (byte offsets, every section 16-byte aligned).
@@ -97,7 +101,7 @@ __host__ __device__ inline QPLayout qp_layout(int E, int k, int G, int nstage)
     QPLayout l;
     l.ring = 0;
     l.nib = (size_t)nstage * G * E * 2;
-    l.hpb = l.nib + (((size_t)2 * G * (E / 8 + 1) * 4 + 15) & ~(size_t)15);
+    l.hpb = l.nib + (((size_t)2 * G * (E / 8 + 2) * 4 + 15) & ~(size_t)15);
     l.bars = l.hpb + (((size_t)2 * G * k * 2 + 15) & ~(size_t)15);
     l.total = l.bars + (size_t)nstage * 8;
     return l;
@@ -143,17 +147,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
 // 8 BF16 (one uint4) -> 8 two's-complement nibbles in feature order.
 // code + 0x4B400000 sits in the bits of fl(u + 1.5*2^23); shifted copies are summed with one
 // shift-add each and the constant parts are removed at the end (offset-binary -> two's complement).
-__device__ __forceinline__ uint32_t quant8(const uint4 v, const float (&inv)[8])
+// Products and magic adds run two at a time (f32x2); each is still one binary32 rounding per element.
+__device__ __forceinline__ uint32_t quant8(const uint4 v, const float2 (&inv)[4])
 {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
     uint32_t acc = 0;
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
-        const uint32_t bits = (n & 1) ? (w[n >> 1] & 0xFFFF0000u) : (w[n >> 1] << 16);
-        float u = __fmul_rn(__uint_as_float(bits), inv[n]);
-        u = fminf(fmaxf(u, -8.0f), 7.0f);
-        const uint32_t r = __float_as_uint(__fadd_rn(u, 12582912.0f));
-        acc += r << (4 * n);
+    for (int i = 0; i < 4; ++i) {
+        float2 u = __fmul2_rn(make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xFFFF0000u)), inv[i]);
+        u.x = fminf(fmaxf(u.x, -8.0f), 7.0f);
+        u.y = fminf(fmaxf(u.y, -8.0f), 7.0f);
+        const float2 r = __fadd2_rn(u, make_float2(12582912.0f, 12582912.0f));
+        acc += __float_as_uint(r.x) << (8 * i);
+        acc += __float_as_uint(r.y) << (8 * i + 4);
     }
     // sum_n (0x4B400000 << 4n) mod 2^32
     constexpr uint32_t K0 = 0x4B400000u + (0x4B400000u << 4) + (0x4B400000u << 8) + (0x4B400000u << 12) +
@@ -161,14 +167,28 @@ __device__ __forceinline__ uint32_t quant8(const uint4 v, const float (&inv)[8])
     return (acc - K0 + 0x88888888u) ^ 0x88888888u;
 }
 
+#ifdef TPQ_TRACE
+static long long *g_trace = nullptr;  // 64 slots per block, globaltimer ns
+__device__ __forceinline__ long long tpq_now()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define TPQ_MARK(slot) do { if (threadIdx.x == 0 && p.trace && (slot) < 64) p.trace[blockIdx.x * 64 + (slot)] = tpq_now(); } while (0)
+#else
+#define TPQ_MARK(slot) do { } while (0)
+#endif
+
 template <int GPT>
 __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
 {
+    TPQ_MARK(0);
     extern __shared__ __align__(128) uint8_t smem[];
     const int tid = threadIdx.x, NT = blockDim.x;
     const int E = p.E, k = p.k, G = p.G, nstage = p.nstage;
     const int E8 = E >> 3, L8 = (E - k) >> 3;
-    const int nib_stride = E8 + 1;
+    const int nib_stride = E8 + 2;
     const uint32_t row_bytes = (uint32_t)E * 2u;
     const uint32_t stage_bytes = (uint32_t)G * row_bytes;
 
@@ -186,11 +206,11 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
+    TPQ_MARK(40);
 
-    auto issue = [&](int64_t it) {
+    auto issue = [&](int it, int st) {  // group blockIdx.x + it*gridDim.x into stage st
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
         if (gi >= p.ngroups) return;
-        const int st = (int)(it % nstage);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
         const uint32_t bar = smem_u32(&bars[st]);
@@ -203,90 +223,109 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
         }
     };
     if (tid == 0)
-        for (int it = 0; it < nstage; ++it) issue(it);
+        for (int it = 0; it < nstage; ++it) issue(it, it);
+    TPQ_MARK(41);
 
-    // per-thread constants (overlap the first copies)
-    float inv[GPT][8];
-    uint32_t gdesc[GPT];
-    int src0[GPT];      // phase 2: source nibble position of output word (tid + a*NT), -1 = none
-    bool contig[GPT];
+    // ---- per-thread constants (their loads overlap the first copies)
+    // phase 1: the reciprocal steps of the thread's 8 features, as four pairs
+    float2 inv[GPT][4];
+    // selected features: thread h < k copies feature my_hp of every row to the BF16 side buffer
+    const int my_hp = (tid < k) ? __ldg(p.hp_idx + tid) : 0;
+    // phase 2: output word wc = tid + a*NT of a row holds the 8 codes whose source features are
+    // lp_idx[8wc .. 8wc+7].  With d = number of selected features skipped so far (0, 1 or 2 inside one
+    // word in all but pathological sets), code c sits at source nibble src0 + c + d: the word is
+    // (W0 & ~(m1|m2)) | (W1 & m1) | (W2 & m2), Wd = the 32-bit window of the code row at nibble src0 + d.
+    int w0[GPT], sh[GPT];
+    uint32_t m1[GPT], m2[GPT];
+    int mode[GPT];  // 0: no word, 1: windows, 2: more than two skipped features, code by code
 #pragma unroll
     for (int a = 0; a < GPT; ++a) {
         const int g = tid + a * NT;
-        gdesc[a] = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
         if (g < E8) {
             const float4 i0 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g));
             const float4 i1 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g + 4));
-            inv[a][0] = i0.x; inv[a][1] = i0.y; inv[a][2] = i0.z; inv[a][3] = i0.w;
-            inv[a][4] = i1.x; inv[a][5] = i1.y; inv[a][6] = i1.z; inv[a][7] = i1.w;
-            gdesc[a] = __ldg(p.grp + g);
-        } else {
-#pragma unroll
-            for (int n = 0; n < 8; ++n) inv[a][n] = 0.0f;
+            inv[a][0] = make_float2(i0.x, i0.y);
+            inv[a][1] = make_float2(i0.z, i0.w);
+            inv[a][2] = make_float2(i1.x, i1.y);
+            inv[a][3] = make_float2(i1.z, i1.w);
         }
-        src0[a] = -1;
-        contig[a] = false;
+        w0[a] = 0; sh[a] = 0; m1[a] = 0; m2[a] = 0; mode[a] = 0;
         if (g < L8) {
-            src0[a] = __ldg(p.lp_idx + 8 * g);
-            contig[a] = (__ldg(p.lp_idx + 8 * g + 7) - src0[a]) == 7;
+            const int4 l0 = __ldg(reinterpret_cast<const int4 *>(p.lp_idx + 8 * g));
+            const int4 l1 = __ldg(reinterpret_cast<const int4 *>(p.lp_idx + 8 * g + 4));
+            const int idx[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
+            w0[a] = idx[0] >> 3;
+            sh[a] = (idx[0] & 7) * 4;
+            mode[a] = (idx[7] - idx[0] - 7 <= 2) ? 1 : 2;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const int d = idx[c] - idx[0] - c;
+                if (d == 1) m1[a] |= 0xFu << (4 * c);
+                if (d == 2) m2[a] |= 0xFu << (4 * c);
+            }
         }
     }
 
-    int64_t it = 0;
+    TPQ_MARK(1);
+    int it = 0, st = 0;       // iteration, its ring stage (it mod nstage, kept without dividing)
+    uint32_t parity = 0;      // (it / nstage) & 1
     for (;; ++it) {
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
         if (gi >= p.ngroups) break;
-        const int st = (int)(it % nstage);
-        const uint32_t parity = (uint32_t)((it / nstage) & 1);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-        const int buf = (int)(it & 1);
+        const int buf = it & 1;
         if (!mbar_wait(smem_u32(&bars[st]), parity)) abort_flag = 1;
+        TPQ_MARK(2 + 3 * (int)it);
 
-        // ---- phase 1: quantise in feature order
+        // ---- phase 1: quantise in feature order; copy the selected features
         const uint4 *stage = reinterpret_cast<const uint4 *>(ring + (size_t)st * stage_bytes);
         uint32_t *nrow = nib + (size_t)buf * G * nib_stride;
         uint16_t *hrow = hpb + (size_t)buf * G * k;
 #pragma unroll
         for (int a = 0; a < GPT; ++a) {
             const int g = tid + a * NT;
-            if (g < E8) {
-                for (int r = 0; r < rows; ++r) {
-                    const uint4 v = stage[r * E8 + g];
-                    nrow[r * nib_stride + g] = quant8(v, inv[a]);
-                    const uint32_t mask = gdesc[a] & 0xFFu;
-                    if (mask) {
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-                        int h = (int)(gdesc[a] >> 8);
-#pragma unroll
-                        for (int n = 0; n < 8; ++n)
-                            if (mask & (1u << n))
-                                hrow[r * k + h++] = (uint16_t)((n & 1) ? (w[n >> 1] >> 16) : (w[n >> 1] & 0xFFFFu));
-                    }
-                }
+            if (g < E8)
+                for (int r = 0; r < rows; ++r) nrow[r * nib_stride + g] = quant8(stage[r * E8 + g], inv[a]);
+        }
+        {
+            const uint16_t *stage16 = reinterpret_cast<const uint16_t *>(stage);
+            for (int h = tid; h < k; h += NT) {
+                const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
+                for (int r = 0; r < rows; ++r) hrow[r * k + h] = stage16[r * E + j];
             }
         }
         __syncthreads();
+        TPQ_MARK(3 + 3 * (int)it);
         if (abort_flag) break;
-        if (tid == 0) issue(it + nstage);  // the stage is free again
+        if (tid == 0) issue(it + nstage, st);  // the stage is free again
 
         // ---- phase 2: squeeze out the selected features, store
 #pragma unroll
         for (int a = 0; a < GPT; ++a) {
             const int wc = tid + a * NT;
-            if (wc < L8) {
+            if (mode[a] != 0) {
                 for (int r = 0; r < rows; ++r) {
-                    const uint32_t *src = nrow + r * nib_stride;
+                    const uint32_t *src = nrow + r * nib_stride + w0[a];
                     uint32_t word;
-                    if (contig[a]) {
-                        const int w0 = src0[a] >> 3;
-                        word = __funnelshift_r(src[w0], src[w0 + 1], (src0[a] & 7) * 4);
+                    if (mode[a] == 1) {
+                        const uint32_t x0 = src[0], x1 = src[1];
+                        const uint32_t W0 = __funnelshift_r(x0, x1, sh[a]);
+                        const uint32_t W1 = __funnelshift_rc(x0, x1, sh[a] + 4);
+                        word = (W0 & ~(m1[a] | m2[a])) | (W1 & m1[a]);
+                        if (m2[a]) {
+                            const uint32_t W2 = (sh[a] == 28) ? __funnelshift_r(x1, src[2], 4)
+                                                              : __funnelshift_rc(x0, x1, sh[a] + 8);
+                            word |= W2 & m2[a];
+                        }
                     } else {
                         word = 0;
 #pragma unroll 1
                         for (int n = 0; n < 8; ++n) {
                             const int j = __ldg(p.lp_idx + 8 * wc + n);
-                            word |= ((src[j >> 3] >> ((j & 7) * 4)) & 0xFu) << (4 * n);
+                            word |= ((nrow[r * nib_stride + (j >> 3)] >> ((j & 7) * 4)) & 0xFu) << (4 * n);
                         }
                     }
                     p.lp_out[(t0 + r) * L8 + wc] = word;
@@ -299,13 +338,18 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
             uint32_t *dst = p.hp_out + t0 * (k / 2);
             for (int a = tid; a < n32; a += NT) dst[a] = h32[a];
         }
+        TPQ_MARK(4 + 3 * (int)it);
+        if (++st == nstage) {
+            st = 0;
+            parity ^= 1u;
+        }
     }
 
     if (abort_flag) {
         // a copy never completed: report, give the copies still in flight a bounded chance to land, leave
         if (tid == 0) {
             atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
-            for (int64_t j = it + 1; j < it + nstage; ++j) {
+            for (int j = it + 1; j < it + nstage; ++j) {
                 if (blockIdx.x + j * (int64_t)gridDim.x >= p.ngroups) break;
                 mbar_wait(smem_u32(&bars[j % nstage]), (uint32_t)((j / nstage) & 1));
             }
@@ -371,9 +415,12 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
     QPParams p;
     const int64_t lpb = tpq_lp_bytes_i(T, E, k);
     p.y = y; p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
-    p.inv_s = c->t.inv_s + (size_t)shard * E; p.grp = c->t.grp; p.lp_idx = c->t.lp_idx;
+    p.inv_s = c->t.inv_s + (size_t)shard * E; p.grp = c->t.grp; p.lp_idx = c->t.lp_idx; p.hp_idx = c->t.hp_idx;
     p.lp_out = reinterpret_cast<uint32_t *>(payload); p.lp_words = lpb / 4;
     p.hp_out = reinterpret_cast<uint32_t *>(payload + lpb); p.status = c->t.status;
+#ifdef TPQ_TRACE
+    p.trace = g_trace;
+#endif
     const size_t smem = qp_smem_bytes(E, k, G, nstage);
 
     cudaError_t e = cudaSuccess;

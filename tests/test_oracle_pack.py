@@ -7,6 +7,30 @@ import pytest
 from util import bf16_bits, finite_bf16_patterns, read_golden
 
 
+def _slot_order_by_definition(E, hp):
+    """The payload's slot order, spelled out independently of the oracle: slot c holds feature c unless
+    c is selected; selected features below L are filled in order with unselected ones from L upwards."""
+    L = E - len(hp)
+    sel = set(hp)
+    spare = [j for j in range(L, E) if j not in sel]
+    out = []
+    for c in range(L):
+        out.append(c if c not in sel else spare.pop(0))
+    assert not spare
+    return out
+
+
+@pytest.mark.parametrize("E,hp", [(8, [1, 6]), (8, []), (8, [6, 7]), (8, [0, 1]), (16, [0, 3, 9, 15]),
+                                  (16, list(range(8))), (16, list(range(8, 16))), (12, [11]), (5, [0, 1, 2, 3, 4])])
+def test_slot_order_definition(corc, norc, E, hp):
+    want = _slot_order_by_definition(E, hp)
+    assert corc.lp_index(E, hp).tolist() == want
+    assert norc.lp_index(E, np.array(hp, np.int64)).tolist() == want
+    # a permutation of the unselected features; most features keep their own index as slot
+    assert sorted(want) == [j for j in range(E) if j not in hp]
+    assert all(want[c] == c for c in range(len(want)) if c not in hp)
+
+
 def _orcs(corc, norc):
     return [("c", corc), ("np", norc)]
 
@@ -53,7 +77,7 @@ def test_roundtrip_and_padding(corc, norc, T, E, k):
     y = bf16_bits(rng.standard_normal((T, E)) * 4)
     hp = np.sort(rng.permutation(E)[:k]).astype(np.int32)
     inv = (1.0 / rng.uniform(0.2, 2.0, E)).astype(np.float32)
-    lp_cols = np.setdiff1d(np.arange(E), hp)
+    lp_cols = _slot_order_by_definition(E, hp.tolist())
     for _, orc in _orcs(corc, norc):
         p = orc.quantize_pack(y, hp, inv)
         codes, hpv = norc.unpack(p, T, E, k)
