@@ -58,178 +58,206 @@ __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
 }
 
 // ----------------------------------------------------------------------------------------------
-// Tiled kernel for E, k and the output stride multiples of 8.
+// Shared pieces of the tiled kernels (E, k and the output stride multiples of 8).
 //
-// Thread <-> 8 adjacent OUTPUT features; block <-> a strip of 8*blockDim.x features; blocks walk
-// row blocks of R rows.  The steps of NC devices for the thread's 8 features live in registers.
-// Because (E-k) is a multiple of 8, the bit offset of the thread's codes inside a 32-bit word of
-// the flat code stream is the same for every row: one (or two) 32-bit loads per device and row
-// plus a funnel shift give its 8 codes; a warp reads 128 contiguous bytes.  Where a selected
-// feature falls inside the thread's 8, the codes are spread around the hole and the BF16 value
-// of every device is added instead.  R*NC independent loads are in flight per thread.
+// In the payload's slot order, output features 8g .. 8g+7 (g < L/8, L = E-k) are the aligned 32-bit
+// word g of every device's code row, so a thread that owns them needs one word per device and row.
+// Slots whose feature is a selected one hold a filler feature's code instead: the thread's step for
+// them is 0, it does not store them, and two small extra jobs complete the row:
+//   - filler feature filler[tau], tau < n_holes, lives in slot hole[tau]: one code per device;
+//   - selected feature hp_idx[h], h < k: the sum of the devices' BF16 values.
 // ----------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t spread_holes(uint32_t raw, uint32_t mask)
+constexpr int DR_WAIT_LIMIT = 1 << 22;
+
+__device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
+
+// 8 two's-complement codes of `raw` times their steps, accumulated.  The codes are decoded in place:
+// (x & 0xF << 4n) | 0x4B000000 is the float 2^23 + (code+8) 16^n; subtracting 2^23 + 8*16^n leaves
+// code * 16^n exactly, and the step was pre-divided by 16^n (an exact scaling), so
+// fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 5..7 use raw >> 20.
+// Subtractions and FMAs run two at a time (f32x2), one binary32 rounding per element as before.
+__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4])
 {
-    // insert a zero nibble at every set position of mask (ascending)
-    while (mask) {
-        const int b = __ffs(mask) - 1;
-        const uint32_t low = (b == 0) ? 0u : (0xFFFFFFFFu >> (32 - 4 * b));
-        raw = (raw & low) | ((raw & ~low) << 4);
-        mask &= mask - 1;
+    const uint32_t xa = raw ^ 0x88888888u;
+    const uint32_t xb = xa >> 20;
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        const int n0 = 2 * h, n1 = 2 * h + 1;
+        const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
+        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | 0x4B000000u);
+        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | 0x4B000000u);
+        const float c0 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n0))));
+        const float c1 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n1))));
+        const float2 d = __fadd2_rn(make_float2(f0, f1), make_float2(c0, c1));
+        acc[h] = __ffma2_rn(d, sc[h], acc[h]);
     }
-    return raw;
 }
 
+// the steps of features 8g .. 8g+7 of device i, pre-divided by the power of 16 of their decode position
+__device__ __forceinline__ void load_steps(const float *s_k_row, int g, float2 (&sc)[4])
+{
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(s_k_row + 8 * g));
+    const float4 b = __ldg(reinterpret_cast<const float4 *>(s_k_row + 8 * g + 4));
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int h = 0; h < 4; ++h)
+        sc[h] = make_float2(v[2 * h] * (1.0f / (float)(1 << (4 * dq_pos(2 * h)))),
+                            v[2 * h + 1] * (1.0f / (float)(1 << (4 * dq_pos(2 * h + 1)))));
+}
+
+template <bool FP32OUT>
+__device__ __forceinline__ void store_one(void *out, int64_t off, float v)
+{
+    if (FP32OUT)
+        static_cast<float *>(out)[off] = v;
+    else
+        static_cast<__nv_bfloat16 *>(out)[off] = __float2bfloat16_rn(v);
+}
+
+// the 8 sums of a thread -> features o .. o+7 of the output row, skipping the selected ones
+template <bool FP32OUT>
+__device__ __forceinline__ void store_group(void *out, int64_t o, const float2 (&acc)[4], uint32_t mask)
+{
+    if (mask == 0) {
+        if (FP32OUT) {
+            float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(out) + o);
+            __stcs(dst, make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
+            __stcs(dst + 1, make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y));
+        } else {
+            uint32_t w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                __nv_bfloat162 b = __floats2bfloat162_rn(acc[h].x, acc[h].y);
+                w[h] = *reinterpret_cast<uint32_t *>(&b);
+            }
+            __stcs(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(out) + o), make_uint4(w[0], w[1], w[2], w[3]));
+        }
+    } else {
+        const float a8[8] = {acc[0].x, acc[0].y, acc[1].x, acc[1].y, acc[2].x, acc[2].y, acc[3].x, acc[3].y};
+#pragma unroll
+        for (int n = 0; n < 8; ++n)
+            if (!(mask & (1u << n))) store_one<FP32OUT>(out, o + n, a8[n]);
+    }
+}
+
+struct DXParams {           // extras shared by the tiled kernels
+    const int32_t *hp_idx;  // [k]
+    const int32_t *hole;    // [n_holes]
+    const int32_t *filler;  // [n_holes]
+    int n_holes;
+    int *status;
+};
+
+// ----------------------------------------------------------------------------------------------
+// Strip kernel (any N): thread <-> 8 adjacent output features, block <-> a strip of 8*blockDim.x
+// features; blocks walk row blocks of R rows with R*NC independent 32-bit loads in flight per thread
+// (a warp reads 128 contiguous bytes).  The steps of NC devices at a time live in registers.
+// Blocks with blockIdx.x == gridDim.x - 1 do the filler and selected features of their rows instead.
+// ----------------------------------------------------------------------------------------------
 template <int NC, int R, bool FP32OUT>
-__global__ void __launch_bounds__(128) dequant_tiled(const DQParams p)
+__global__ void __launch_bounds__(128) dequant_strips(const DQParams p, const DXParams x)
 {
     const int E8 = p.E >> 3, L8 = (p.E - p.k) >> 3;
-    const int g = blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= E8) return;
-    const uint32_t gd = __ldg(p.grp + g);
-    const uint32_t mask = gd & 0xFFu;
-    const int hb = (int)(gd >> 8);
-    const int c0 = 8 * g - hb;              // compacted slot of the group's first code
-    const int n_lp = 8 - __popc(mask);
-    const int sh = (c0 & 7) * 4;
-    const int wbase = c0 >> 3;
-    const bool need_lo = n_lp > 0;
-    const bool need_hi = (c0 & 7) + n_lp > 8;
     const int64_t n_rb = (p.T + R - 1) / R;
-    const bool single = p.N <= NC;
 
-    float sc[NC][8];
+    if (blockIdx.x == gridDim.x - 1) {
+        // ---- extras: one (row, feature) pair per thread step
+        const int64_t L = p.E - p.k;
+        const int per_row = x.n_holes + p.k;
+        for (int64_t rb = blockIdx.y; rb < n_rb; rb += gridDim.y) {
+            const int64_t t0 = rb * R;
+            const int rows = (int)((p.T - t0 < R) ? p.T - t0 : R);
+            for (int a = threadIdx.x; a < rows * per_row; a += blockDim.x) {
+                const int r = a / per_row, e = a - r * per_row;
+                const int64_t t = t0 + r;
+                float acc = 0.0f;
+                int j;
+                if (e < x.n_holes) {
+                    j = __ldg(x.filler + e);
+                    const int slot = __ldg(x.hole + e);
+                    for (int i = 0; i < p.N; ++i) {
+                        const uint32_t w = reinterpret_cast<const uint32_t *>(p.pl[i])[t * (L >> 3) + (slot >> 3)];
+                        const int code = (int)(((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) - 8;
+                        acc = __fmaf_rn((float)code, __ldg(p.s_k + (size_t)i * p.E + j), acc);
+                    }
+                } else {
+                    const int h = e - x.n_holes;
+                    j = __ldg(x.hp_idx + h);
+                    for (int i = 0; i < p.N; ++i) {
+                        const uint16_t v = reinterpret_cast<const uint16_t *>(p.pl[i] + p.lp_bytes)[t * p.k + h];
+                        acc = __fadd_rn(acc, __uint_as_float((uint32_t)v << 16));
+                    }
+                }
+                store_one<FP32OUT>(p.out, t * p.out_stride + j, acc);
+            }
+        }
+        return;
+    }
+
+    const int g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= L8) return;
+    const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
+    const bool single = p.N <= NC;
+    float2 sc[NC][4];
     if (single) {
 #pragma unroll
         for (int i = 0; i < NC; ++i) {
-            if (i < p.N) {
-                const float4 a = __ldg(reinterpret_cast<const float4 *>(p.s_k + (size_t)i * p.E + 8 * g));
-                const float4 b = __ldg(reinterpret_cast<const float4 *>(p.s_k + (size_t)i * p.E + 8 * g + 4));
-                sc[i][0] = a.x; sc[i][1] = a.y; sc[i][2] = a.z; sc[i][3] = a.w;
-                sc[i][4] = b.x; sc[i][5] = b.y; sc[i][6] = b.z; sc[i][7] = b.w;
-            } else {
 #pragma unroll
-                for (int n = 0; n < 8; ++n) sc[i][n] = 0.0f;
-            }
+            for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
+            if (i < p.N) load_steps(p.s_k + (size_t)i * p.E, g, sc[i]);
         }
     }
-
     for (int64_t rb = blockIdx.y; rb < n_rb; rb += gridDim.y) {
         const int64_t t0 = rb * R;
-        float acc[R][8];
+        float2 acc[R][4];
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
-            for (int n = 0; n < 8; ++n) acc[r][n] = 0.0f;
-
+            for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
         for (int i0 = 0; i0 < p.N; i0 += NC) {
             if (!single) {
 #pragma unroll
-                for (int i = 0; i < NC; ++i) {
-                    if (i0 + i < p.N) {
-                        const float4 a = __ldg(reinterpret_cast<const float4 *>(p.s_k + (size_t)(i0 + i) * p.E + 8 * g));
-                        const float4 b =
-                            __ldg(reinterpret_cast<const float4 *>(p.s_k + (size_t)(i0 + i) * p.E + 8 * g + 4));
-                        sc[i][0] = a.x; sc[i][1] = a.y; sc[i][2] = a.z; sc[i][3] = a.w;
-                        sc[i][4] = b.x; sc[i][5] = b.y; sc[i][6] = b.z; sc[i][7] = b.w;
-                    }
-                }
+                for (int i = 0; i < NC; ++i)
+                    if (i0 + i < p.N) load_steps(p.s_k + (size_t)(i0 + i) * p.E, g, sc[i]);
             }
-            uint32_t lo[R][NC], hi[R][NC], hv[R][NC];
+            uint32_t w[R][NC];
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
                 for (int i = 0; i < NC; ++i) {
-                    lo[r][i] = 0u;
-                    hi[r][i] = 0u;
-                    hv[r][i] = 0u;
-                    if (t0 + r < p.T && i0 + i < p.N) {
-                        const uint32_t *w = reinterpret_cast<const uint32_t *>(p.pl[i0 + i]) + (t0 + r) * L8 + wbase;
-                        if (need_lo) lo[r][i] = __ldcs(w);
-                        if (need_hi) hi[r][i] = __ldcs(w + 1);
-                        if (mask) {  // the first two selected features' values travel with the codes
-                            const uint16_t *hp = reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + p.lp_bytes) +
-                                                 (t0 + r) * p.k + hb;
-                            hv[r][i] = __ldcs(hp);
-                            if (n_lp < 7) hv[r][i] |= (uint32_t)__ldcs(hp + 1) << 16;
-                        }
-                    }
+                    w[r][i] = 0x88888888u;  // all codes zero... (unused when out of range)
+                    if (t0 + r < p.T && i0 + i < p.N)
+                        w[r][i] = __ldcs(reinterpret_cast<const uint32_t *>(p.pl[i0 + i]) + (t0 + r) * L8 + g);
                 }
 #pragma unroll
             for (int r = 0; r < R; ++r)
 #pragma unroll
-                for (int i = 0; i < NC; ++i) {
-                    if (t0 + r < p.T && i0 + i < p.N) {
-                        uint32_t raw = __funnelshift_r(lo[r][i], hi[r][i], sh);
-                        if (mask) raw = spread_holes(raw, mask);
-                        const uint32_t x = raw ^ 0x88888888u;  // two's complement -> offset binary
-#pragma unroll
-                        for (int n = 0; n < 8; ++n) {
-                            // 2^23 + (code + 8) as a float, minus (2^23 + 8): the code, exactly
-                            const float f =
-                                __fsub_rn(__uint_as_float(0x4B000000u | ((x >> (4 * n)) & 0xFu)), 8388616.0f);
-                            acc[r][n] = __fmaf_rn(f, sc[i][n], acc[r][n]);
-                        }
-                        if (mask) {
-                            const uint16_t *hp = reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + p.lp_bytes) +
-                                                 (t0 + r) * p.k + hb;
-                            int h = 0;
-#pragma unroll
-                            for (int n = 0; n < 8; ++n)
-                                if (mask & (1u << n)) {
-                                    const uint32_t bits = (h == 0)   ? (hv[r][i] << 16)
-                                                          : (h == 1) ? (hv[r][i] & 0xFFFF0000u)
-                                                                     : ((uint32_t)__ldcs(hp + h) << 16);
-                                    acc[r][n] = __fadd_rn(acc[r][n], __uint_as_float(bits));
-                                    ++h;
-                                }
-                        }
-                    }
-                }
+                for (int i = 0; i < NC; ++i)
+                    if (t0 + r < p.T && i0 + i < p.N) decode8(w[r][i], sc[i], acc[r]);
         }
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (t0 + r < p.T) {
-                if (FP32OUT) {
-                    float4 *o = reinterpret_cast<float4 *>(static_cast<float *>(p.out) + (t0 + r) * p.out_stride + 8 * g);
-                    __stcs(o, make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]));
-                    __stcs(o + 1, make_float4(acc[r][4], acc[r][5], acc[r][6], acc[r][7]));
-                } else {
-                    uint32_t w[4];
-#pragma unroll
-                    for (int n = 0; n < 4; ++n) {
-                        __nv_bfloat162 b = __floats2bfloat162_rn(acc[r][2 * n], acc[r][2 * n + 1]);
-                        w[n] = *reinterpret_cast<uint32_t *>(&b);
-                    }
-                    uint4 *o = reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.out) + (t0 + r) * p.out_stride + 8 * g);
-                    __stcs(o, make_uint4(w[0], w[1], w[2], w[3]));
-                }
-            }
-        }
+        for (int r = 0; r < R; ++r)
+            if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], mask);
     }
 }
 
-
 // ----------------------------------------------------------------------------------------------
-// Row kernel for N <= 8 devices (E, k, output stride multiples of 8; E/8 <= MAXT consumer threads).
+// Row kernel for N <= 8 devices and E/8 <= MAXT consumer threads.
 //
 // One persistent block per SM; a producer warp streams groups of G rows of all N payloads (code rows
 // and BF16 rows) into a ring of shared-memory stages with 1-D bulk asynchronous copies, completion on
 // "full" mbarriers; consumer warps release a stage through an "empty" mbarrier, so there is no
-// block-wide barrier in the loop.  Thread <-> 8 adjacent output features for every row: the N x 8
-// steps live in registers for the life of the block, pre-scaled by the power of 16 of the position at
-// which the code is decoded (see decode8), so each code costs one logic op, one subtract, one FMA.
-// G is a multiple of 4/gcd(4, (E-k)/8) so that every stage starts 16-byte aligned in the code stream.
+// block-wide barrier in the loop.  Thread <-> 8 adjacent output features for every row: its N x 8
+// steps live in registers for the life of the block.  G is a multiple of 4/gcd(4, L/8) so that every
+// stage starts 16-byte aligned in the code stream.
 // ----------------------------------------------------------------------------------------------
-constexpr int DR_WAIT_LIMIT = 1 << 22;
-
 struct DRLayout {
     size_t lp_stage, hp_stage, stage, bars, total;
 };
 __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int nstage)
 {
     DRLayout l;
-    l.lp_stage = (((size_t)G * (E - k) / 2) + 4 + 15) & ~(size_t)15;  // + one spare word: w[1] is read unconditionally
+    l.lp_stage = (((size_t)G * (E - k) / 2) + 15) & ~(size_t)15;
     l.hp_stage = (size_t)G * k * 2;
     l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
     l.bars = (size_t)nstage * l.stage;
@@ -272,56 +300,23 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
                  : "memory");
 }
 
-// 8 two's-complement codes of `raw` times their steps, accumulated.  The codes are decoded in place:
-// (x & 0xF << 4n) | 0x4B000000 is the float 2^23 + (code+8) 16^n; subtracting 2^23 + 8*16^n leaves
-// code * 16^n exactly, and the step was pre-divided by 16^n (an exact scaling), so
-// fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 5..7 use raw >> 20.
-// Subtractions and FMAs run two at a time (f32x2), one binary32 rounding per element as before.
-__device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
-
-__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4])
-{
-    const uint32_t xa = raw ^ 0x88888888u;
-    const uint32_t xb = xa >> 20;
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        const int n0 = 2 * h, n1 = 2 * h + 1;
-        const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
-        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | 0x4B000000u);
-        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | 0x4B000000u);
-        const float c0 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n0))));
-        const float c1 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n1))));
-        const float2 d = __fadd2_rn(make_float2(f0, f1), make_float2(c0, c1));
-        acc[h] = __ffma2_rn(d, sc[h], acc[h]);
-    }
-}
-
 struct DRParams {
     DQParams q;
-    const int32_t *hp_idx;
+    DXParams x;
     int G, nstage;
     int64_t ngroups;
-    int *status;
 };
-
-template <bool FP32OUT>
-__device__ __forceinline__ void store_one(void *out, int64_t off, float v)
-{
-    if (FP32OUT)
-        static_cast<float *>(out)[off] = v;
-    else
-        static_cast<__nv_bfloat16 *>(out)[off] = __float2bfloat16_rn(v);
-}
 
 template <int NMAX, int MAXT, bool FP32OUT>
 __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const DQParams &p = pp.q;
+    const DXParams &x = pp.x;
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
     const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;
-    const int E8 = E >> 3, L8 = (E - k) >> 3;
+    const int L8 = (E - k) >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
     uint64_t *empty = full + nstage;
@@ -334,18 +329,45 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+
+    // consumer constants: loads issued before the barrier that releases the producer (so that they
+    // are not queued behind the bulk copies)
+    const int g = tid;
+    const bool live = tid < NT && g < L8;
+    uint32_t mask = 0;
+    float2 sc[NMAX][4];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) {
+#pragma unroll
+        for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
+        if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
+    }
+    if (live) mask = __ldg(p.grp + g) & 0xFFu;
+    // extra job 1: filler feature my_fill (slot my_slot), extra job 2: selected feature my_hp
+    int my_fill = 0, my_slot = 0, my_hp = 0;
+    float fsc[NMAX];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) fsc[i] = 0.0f;
+    if (tid < NT && tid < x.n_holes) {
+        my_fill = __ldg(x.filler + tid);
+        my_slot = __ldg(x.hole + tid);
+#pragma unroll
+        for (int i = 0; i < NMAX; ++i)
+            if (i < N) fsc[i] = __ldg(p.s_k + (size_t)i * E + my_fill);
+    }
+    if (tid < NT && tid < k) my_hp = __ldg(x.hp_idx + tid);
     __syncthreads();
 
     if (tid >= NT) {
         // ---------------- producer warp: one lane streams the row groups
         if (tid == NT) {
             int st = 0;
-            uint32_t parity = 1;  // parity of the "empty" phase to wait for: ((it / nstage) - 1) & 1
+            uint32_t parity = 1;  // parity of the "empty" phase to wait for
             for (int it = 0;; ++it) {
                 const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
                 if (gi >= pp.ngroups) break;
                 if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
-                    atomicExch(pp.status, (int)TPQ_ERR_TIMEOUT);
+                    atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
                     break;
                 }
                 const int64_t t0 = gi * G;
@@ -371,54 +393,13 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
     }
 
     // ---------------- consumers
-    // Thread <-> output features 8g .. 8g+7.  Its n_lp quantised ones are adjacent in the code stream
-    // (slots c0 ..); slot c belongs to feature 8g + ofs(c).  The codes are NOT moved to their feature
-    // positions: the step of slot c is the step of feature 8g + ofs(c), and the row store puts slot c
-    // where it belongs.  Selected features are summed and stored by the threads h < k below.
-    const int g = tid;
-    const bool live = g < E8;
-    uint32_t mask = 0;
-    int hb = 0;
-    if (live) {
-        const uint32_t gd = __ldg(p.grp + g);
-        mask = gd & 0xFFu;
-        hb = (int)(gd >> 8);
-    }
-    const int c0 = 8 * g - hb;
-    const int n_lp = 8 - __popc(mask);
-    const int sh = (c0 & 7) * 4;
-    const int wbase = c0 >> 3;
-    uint32_t ofs_pack = 0;
-    {
-        int c = 0;
-#pragma unroll
-        for (int n = 0; n < 8; ++n)
-            if (!(mask & (1u << n))) ofs_pack |= (uint32_t)n << (3 * c++);
-    }
-
-    float2 sc[NMAX][4];
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) {
-        float v[8];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-            v[c] = 0.0f;
-            if (live && i < N && c < n_lp)
-                v[c] = __ldg(p.s_k + (size_t)i * E + 8 * g + ((ofs_pack >> (3 * c)) & 7)) *
-                       (1.0f / (float)(1 << (4 * dq_pos(c))));
-        }
-#pragma unroll
-        for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(v[2 * h], v[2 * h + 1]);
-    }
-    const int my_hp = (tid < k) ? __ldg(pp.hp_idx + tid) : 0;
-
     int st = 0;
-    uint32_t parity = 0;  // (it / nstage) & 1
+    uint32_t parity = 0;
     for (int it = 0;; ++it) {
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
         if (gi >= pp.ngroups) break;
         if (!mbar_wait(smem_u32(&full[st]), parity)) {
-            atomicExch(pp.status, (int)TPQ_ERR_TIMEOUT);
+            atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
         const int64_t t0 = gi * G;
@@ -430,40 +411,34 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
 #pragma unroll
                 for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
 #pragma unroll
-                for (int i = 0; i < NMAX; ++i) {
+                for (int i = 0; i < NMAX; ++i)
+                    if (i < N)
+                        decode8(reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + g], sc[i],
+                                acc);
+                store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc, mask);
+            }
+        }
+        // filler features: one code per device, from the slot they fill
+        for (int tau = tid; tau < x.n_holes; tau += NT) {
+            const bool mine = tau == tid;
+            const int j = mine ? my_fill : __ldg(x.filler + tau);
+            const int slot = mine ? my_slot : __ldg(x.hole + tau);
+            for (int r = 0; r < rows; ++r) {
+                float acc = 0.0f;
+#pragma unroll
+                for (int i = 0; i < NMAX; ++i)
                     if (i < N) {
-                        const uint32_t *w =
-                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage) + r * L8 + wbase;
-                        decode8(__funnelshift_r(w[0], w[1], sh), sc[i], acc);
+                        const uint32_t w =
+                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + (slot >> 3)];
+                        const int code = (int)(((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) - 8;
+                        acc = __fmaf_rn((float)code, mine ? fsc[i] : __ldg(p.s_k + (size_t)i * E + j), acc);
                     }
-                }
-                const int64_t o = (t0 + r) * p.out_stride + 8 * g;
-                if (mask == 0) {
-                    if (FP32OUT) {
-                        float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.out) + o);
-                        __stcs(dst, make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
-                        __stcs(dst + 1, make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y));
-                    } else {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) {
-                            __nv_bfloat162 b = __floats2bfloat162_rn(acc[h].x, acc[h].y);
-                            w[h] = *reinterpret_cast<uint32_t *>(&b);
-                        }
-                        __stcs(reinterpret_cast<uint4 *>(static_cast<uint16_t *>(p.out) + o),
-                               make_uint4(w[0], w[1], w[2], w[3]));
-                    }
-                } else {
-                    const float a8[8] = {acc[0].x, acc[0].y, acc[1].x, acc[1].y, acc[2].x, acc[2].y, acc[3].x, acc[3].y};
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        if (c < n_lp) store_one<FP32OUT>(p.out, o + ((ofs_pack >> (3 * c)) & 7), a8[c]);
-                }
+                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + j, acc);
             }
         }
         // selected features: sum of the BF16 values, devices ascending
         for (int h = tid; h < k; h += NT) {
-            const int j = (h == tid) ? my_hp : __ldg(pp.hp_idx + h);
+            const int j = (h == tid) ? my_hp : __ldg(x.hp_idx + h);
             const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
             for (int r = 0; r < rows; ++r) {
                 float acc = 0.0f;
@@ -496,6 +471,7 @@ bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int f
 {
     (void)fp32_out;
     if (c->E % 8 || c->k % 8 || out_stride % 8 || T <= 0) return false;
+    if (c->E - c->k < 8) return false;
     return true;
 }
 
@@ -534,9 +510,9 @@ cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads,
 bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *ngroups_out, int *grid_out)
 {
     const int N = c->N, E = c->E, k = c->k;
-    const int E8 = E / 8, L8 = (E - k) / 8;
-    if (N > 8 || E - k < 8) return false;
-    if (E8 > (N <= 4 ? 768 : 576)) return false;
+    const int L8 = (E - k) / 8;
+    if (N > 8) return false;
+    if (L8 > (N <= 4 ? 768 : 576)) return false;
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
     else if (L8 % 2 == 0) g0 = 2;
@@ -560,15 +536,19 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
 {
     DQParams p;
     fill_params(p, c, payloads, T, out, out_stride);
+    DXParams x;
+    x.hp_idx = c->t.hp_idx; x.hole = c->t.hole; x.filler = c->t.filler; x.n_holes = c->n_holes; x.status = c->t.status;
     {
         DRParams pp;
         int grid = 0;
         if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.ngroups, &grid)) {
             pp.q = p;
-            pp.hp_idx = c->t.hp_idx;
-            pp.status = c->t.status;
+            pp.x = x;
             const size_t smem = dr_layout(c->N, c->E, c->k, pp.G, pp.nstage).total;
-            const int threads = ((c->E / 8 + 31) / 32) * 32 + 32;
+            const int L8 = (c->E - c->k) / 8;
+            int consumers = ((L8 + 31) / 32) * 32;
+            if (consumers < 32) consumers = 32;
+            const int threads = consumers + 32;
             cudaError_t e = (c->N <= 4) ? launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st)
                                         : launch_rows<8, 576>(pp, fp32_out, grid, threads, smem, st);
             if (e != cudaSuccess) return e;
@@ -576,21 +556,21 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             return cudaGetLastError();
         }
     }
-    const int E8 = c->E / 8;
-    const int strips = (E8 + 127) / 128;
+    const int L8 = (c->E - c->k) / 8;
+    const int strips = (L8 + 127) / 128;
     constexpr int R = 4;
     const int64_t n_rb = (T + R - 1) / R;
     int64_t gy = ((int64_t)c->sm_count * 4 + strips - 1) / strips;
     if (gy > n_rb) gy = n_rb;
     if (gy > 65535) gy = 65535;
     if (gy < 1) gy = 1;
-    dim3 grid(strips, (unsigned)gy), block(128);
+    dim3 grid(strips + 1, (unsigned)gy), block(128);   // the last x-block does the filler / selected features
     if (c->N <= 4) {
-        if (fp32_out) dequant_tiled<4, R, true><<<grid, block, 0, st>>>(p);
-        else          dequant_tiled<4, R, false><<<grid, block, 0, st>>>(p);
+        if (fp32_out) dequant_strips<4, R, true><<<grid, block, 0, st>>>(p, x);
+        else          dequant_strips<4, R, false><<<grid, block, 0, st>>>(p, x);
     } else {
-        if (fp32_out) dequant_tiled<8, R, true><<<grid, block, 0, st>>>(p);
-        else          dequant_tiled<8, R, false><<<grid, block, 0, st>>>(p);
+        if (fp32_out) dequant_strips<8, R, true><<<grid, block, 0, st>>>(p, x);
+        else          dequant_strips<8, R, false><<<grid, block, 0, st>>>(p, x);
     }
     ++*launches;
     return cudaGetLastError();

@@ -58,17 +58,20 @@ __global__ void __launch_bounds__(256) quantize_generic(const uint16_t *__restri
 // ----------------------------------------------------------------------------------------------
 // Tiled kernel for E, k and stride multiples of 8.
 //
-// One persistent block per SM.  Rows reach shared memory through 1-D bulk asynchronous copies
-// (cp.async.bulk, completion on an mbarrier) into a ring of stages of G rows each, so the
-// whole share of a block can be in flight while it computes.  Thread <-> 8 adjacent features:
-// the reciprocal steps stay in registers for the life of the block.
-//   phase 1: 128-bit shared load of 8 BF16 -> 8 codes in feature order -> one word of a
-//            shared "code row"; selected features' BF16 patterns go to a shared side buffer
-//   phase 2: the selected features are squeezed out of the code row: output word w of a row
-//            is an unaligned 32-bit window of the code row (one funnel shift) unless a
-//            selected feature falls inside it (then code by code); coalesced 32-bit stores.
+// One persistent block per SM: a producer warp streams groups of G rows into a ring of shared-memory
+// stages with 1-D bulk asynchronous copies (cp.async.bulk, completion on "full" mbarriers); consumer
+// warps release a stage through an "empty" mbarrier.  There is no block-wide barrier in the loop.
+//
+// Consumer thread <-> 8 adjacent features (one 128-bit shared load per row); their reciprocal steps
+// stay in registers for the life of the block.  In the payload's slot order a group of 8 adjacent
+// features below L = E-k IS one 32-bit word of the code stream, so the thread stores its word
+// directly (coalesced 32-bit stores).  Where one of its 8 features is a selected one (a "hole"), the
+// slot belongs to a filler feature from the last k: the thread quantises that one element too
+// (16-bit shared load) and drops its code into the hole.  Threads h < k copy selected feature h of
+// every row to the BF16 block.
 // ----------------------------------------------------------------------------------------------
 constexpr int QP_MAX_GPT = 4;          // groups of 8 features per thread
+constexpr int QP_MAX_CONSUMERS = 992;  // 31 consumer warps + 1 producer warp per block
 constexpr int QP_WAIT_LIMIT = 1 << 22; // bounded mbarrier polling
 
 struct QPParams {
@@ -79,31 +82,29 @@ struct QPParams {
     int G;        // rows per stage
     int nstage;
     int64_t ngroups;
-    const float *inv_s;    // this device's [E]
-    const uint32_t *grp;   // [E/8]
-    const int32_t *lp_idx; // [E-k]
-    const int32_t *hp_idx; // [k]
+    const float *inv_s;     // this device's [E]
+    const uint32_t *grp;    // [E/8]
+    const int32_t *filler;  // [n_holes]
+    const int32_t *hp_idx;  // [k]
     uint32_t *lp_out;
-    int64_t lp_words;      // words of the code section, padding included
-    uint32_t *hp_out;      // as 32-bit words (k even)
+    int64_t lp_words;       // words of the code section, padding included
+    uint16_t *hp_out;
     int *status;
 #ifdef TPQ_TRACE
     long long *trace;
 #endif
 };
 
-// Dynamic shared memory layout (byte offsets, every section 16-byte aligned).
+// Dynamic shared memory layout (byte offsets).
 struct QPLayout {
-    size_t ring, nib, hpb, bars, total;
+    size_t ring, bars, total;
 };
-__host__ __device__ inline QPLayout qp_layout(int E, int k, int G, int nstage)
+__host__ __device__ inline QPLayout qp_layout(int E, int G, int nstage)
 {
     QPLayout l;
     l.ring = 0;
-    l.nib = (size_t)nstage * G * E * 2;
-    l.hpb = l.nib + (((size_t)2 * G * (E / 8 + 2) * 4 + 15) & ~(size_t)15);
-    l.bars = l.hpb + (((size_t)2 * G * k * 2 + 15) & ~(size_t)15);
-    l.total = l.bars + (size_t)nstage * 8;
+    l.bars = (size_t)nstage * G * E * 2;
+    l.total = l.bars + (size_t)nstage * 16;
     return l;
 }
 
@@ -117,23 +118,24 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // bounded wait: false if the phase never completed
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
-    for (int i = 0; i < QP_WAIT_LIMIT; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < QP_WAIT_LIMIT; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
     return false;
 }
 // global -> this block's shared memory, bytes a multiple of 16, both addresses 16-byte aligned
@@ -142,6 +144,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
+}
+
+// One element: product rounded to binary32, clamped, rounded half-to-even by the magic add; returns the
+// bits of fl(u + 1.5*2^23) = 0x4B400000 + code.
+__device__ __forceinline__ uint32_t quant_bits(uint32_t x_bf16, float inv_s)
+{
+    float u = __fmul_rn(__uint_as_float(x_bf16 << 16), inv_s);
+    u = fminf(fmaxf(u, -8.0f), 7.0f);
+    return __float_as_uint(__fadd_rn(u, 12582912.0f));
 }
 
 // 8 BF16 (one uint4) -> 8 two's-complement nibbles in feature order.
@@ -183,178 +194,173 @@ __device__ __forceinline__ long long tpq_now()
 template <int GPT>
 __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
 {
-    TPQ_MARK(0);
     extern __shared__ __align__(128) uint8_t smem[];
-    const int tid = threadIdx.x, NT = blockDim.x;
+    TPQ_MARK(0);
+    const int tid = threadIdx.x;
+    const int NT = blockDim.x - 32;  // consumer threads
     const int E = p.E, k = p.k, G = p.G, nstage = p.nstage;
     const int E8 = E >> 3, L8 = (E - k) >> 3;
-    const int nib_stride = E8 + 2;
     const uint32_t row_bytes = (uint32_t)E * 2u;
     const uint32_t stage_bytes = (uint32_t)G * row_bytes;
-
-    const QPLayout lay = qp_layout(E, k, G, nstage);
+    const QPLayout lay = qp_layout(E, G, nstage);
     uint8_t *ring = smem + lay.ring;
-    uint32_t *nib = reinterpret_cast<uint32_t *>(smem + lay.nib);
-    uint16_t *hpb = reinterpret_cast<uint16_t *>(smem + lay.hpb);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + lay.bars);
-    __shared__ int abort_flag;
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
+    uint64_t *empty = full + nstage;
 
     if (tid == 0) {
-        abort_flag = 0;
-        for (int s = 0; s < nstage; ++s) mbar_init(smem_u32(&bars[s]), 1);
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), NT / 32);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+
+    // ---- consumer constants: their loads are issued BEFORE the block-wide barrier that releases the
+    // producer, so they are not queued behind the bulk copies in the memory system.
+    float2 inv[GPT][4];
+    uint32_t mask[GPT];      // selected features among the thread's 8 (only where the group is below L)
+    int hb[GPT];             // holes before the group
+    // the first two holes of the group, ready to use: byte offset of the filler feature in a staged
+    // row, its reciprocal step, and the bit position of the hole's nibble in the word
+    uint32_t f_off[GPT][2], f_sh[GPT][2];
+    float f_inv[GPT][2];
+    int my_hp = 0;
+    if (tid < NT) {
+#pragma unroll
+        for (int a = 0; a < GPT; ++a) {
+            const int g = tid + a * NT;
+            mask[a] = 0; hb[a] = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
+            f_off[a][0] = f_off[a][1] = 0;
+            f_sh[a][0] = f_sh[a][1] = 0;
+            f_inv[a][0] = f_inv[a][1] = 0.0f;
+            if (g < L8) {
+                const float4 i0 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g));
+                const float4 i1 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g + 4));
+                const uint32_t gd = __ldg(p.grp + g);
+                inv[a][0] = make_float2(i0.x, i0.y);
+                inv[a][1] = make_float2(i0.z, i0.w);
+                inv[a][2] = make_float2(i1.x, i1.y);
+                inv[a][3] = make_float2(i1.z, i1.w);
+                mask[a] = gd & 0xFFu;
+                hb[a] = (int)(gd >> 8);
+            }
+        }
+        if (tid < k) my_hp = __ldg(p.hp_idx + tid);
     }
     __syncthreads();
     TPQ_MARK(40);
 
-    auto issue = [&](int it, int st) {  // group blockIdx.x + it*gridDim.x into stage st
-        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-        if (gi >= p.ngroups) return;
-        const int64_t t0 = gi * G;
-        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-        const uint32_t bar = smem_u32(&bars[st]);
-        const uint32_t dst = smem_u32(ring + (size_t)st * stage_bytes);
-        mbar_expect_tx(bar, rows * row_bytes);
-        if (p.stride == E) {
-            bulk_g2s(dst, p.y + t0 * p.stride, rows * row_bytes, bar);
-        } else {
-            for (int r = 0; r < rows; ++r) bulk_g2s(dst + r * row_bytes, p.y + (t0 + r) * p.stride, row_bytes, bar);
-        }
-    };
-    if (tid == 0)
-        for (int it = 0; it < nstage; ++it) issue(it, it);
-    TPQ_MARK(41);
-
-    // ---- per-thread constants (their loads overlap the first copies)
-    // phase 1: the reciprocal steps of the thread's 8 features, as four pairs
-    float2 inv[GPT][4];
-    // selected features: thread h < k copies feature my_hp of every row to the BF16 side buffer
-    const int my_hp = (tid < k) ? __ldg(p.hp_idx + tid) : 0;
-    // phase 2: output word wc = tid + a*NT of a row holds the 8 codes whose source features are
-    // lp_idx[8wc .. 8wc+7].  With d = number of selected features skipped so far (0, 1 or 2 inside one
-    // word in all but pathological sets), code c sits at source nibble src0 + c + d: the word is
-    // (W0 & ~(m1|m2)) | (W1 & m1) | (W2 & m2), Wd = the 32-bit window of the code row at nibble src0 + d.
-    int w0[GPT], sh[GPT];
-    uint32_t m1[GPT], m2[GPT];
-    int mode[GPT];  // 0: no word, 1: windows, 2: more than two skipped features, code by code
-#pragma unroll
-    for (int a = 0; a < GPT; ++a) {
-        const int g = tid + a * NT;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
-        if (g < E8) {
-            const float4 i0 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g));
-            const float4 i1 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g + 4));
-            inv[a][0] = make_float2(i0.x, i0.y);
-            inv[a][1] = make_float2(i0.z, i0.w);
-            inv[a][2] = make_float2(i1.x, i1.y);
-            inv[a][3] = make_float2(i1.z, i1.w);
-        }
-        w0[a] = 0; sh[a] = 0; m1[a] = 0; m2[a] = 0; mode[a] = 0;
-        if (g < L8) {
-            const int4 l0 = __ldg(reinterpret_cast<const int4 *>(p.lp_idx + 8 * g));
-            const int4 l1 = __ldg(reinterpret_cast<const int4 *>(p.lp_idx + 8 * g + 4));
-            const int idx[8] = {l0.x, l0.y, l0.z, l0.w, l1.x, l1.y, l1.z, l1.w};
-            w0[a] = idx[0] >> 3;
-            sh[a] = (idx[0] & 7) * 4;
-            mode[a] = (idx[7] - idx[0] - 7 <= 2) ? 1 : 2;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const int d = idx[c] - idx[0] - c;
-                if (d == 1) m1[a] |= 0xFu << (4 * c);
-                if (d == 2) m2[a] |= 0xFu << (4 * c);
-            }
-        }
-    }
-
-    TPQ_MARK(1);
-    int it = 0, st = 0;       // iteration, its ring stage (it mod nstage, kept without dividing)
-    uint32_t parity = 0;      // (it / nstage) & 1
-    for (;; ++it) {
-        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-        if (gi >= p.ngroups) break;
-        const int64_t t0 = gi * G;
-        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-        const int buf = it & 1;
-        if (!mbar_wait(smem_u32(&bars[st]), parity)) abort_flag = 1;
-        TPQ_MARK(2 + 3 * (int)it);
-
-        // ---- phase 1: quantise in feature order; copy the selected features
-        const uint4 *stage = reinterpret_cast<const uint4 *>(ring + (size_t)st * stage_bytes);
-        uint32_t *nrow = nib + (size_t)buf * G * nib_stride;
-        uint16_t *hrow = hpb + (size_t)buf * G * k;
-#pragma unroll
-        for (int a = 0; a < GPT; ++a) {
-            const int g = tid + a * NT;
-            if (g < E8)
-                for (int r = 0; r < rows; ++r) nrow[r * nib_stride + g] = quant8(stage[r * E8 + g], inv[a]);
-        }
-        {
-            const uint16_t *stage16 = reinterpret_cast<const uint16_t *>(stage);
-            for (int h = tid; h < k; h += NT) {
-                const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
-                for (int r = 0; r < rows; ++r) hrow[r * k + h] = stage16[r * E + j];
-            }
-        }
-        __syncthreads();
-        TPQ_MARK(3 + 3 * (int)it);
-        if (abort_flag) break;
-        if (tid == 0) issue(it + nstage, st);  // the stage is free again
-
-        // ---- phase 2: squeeze out the selected features, store
-#pragma unroll
-        for (int a = 0; a < GPT; ++a) {
-            const int wc = tid + a * NT;
-            if (mode[a] != 0) {
-                for (int r = 0; r < rows; ++r) {
-                    const uint32_t *src = nrow + r * nib_stride + w0[a];
-                    uint32_t word;
-                    if (mode[a] == 1) {
-                        const uint32_t x0 = src[0], x1 = src[1];
-                        const uint32_t W0 = __funnelshift_r(x0, x1, sh[a]);
-                        const uint32_t W1 = __funnelshift_rc(x0, x1, sh[a] + 4);
-                        word = (W0 & ~(m1[a] | m2[a])) | (W1 & m1[a]);
-                        if (m2[a]) {
-                            const uint32_t W2 = (sh[a] == 28) ? __funnelshift_r(x1, src[2], 4)
-                                                              : __funnelshift_rc(x0, x1, sh[a] + 8);
-                            word |= W2 & m2[a];
-                        }
-                    } else {
-                        word = 0;
-#pragma unroll 1
-                        for (int n = 0; n < 8; ++n) {
-                            const int j = __ldg(p.lp_idx + 8 * wc + n);
-                            word |= ((nrow[r * nib_stride + (j >> 3)] >> ((j & 7) * 4)) & 0xFu) << (4 * n);
-                        }
-                    }
-                    p.lp_out[(t0 + r) * L8 + wc] = word;
+    if (tid >= NT) {
+        // ---------------- producer warp: one lane streams the row groups
+        if (tid == NT) {
+            int st = 0;
+            uint32_t parity = 1;  // parity of the "empty" phase to wait for
+            for (int it = 0;; ++it) {
+                const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+                if (gi >= p.ngroups) break;
+                if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
+                    atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
+                    break;
+                }
+                const int64_t t0 = gi * G;
+                const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+                const uint32_t bar = smem_u32(&full[st]);
+                const uint32_t dst = smem_u32(ring + (size_t)st * stage_bytes);
+                mbar_expect_tx(bar, rows * row_bytes);
+                if (p.stride == E) {
+                    bulk_g2s(dst, p.y + t0 * p.stride, rows * row_bytes, bar);
+                } else {
+                    for (int r = 0; r < rows; ++r)
+                        bulk_g2s(dst + r * row_bytes, p.y + (t0 + r) * p.stride, row_bytes, bar);
+                }
+                if (++st == nstage) {
+                    st = 0;
+                    parity ^= 1u;
                 }
             }
         }
-        {
-            const uint32_t *h32 = reinterpret_cast<const uint32_t *>(hrow);
-            const int n32 = rows * k / 2;
-            uint32_t *dst = p.hp_out + t0 * (k / 2);
-            for (int a = tid; a < n32; a += NT) dst[a] = h32[a];
+        return;
+    }
+
+    // ---------------- consumers
+#pragma unroll
+    for (int a = 0; a < GPT; ++a) {
+        uint32_t m = mask[a];
+        for (int h = 0; h < 2 && m; ++h) {
+            const int f = __ldg(p.filler + hb[a] + h);
+            f_off[a][h] = (uint32_t)f * 2u;
+            f_inv[a][h] = __ldg(p.inv_s + f);
+            f_sh[a][h] = (uint32_t)(__ffs(m) - 1) * 4u;
+            m &= m - 1;
         }
-        TPQ_MARK(4 + 3 * (int)it);
+    }
+    TPQ_MARK(1);
+
+    int st = 0;
+    uint32_t parity = 0;
+    for (int it = 0;; ++it) {
+        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+        if (gi >= p.ngroups) break;
+        if (!mbar_wait(smem_u32(&full[st]), parity)) {
+            atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
+            break;
+        }
+        TPQ_MARK(2 + 2 * it);
+        const int64_t t0 = gi * G;
+        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+        const uint4 *stage = reinterpret_cast<const uint4 *>(ring + (size_t)st * stage_bytes);
+        const uint16_t *stage16 = reinterpret_cast<const uint16_t *>(stage);
+#pragma unroll
+        for (int a = 0; a < GPT; ++a) {
+            const int g = tid + a * NT;
+            if (g < L8) {
+                const uint32_t nh = __popc(mask[a]);
+                for (int r = 0; r < rows; ++r) {
+                    uint32_t word = quant8(stage[r * E8 + g], inv[a]);
+                    if (nh) {
+                        // a hole's slot belongs to a filler feature: quantise that element, drop its code in
+                        const uint8_t *row8 = reinterpret_cast<const uint8_t *>(stage) + (size_t)r * row_bytes;
+                        {
+                            const uint32_t x = *reinterpret_cast<const uint16_t *>(row8 + f_off[a][0]);
+                            const uint32_t q = quant_bits(x, f_inv[a][0]) & 0xFu;
+                            word = (word & ~(0xFu << f_sh[a][0])) | (q << f_sh[a][0]);
+                        }
+                        if (nh > 1) {
+                            const uint32_t x = *reinterpret_cast<const uint16_t *>(row8 + f_off[a][1]);
+                            const uint32_t q = quant_bits(x, f_inv[a][1]) & 0xFu;
+                            word = (word & ~(0xFu << f_sh[a][1])) | (q << f_sh[a][1]);
+                        }
+                        if (nh > 2) {  // rare: more than two selected features among 8 adjacent ones
+                            uint32_t m = mask[a];
+                            m &= m - 1;
+                            m &= m - 1;
+                            for (int h = 2; m; ++h) {
+                                const int n = __ffs(m) - 1;
+                                m &= m - 1;
+                                const int f = __ldg(p.filler + hb[a] + h);
+                                const uint32_t q = quant_bits(stage16[r * E + f], __ldg(p.inv_s + f)) & 0xFu;
+                                word = (word & ~(0xFu << (4 * n))) | (q << (4 * n));
+                            }
+                        }
+                    }
+                    p.lp_out[(t0 + r) * L8 + g] = word;
+                }
+            }
+        }
+        for (int h = tid; h < k; h += NT) {
+            const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
+            for (int r = 0; r < rows; ++r) p.hp_out[(t0 + r) * k + h] = stage16[r * E + j];
+        }
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
+        TPQ_MARK(3 + 2 * it);
         if (++st == nstage) {
             st = 0;
             parity ^= 1u;
         }
-    }
-
-    if (abort_flag) {
-        // a copy never completed: report, give the copies still in flight a bounded chance to land, leave
-        if (tid == 0) {
-            atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
-            for (int j = it + 1; j < it + nstage; ++j) {
-                if (blockIdx.x + j * (int64_t)gridDim.x >= p.ngroups) break;
-                mbar_wait(smem_u32(&bars[j % nstage]), (uint32_t)((j / nstage) & 1));
-            }
-        }
-        return;
     }
     // zero padding of the code section (at most 3 words), by the block that owned the last rows
     if ((p.ngroups - 1) % gridDim.x == blockIdx.x) {
@@ -363,7 +369,7 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
     }
 }
 
-size_t qp_smem_bytes(int E, int k, int G, int nstage) { return qp_layout(E, k, G, nstage).total; }
+size_t qp_smem_bytes(int E, int G, int nstage) { return qp_layout(E, G, nstage).total; }
 
 }  // namespace
 
@@ -371,9 +377,9 @@ bool tpq_quantize_tiled_ok(const tpq_ctx *c, int64_t T, int64_t stride)
 {
     const int E = c->E, k = c->k;
     if (E % 8 || k % 8 || stride % 8 || T <= 0) return false;
-    if (E - k < 8) return false;                       // nothing (or too little) to squeeze
-    if (E / 8 > 1024 * QP_MAX_GPT) return false;
-    if (qp_smem_bytes(E, k, 1, 2) > (size_t)c->smem_optin) return false;
+    if (E - k < 8) return false;
+    if (E / 8 > QP_MAX_CONSUMERS * QP_MAX_GPT) return false;
+    if (qp_smem_bytes(E, 1, 2) > (size_t)c->smem_optin) return false;
     return true;
 }
 
@@ -399,35 +405,35 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
 {
     const int E = c->E, k = c->k;
     const int E8 = E / 8;
-    const int gpt = (E8 + 1023) / 1024;
-    int nt = ((E8 + gpt - 1) / gpt + 31) / 32 * 32;
-    // rows per stage: small enough that every SM gets work, large enough to amortise the barrier
+    const int gpt = (E8 + QP_MAX_CONSUMERS - 1) / QP_MAX_CONSUMERS;
+    const int nt = ((E8 + gpt - 1) / gpt + 31) / 32 * 32;
+    // rows per stage: small enough that every SM gets work
     int G = 2;
     if ((T + G - 1) / G < c->sm_count) G = 1;
-    while (G > 1 && qp_smem_bytes(E, k, G, 2) > (size_t)c->smem_optin) G >>= 1;
+    while (G > 1 && qp_smem_bytes(E, G, 2) > (size_t)c->smem_optin) G >>= 1;
     const int64_t ngroups = (T + G - 1) / G;
-    int64_t grid = ngroups < c->sm_count ? ngroups : c->sm_count;
-    int64_t per_block = (ngroups + grid - 1) / grid;
+    const int64_t grid = ngroups < c->sm_count ? ngroups : c->sm_count;
+    const int64_t per_block = (ngroups + grid - 1) / grid;
     int nstage = (int)(per_block < 8 ? per_block : 8);
-    if (nstage < 1) nstage = 1;
-    while (nstage > 1 && qp_smem_bytes(E, k, G, nstage) > (size_t)c->smem_optin) --nstage;
+    if (nstage < 2) nstage = 2;
+    while (nstage > 2 && qp_smem_bytes(E, G, nstage) > (size_t)c->smem_optin) --nstage;
 
     QPParams p;
     const int64_t lpb = tpq_lp_bytes_i(T, E, k);
     p.y = y; p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
-    p.inv_s = c->t.inv_s + (size_t)shard * E; p.grp = c->t.grp; p.lp_idx = c->t.lp_idx; p.hp_idx = c->t.hp_idx;
+    p.inv_s = c->t.inv_s + (size_t)shard * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
     p.lp_out = reinterpret_cast<uint32_t *>(payload); p.lp_words = lpb / 4;
-    p.hp_out = reinterpret_cast<uint32_t *>(payload + lpb); p.status = c->t.status;
+    p.hp_out = reinterpret_cast<uint16_t *>(payload + lpb); p.status = c->t.status;
 #ifdef TPQ_TRACE
     p.trace = g_trace;
 #endif
-    const size_t smem = qp_smem_bytes(E, k, G, nstage);
+    const size_t smem = qp_smem_bytes(E, G, nstage);
 
     cudaError_t e = cudaSuccess;
 #define TPQ_QP_LAUNCH(GPT)                                                                                       \
     do {                                                                                                         \
         e = cudaFuncSetAttribute(quantize_tiled<GPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
-        if (e == cudaSuccess) quantize_tiled<GPT><<<(unsigned)grid, nt, smem, st>>>(p);                          \
+        if (e == cudaSuccess) quantize_tiled<GPT><<<(unsigned)grid, nt + 32, smem, st>>>(p);                     \
     } while (0)
     switch (gpt) {
         case 1: TPQ_QP_LAUNCH(1); break;

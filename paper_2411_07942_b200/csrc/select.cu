@@ -50,13 +50,14 @@ __global__ void __launch_bounds__(256) topk_flags_kernel(const float *__restrict
     if (j < E) flag[j] = (beats < k) ? 1 : 0;
 }
 
-// One block: exclusive scan of the flags -> index lists, per-feature slots, the
-// dequantiser's zeroed-step copy and the per-8-feature group descriptors.
-__global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E)
+// One block: exclusive scan of the flags -> selected list, hole / filler lists, slot order,
+// per-feature slots, the dequantiser's zeroed-step copy and the per-8-feature group descriptors.
+__global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E, int k)
 {
     __shared__ int warp_sums[32];
     __shared__ int carry;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int L = E - k;
     if (tid == 0) carry = 0;
     __syncthreads();
     for (int j0 = 0; j0 < E; j0 += 1024) {
@@ -84,18 +85,28 @@ __global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E
         const int before = carry + warp_sums[wid] + incl - f;  // selected features before j
         if (j < E) {
             t.hpre[j] = before;
-            if (f) {
-                t.hp_idx[before] = j;
-                t.pos[j] = -(before + 1);
-            } else {
-                t.lp_idx[j - before] = j;
-                t.pos[j] = j - before;
-            }
+            if (f) t.hp_idx[before] = j;
             for (int i = 0; i < N; ++i) t.s_k[(size_t)i * E + j] = f ? 0.0f : t.s[(size_t)i * E + j];
         }
         __syncthreads();
         if (tid == 1023) carry = before + f;
         __syncthreads();
+    }
+    // holes: selected features below L; fillers: unselected features at or above L (equally many)
+    const int m = (L < E) ? t.hpre[L] : 0;
+    for (int j = tid; j < E; j += 1024) {
+        const int f = t.flag[j];
+        if (f && j < L) t.hole[t.hpre[j]] = j;
+        if (!f && j >= L) t.filler[(j - L) - (t.hpre[j] - m)] = j;
+    }
+    __syncthreads();
+    for (int j = tid; j < E; j += 1024) {
+        const int f = t.flag[j];
+        if (j < L) t.lp_idx[j] = f ? t.filler[t.hpre[j]] : j;
+        if (f)
+            t.pos[j] = -(t.hpre[j] + 1);
+        else
+            t.pos[j] = (j < L) ? j : t.hole[(j - L) - (t.hpre[j] - m)];
     }
     const int n_grp = (E + 7) / 8;
     for (int g = tid; g < n_grp; g += 1024) {
@@ -122,9 +133,9 @@ cudaError_t tpq_launch_topk_flags(const tpq_tables &t, int E, int k, cudaStream_
     return cudaGetLastError();
 }
 
-cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches)
+cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, int k, cudaStream_t st, int64_t *launches)
 {
-    tables_kernel<<<1, 1024, 0, st>>>(t, N, E);
+    tables_kernel<<<1, 1024, 0, st>>>(t, N, E, k);
     ++*launches;
     return cudaGetLastError();
 }

@@ -46,7 +46,7 @@ void free_tables(tpq_tables &t)
 {
     cudaFree(t.m); cudaFree(t.M); cudaFree(t.R); cudaFree(t.Rbar); cudaFree(t.s); cudaFree(t.inv_s);
     cudaFree(t.s_k); cudaFree(t.flag); cudaFree(t.hpre); cudaFree(t.pos); cudaFree(t.hp_idx);
-    cudaFree(t.lp_idx); cudaFree(t.grp); cudaFree(t.status);
+    cudaFree(t.lp_idx); cudaFree(t.hole); cudaFree(t.filler); cudaFree(t.grp); cudaFree(t.status);
     memset(&t, 0, sizeof t);
 }
 
@@ -66,9 +66,12 @@ tpq_status build_tables(tpq_ctx *c, int k, bool topk)
         e = tpq_launch_topk_flags(c->t, c->E, k, 0, &c->launches);
         if (e != cudaSuccess) return cuda_fail(c, e, "top-k kernel");
     }
-    e = tpq_launch_tables(c->t, c->N, c->E, 0, &c->launches);
+    e = tpq_launch_tables(c->t, c->N, c->E, k, 0, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e, "tables kernel");
     TPQ_CUDA(c, cudaDeviceSynchronize());
+    c->n_holes = 0;
+    if (k > 0 && k < c->E)
+        TPQ_CUDA(c, cudaMemcpy(&c->n_holes, c->t.hpre + (c->E - k), sizeof(int), cudaMemcpyDeviceToHost));
     c->k = k;
     return TPQ_OK;
 }
@@ -131,6 +134,8 @@ tpq_status tpq_create(tpq_ctx **out, int n_shards, int n_features, int bits, flo
     if (e == cudaSuccess) e = dalloc(&t.pos, E);
     if (e == cudaSuccess) e = dalloc(&t.hp_idx, E);
     if (e == cudaSuccess) e = dalloc(&t.lp_idx, E);
+    if (e == cudaSuccess) e = dalloc(&t.hole, E);
+    if (e == cudaSuccess) e = dalloc(&t.filler, E);
     if (e == cudaSuccess) e = dalloc(&t.grp, (E + 7) / 8);
     if (e == cudaSuccess) e = dalloc(&t.status, 1);
     if (e == cudaSuccess) e = cudaMemset(t.m, 0, NE * sizeof(float));

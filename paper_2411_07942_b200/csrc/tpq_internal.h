@@ -17,9 +17,11 @@ struct tpq_tables {
     float *s_k;          // [N][E] step with 0 at selected features (dequantiser's copy)
     uint8_t *flag;       // [E]    1 = selected (kept in BF16)
     int32_t *hpre;       // [E]    number of selected features before j
-    int32_t *pos;        // [E]    >= 0: slot in the compacted code stream; < 0: -(h+1), h = rank among selected
+    int32_t *pos;        // [E]    >= 0: code slot of feature j; < 0: -(h+1), h = rank among selected
     int32_t *hp_idx;     // [E]    first k entries: selected features, ascending
-    int32_t *lp_idx;     // [E]    first E-k entries: the others, ascending
+    int32_t *lp_idx;     // [E]    first L = E-k entries: feature held by code slot c (slot order below)
+    int32_t *hole;       // [E]    first n_holes entries: selected features below L, ascending (slots to fill)
+    int32_t *filler;     // [E]    first n_holes entries: unselected features at or above L, ascending
     uint32_t *grp;       // [ceil(E/8)] per group of 8 features: (selected before the group << 8) | 8-bit mask
     int *status;         // device status word (0 = ok)
 };
@@ -28,6 +30,7 @@ struct tpq_ctx {
     int N, E, bits;
     float gamma;
     int k;              // -1 until a feature set exists
+    int n_holes;        // selected features below E-k (= unselected ones at or above it)
     int device;
     int sm_count;
     int smem_optin;     // max dynamic shared memory per block
@@ -40,6 +43,11 @@ struct tpq_ctx {
     char err[512];
 };
 
+// Slot order of a token's L = E-k codes ("hole filling"): slot c holds feature c unless c is selected;
+// the selected features below L (hole[], ascending) are filled in order with the unselected features
+// at or above L (filler[], ascending).  Most features keep their own index as slot, so a group of 8
+// adjacent features is one aligned 32-bit word of the code stream.
+//
 // Payload geometry (Section 4 bit count; layout documented in tpq.h).
 static inline int64_t tpq_lp_bytes_i(int64_t T, int64_t E, int64_t k)
 {
@@ -59,7 +67,7 @@ cudaError_t tpq_launch_calibrate(const uint16_t *y, int64_t n_seq, int64_t S, in
 // Section 3: ranges, aggregate, steps; top-k flags (or flags given); index tables.
 cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_topk_flags(const tpq_tables &t, int E, int k, cudaStream_t st, int64_t *launches);
-cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, int k, cudaStream_t st, int64_t *launches);
 
 // C^(i): quantise + pack.
 bool tpq_quantize_tiled_ok(const tpq_ctx *c, int64_t T, int64_t stride);
