@@ -191,14 +191,14 @@ __device__ __forceinline__ long long tpq_now()
 #define TPQ_MARK(slot) do { } while (0)
 #endif
 
-template <int GPT>
-__global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
+template <int GPT, int G, int TB>  // TB: upper bound of the block size (register budget)
+__global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     TPQ_MARK(0);
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
-    const int E = p.E, k = p.k, G = p.G, nstage = p.nstage;
+    const int E = p.E, k = p.k, nstage = p.nstage;  // G rows per stage, unrolled: G independent chains per thread
     const int E8 = E >> 3, L8 = (E - k) >> 3;
     const uint32_t row_bytes = (uint32_t)E * 2u;
     const uint32_t stage_bytes = (uint32_t)G * row_bytes;
@@ -221,10 +221,8 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
     float2 inv[GPT][4];
     uint32_t mask[GPT];      // selected features among the thread's 8 (only where the group is below L)
     int hb[GPT];             // holes before the group
-    // the first two holes of the group, ready to use: byte offset of the filler feature in a staged
-    // row, its reciprocal step, and the bit position of the hole's nibble in the word
-    uint32_t f_off[GPT][2], f_sh[GPT][2];
-    float f_inv[GPT][2];
+    // the first two holes of the group: bit position of the hole's nibble in the word and its mask
+    uint32_t f_sh[GPT][2], hmask[GPT][2];
     int my_hp = 0;
     if (tid < NT) {
 #pragma unroll
@@ -233,9 +231,8 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
             mask[a] = 0; hb[a] = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
-            f_off[a][0] = f_off[a][1] = 0;
             f_sh[a][0] = f_sh[a][1] = 0;
-            f_inv[a][0] = f_inv[a][1] = 0.0f;
+            hmask[a][0] = hmask[a][1] = 0;
             if (g < L8) {
                 const float4 i0 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g));
                 const float4 i1 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g + 4));
@@ -286,14 +283,42 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
     }
 
     // ---------------- consumers
+    // Holes are patched warp-cooperatively.  The holes of a warp's 32 groups are consecutive in the
+    // global hole order, so lane i quantises the filler element of the warp's i-th hole (w_off / w_inv)
+    // and the owner of a hole fetches the code with a shuffle (from lane src0, src0 + 1 for a second
+    // hole).  A warp with more than 32 holes, or a lane with more than two, takes the serial path.
+    const int lane = tid & 31;
+    uint32_t w_off[GPT];     // byte offset of "my" filler element in a staged row (lane < n_wh)
+    float w_inv[GPT];
+    int n_wh[GPT], src0[GPT];
+    bool serial[GPT];
+    uint32_t keep[GPT];      // word bits that are not holes
 #pragma unroll
     for (int a = 0; a < GPT; ++a) {
+        const int nh = __popc(mask[a]);
+        int incl = nh;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += o;
+        }
+        src0[a] = incl - nh;
+        n_wh[a] = __shfl_sync(0xffffffffu, incl, 31);
+        const int hb_warp = __shfl_sync(0xffffffffu, hb[a], 0);
+        serial[a] = n_wh[a] > 32 || __any_sync(0xffffffffu, nh > 2);
+        w_off[a] = 0;
+        w_inv[a] = 0.0f;
+        if (lane < n_wh[a] && !serial[a]) {
+            const int f = __ldg(p.filler + hb_warp + lane);
+            w_off[a] = (uint32_t)f * 2u;
+            w_inv[a] = __ldg(p.inv_s + f);
+        }
         uint32_t m = mask[a];
+        keep[a] = 0xFFFFFFFFu;
         for (int h = 0; h < 2 && m; ++h) {
-            const int f = __ldg(p.filler + hb[a] + h);
-            f_off[a][h] = (uint32_t)f * 2u;
-            f_inv[a][h] = __ldg(p.inv_s + f);
             f_sh[a][h] = (uint32_t)(__ffs(m) - 1) * 4u;
+            hmask[a][h] = 0xFu << f_sh[a][h];
+            keep[a] &= ~hmask[a][h];
             m &= m - 1;
         }
     }
@@ -316,39 +341,52 @@ __global__ void __launch_bounds__(1024, 1) quantize_tiled(const QPParams p)
 #pragma unroll
         for (int a = 0; a < GPT; ++a) {
             const int g = tid + a * NT;
-            if (g < L8) {
-                const uint32_t nh = __popc(mask[a]);
+            const bool live = g < L8;
+            const int g_ld = live ? g : 0;  // idle lanes load something harmless: straight-line code below
+            const uint32_t nh = __popc(mask[a]);
+            const uint8_t *stage8 = reinterpret_cast<const uint8_t *>(stage);
+            if (!serial[a] && rows == G) {
+                // full stage: all shared loads of the G rows first, then G independent chains, no branches
+                uint4 v[G];
+                uint32_t fx[G];
+#pragma unroll
+                for (int r = 0; r < G; ++r) {
+                    v[r] = stage[r * E8 + g_ld];
+                    fx[r] = *reinterpret_cast<const uint16_t *>(stage8 + (size_t)r * row_bytes + w_off[a]);
+                }
+                uint32_t word[G];
+#pragma unroll
+                for (int r = 0; r < G; ++r) word[r] = quant8(v[r], inv[a]);
+                if (n_wh[a]) {  // uniform over the warp
+#pragma unroll
+                    for (int r = 0; r < G; ++r) {
+                        const uint32_t qv = quant_bits(fx[r], w_inv[a]) & 0xFu;
+                        const uint32_t q0 = __shfl_sync(0xffffffffu, qv, src0[a]) << f_sh[a][0];
+                        const uint32_t q1 = __shfl_sync(0xffffffffu, qv, src0[a] + 1) << f_sh[a][1];
+                        word[r] = (word[r] & keep[a]) | (q0 & hmask[a][0]) | (q1 & hmask[a][1]);
+                    }
+                }
+                if (live) {
+#pragma unroll
+                    for (int r = 0; r < G; ++r) p.lp_out[(t0 + r) * L8 + g] = word[r];
+                }
+            } else if (live) {
+                // ragged last stage, or a warp on the serial path: every hole patched by its owner
                 for (int r = 0; r < rows; ++r) {
                     uint32_t word = quant8(stage[r * E8 + g], inv[a]);
-                    if (nh) {
-                        // a hole's slot belongs to a filler feature: quantise that element, drop its code in
-                        const uint8_t *row8 = reinterpret_cast<const uint8_t *>(stage) + (size_t)r * row_bytes;
-                        {
-                            const uint32_t x = *reinterpret_cast<const uint16_t *>(row8 + f_off[a][0]);
-                            const uint32_t q = quant_bits(x, f_inv[a][0]) & 0xFu;
-                            word = (word & ~(0xFu << f_sh[a][0])) | (q << f_sh[a][0]);
-                        }
-                        if (nh > 1) {
-                            const uint32_t x = *reinterpret_cast<const uint16_t *>(row8 + f_off[a][1]);
-                            const uint32_t q = quant_bits(x, f_inv[a][1]) & 0xFu;
-                            word = (word & ~(0xFu << f_sh[a][1])) | (q << f_sh[a][1]);
-                        }
-                        if (nh > 2) {  // rare: more than two selected features among 8 adjacent ones
-                            uint32_t m = mask[a];
-                            m &= m - 1;
-                            m &= m - 1;
-                            for (int h = 2; m; ++h) {
-                                const int n = __ffs(m) - 1;
-                                m &= m - 1;
-                                const int f = __ldg(p.filler + hb[a] + h);
-                                const uint32_t q = quant_bits(stage16[r * E + f], __ldg(p.inv_s + f)) & 0xFu;
-                                word = (word & ~(0xFu << (4 * n))) | (q << (4 * n));
-                            }
-                        }
+                    uint32_t m = mask[a];
+                    for (int h = 0; m; ++h) {
+                        const int n = __ffs(m) - 1;
+                        m &= m - 1;
+                        const int f = __ldg(p.filler + hb[a] + h);
+                        const uint32_t x = *reinterpret_cast<const uint16_t *>(stage8 + (size_t)r * row_bytes + 2 * f);
+                        const uint32_t q = quant_bits(x, __ldg(p.inv_s + f)) & 0xFu;
+                        word = (word & ~(0xFu << (4 * n))) | (q << (4 * n));
                     }
                     p.lp_out[(t0 + r) * L8 + g] = word;
                 }
             }
+            (void)nh;
         }
         for (int h = tid; h < k; h += NT) {
             const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
@@ -407,10 +445,9 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
     const int E8 = E / 8;
     const int gpt = (E8 + QP_MAX_CONSUMERS - 1) / QP_MAX_CONSUMERS;
     const int nt = ((E8 + gpt - 1) / gpt + 31) / 32 * 32;
-    // rows per stage: small enough that every SM gets work
-    int G = 2;
-    if ((T + G - 1) / G < c->sm_count) G = 1;
-    while (G > 1 && qp_smem_bytes(E, G, 2) > (size_t)c->smem_optin) G >>= 1;
+    // rows per stage (= independent chains per thread): small enough that every SM gets work
+    int G = 4;
+    while (G > 1 && ((T + G - 1) / G < 2 * (int64_t)c->sm_count || qp_smem_bytes(E, G, 3) > (size_t)c->smem_optin)) G >>= 1;
     const int64_t ngroups = (T + G - 1) / G;
     const int64_t grid = ngroups < c->sm_count ? ngroups : c->sm_count;
     const int64_t per_block = (ngroups + grid - 1) / grid;
@@ -430,17 +467,34 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
     const size_t smem = qp_smem_bytes(E, G, nstage);
 
     cudaError_t e = cudaSuccess;
-#define TPQ_QP_LAUNCH(GPT)                                                                                       \
-    do {                                                                                                         \
-        e = cudaFuncSetAttribute(quantize_tiled<GPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
-        if (e == cudaSuccess) quantize_tiled<GPT><<<(unsigned)grid, nt + 32, smem, st>>>(p);                     \
+#define TPQ_QP_LAUNCH(GPT, GG, TB)                                                                                   \
+    do {                                                                                                             \
+        e = cudaFuncSetAttribute(quantize_tiled<GPT, GG, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
+                                 (int)smem);                                                                         \
+        if (e == cudaSuccess) quantize_tiled<GPT, GG, TB><<<(unsigned)grid, nt + 32, smem, st>>>(p);                 \
     } while (0)
-    switch (gpt) {
-        case 1: TPQ_QP_LAUNCH(1); break;
-        case 2: TPQ_QP_LAUNCH(2); break;
-        case 3: TPQ_QP_LAUNCH(3); break;
-        default: TPQ_QP_LAUNCH(4); break;
+#define TPQ_QP_LAUNCH_G(GPT, TB)                          \
+    do {                                                  \
+        if (G == 4) TPQ_QP_LAUNCH(GPT, 4, TB);            \
+        else if (G == 2) TPQ_QP_LAUNCH(GPT, 2, TB);       \
+        else TPQ_QP_LAUNCH(GPT, 1, TB);                   \
+    } while (0)
+    if (nt + 32 <= 704) {
+        switch (gpt) {
+            case 1: TPQ_QP_LAUNCH_G(1, 704); break;
+            case 2: TPQ_QP_LAUNCH_G(2, 704); break;
+            case 3: TPQ_QP_LAUNCH_G(3, 704); break;
+            default: TPQ_QP_LAUNCH_G(4, 704); break;
+        }
+    } else {
+        switch (gpt) {
+            case 1: TPQ_QP_LAUNCH_G(1, 1024); break;
+            case 2: TPQ_QP_LAUNCH_G(2, 1024); break;
+            case 3: TPQ_QP_LAUNCH_G(3, 1024); break;
+            default: TPQ_QP_LAUNCH_G(4, 1024); break;
+        }
     }
+#undef TPQ_QP_LAUNCH_G
 #undef TPQ_QP_LAUNCH
     if (e != cudaSuccess) return e;
     ++*launches;
