@@ -305,18 +305,35 @@ struct DRParams {
     DXParams x;
     int G, nstage;
     int64_t ngroups;
+#ifdef TPQ_TRACE
+    long long *trace;
+#endif
 };
+
+#ifdef TPQ_TRACE
+static long long *g_dtrace = nullptr;  // 64 slots per block, globaltimer ns
+__device__ __forceinline__ long long tpq_dnow()
+{
+    long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+#define TPQ_DMARK(slot) do { if (threadIdx.x == 0 && pp.trace && (slot) < 64) pp.trace[blockIdx.x * 64 + (slot)] = tpq_dnow(); } while (0)
+#else
+#define TPQ_DMARK(slot) do { } while (0)
+#endif
 
 template <int NMAX, int MAXT, bool FP32OUT>
 __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
+    TPQ_DMARK(0);
     const DQParams &p = pp.q;
     const DXParams &x = pp.x;
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
-    const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;
-    const int L8 = (E - k) >> 3;
+    const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;  // G rows per stage, even
+    const int L = E - k, L8 = L >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
     uint64_t *empty = full + nstage;
@@ -334,7 +351,16 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
     // are not queued behind the bulk copies)
     const int g = tid;
     const bool live = tid < NT && g < L8;
+    const int g_ld = live ? g : 0;
     uint32_t mask = 0;
+    int hb = 0;
+    if (live) {
+        const uint32_t gd = __ldg(p.grp + g);
+        mask = gd & 0xFFu;
+        hb = (int)(gd >> 8);
+    }
+    // steps of the thread's 8 slots; 0 where the slot's own feature is a selected one (a hole)
+    const int nh = __popc(mask);
     float2 sc[NMAX][4];
 #pragma unroll
     for (int i = 0; i < NMAX; ++i) {
@@ -342,57 +368,89 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
         for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
     }
-    if (live) mask = __ldg(p.grp + g) & 0xFFu;
-    // extra job 1: filler feature my_fill (slot my_slot), extra job 2: selected feature my_hp
-    int my_fill = 0, my_slot = 0, my_hp = 0;
-    float fsc[NMAX];
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) fsc[i] = 0.0f;
-    if (tid < NT && tid < x.n_holes) {
-        my_fill = __ldg(x.filler + tid);
-        my_slot = __ldg(x.hole + tid);
-#pragma unroll
-        for (int i = 0; i < NMAX; ++i)
-            if (i < N) fsc[i] = __ldg(p.s_k + (size_t)i * E + my_fill);
-    }
-    if (tid < NT && tid < k) my_hp = __ldg(x.hp_idx + tid);
+    // tail job: the selected features at or above L (ranks n_holes .. k-1; about one per row on
+    // average) are summed by the LAST consumer threads, one feature each
+    const int n_tail = k - x.n_holes;
+    const int tail_t = NT - 1 - tid;
+    int tail_col = 0;
+    if (tid < NT && tail_t < n_tail) tail_col = __ldg(x.hp_idx + x.n_holes + tail_t);
     __syncthreads();
 
     if (tid >= NT) {
-        // ---------------- producer warp: one lane streams the row groups
-        if (tid == NT) {
-            int st = 0;
-            uint32_t parity = 1;  // parity of the "empty" phase to wait for
-            for (int it = 0;; ++it) {
-                const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-                if (gi >= pp.ngroups) break;
+        // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
+        // copies of the stage (a code-row block and a BF16 block per device) are issued by 2N lanes at once
+        const int pl = tid - NT;
+        int st = 0;
+        uint32_t parity = 1;  // parity of the "empty" phase to wait for
+        for (int it = 0;; ++it) {
+            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+            if (gi >= pp.ngroups) break;
+            const int64_t t0 = gi * G;
+            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+            const uint32_t lp_bytes = (uint32_t)((((size_t)rows * (E - k) / 2) + 15) & ~(size_t)15);
+            const uint32_t hp_bytes = (uint32_t)rows * k * 2u;
+            const uint32_t bar = smem_u32(&full[st]);
+            uint8_t *stage = smem + (size_t)st * lay.stage;
+            int ok = 1;
+            if (pl == 0) {
                 if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
                     atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
-                    break;
+                    ok = 0;
+                } else {
+                    mbar_expect_tx(bar, (uint32_t)N * (lp_bytes + hp_bytes));
                 }
-                const int64_t t0 = gi * G;
-                const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-                const uint32_t lp_bytes = (uint32_t)((((size_t)rows * (E - k) / 2) + 15) & ~(size_t)15);
-                const uint32_t hp_bytes = (uint32_t)rows * k * 2u;
-                const uint32_t bar = smem_u32(&full[st]);
-                uint8_t *stage = smem + (size_t)st * lay.stage;
-                mbar_expect_tx(bar, (uint32_t)N * (lp_bytes + hp_bytes));
-                for (int i = 0; i < N; ++i) {
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            for (int c = pl; c < 2 * N; c += 32) {
+                const int i = c >> 1;
+                if ((c & 1) == 0)
                     bulk_g2s(smem_u32(stage + (size_t)i * lay.lp_stage), p.pl[i] + t0 * ((E - k) / 2), lp_bytes, bar);
-                    if (hp_bytes)
-                        bulk_g2s(smem_u32(stage + (size_t)N * lay.lp_stage + (size_t)i * lay.hp_stage),
-                                 p.pl[i] + p.lp_bytes + t0 * k * 2, hp_bytes, bar);
-                }
-                if (++st == nstage) {
-                    st = 0;
-                    parity ^= 1u;
-                }
+                else if (hp_bytes)
+                    bulk_g2s(smem_u32(stage + (size_t)N * lay.lp_stage + (size_t)i * lay.hp_stage),
+                             p.pl[i] + p.lp_bytes + t0 * k * 2, hp_bytes, bar);
+            }
+            if (++st == nstage) {
+                st = 0;
+                parity ^= 1u;
             }
         }
         return;
     }
 
     // ---------------- consumers
+    // Holes are completed warp-cooperatively.  The holes of a warp's 32 groups are consecutive in the
+    // hole order, so lane i takes the warp's i-th hole: it sums the selected feature's BF16 values
+    // (output column hole[], the hole itself) and decodes the filler feature whose codes the hole's
+    // slot holds (output column filler[]).  It stores both after a __syncwarp() that orders them behind
+    // the owner's 128-bit row store, which wrote a placeholder (0) at the hole.  A warp with more than
+    // 32 holes and the ragged last stage take the serial path.
+    const int lane = tid & 31;
+    int n_wh, c_rank = 0, c_hole = 0, c_fill = 0;
+    float c_sc[NMAX];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) c_sc[i] = 0.0f;
+    bool serial;
+    {
+        int tot = nh;
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, d);
+        n_wh = tot;
+        serial = n_wh > 32;
+        const int first = __shfl_sync(0xffffffffu, hb, 0);
+        if (lane < n_wh && !serial) {
+            c_rank = first + lane;
+            c_hole = __ldg(x.hole + c_rank);
+            c_fill = __ldg(x.filler + c_rank);
+#pragma unroll
+            for (int i = 0; i < NMAX; ++i)
+                if (i < N) c_sc[i] = __ldg(p.s_k + (size_t)i * E + c_fill);
+        }
+    }
+    const int c_word = c_hole >> 3;
+    const int c_shift = (c_hole & 7) * 4;
+    TPQ_DMARK(1);
+
     int st = 0;
     uint32_t parity = 0;
     for (int it = 0;; ++it) {
@@ -402,10 +460,65 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
             atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
+        TPQ_DMARK(2 + 3 * it);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
         const uint8_t *stage = smem + (size_t)st * lay.stage;
-        if (live) {
+        const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
+        const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
+
+        if (!serial && rows == G) {
+            // ---- full stage, two rows at a time, straight-line: 2 x N devices of independent work
+            for (int r0 = 0; r0 < G; r0 += 2) {
+                float2 acc[2][4];
+                float hv[2], fv[2];
+#pragma unroll
+                for (int r = 0; r < 2; ++r) {
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
+                    hv[r] = 0.0f;
+                    fv[r] = 0.0f;
+                }
+#pragma unroll
+                for (int i = 0; i < NMAX; ++i) {
+                    if (i < N) {  // uniform
+                        const uint32_t *lp = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage);
+                        uint32_t w[2];
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) w[r] = lp[(r0 + r) * L8 + g_ld];
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) decode8(w[r], sc[i], acc[r]);
+                        if (lane < n_wh) {  // "my" hole: the selected feature's value and the filler's code
+#pragma unroll
+                            for (int r = 0; r < 2; ++r) {
+                                const uint32_t hx = hp[i * hp_dev + (r0 + r) * k + c_rank];
+                                const uint32_t cw = lp[(r0 + r) * L8 + c_word];
+                                hv[r] = __fadd_rn(hv[r], __uint_as_float(hx << 16));
+                                const float code = __fsub_rn(
+                                    __uint_as_float((((cw >> c_shift) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
+                                fv[r] = __fmaf_rn(code, c_sc[i], fv[r]);
+                            }
+                        }
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < 2; ++r)
+                    if (live) store_group<FP32OUT>(p.out, (t0 + r0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
+                if (n_wh) {  // uniform over the warp
+                    __syncwarp();
+                    if (lane < n_wh) {
+#pragma unroll
+                        for (int r = 0; r < 2; ++r) {
+                            const int64_t orow = (t0 + r0 + r) * p.out_stride;
+                            store_one<FP32OUT>(p.out, orow + c_hole, hv[r]);
+                            store_one<FP32OUT>(p.out, orow + c_fill, fv[r]);
+                        }
+                    }
+                }
+            }
+        } else if (live) {
+            // ---- serial path: element-wise; the owner of a hole sums the selected feature's BF16 values
+            // and decodes the filler feature whose codes the hole's slot holds
             for (int r = 0; r < rows; ++r) {
                 float2 acc[4];
 #pragma unroll
@@ -415,40 +528,41 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
                     if (i < N)
                         decode8(reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + g], sc[i],
                                 acc);
-                store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc, mask);
-            }
-        }
-        // filler features: one code per device, from the slot they fill
-        for (int tau = tid; tau < x.n_holes; tau += NT) {
-            const bool mine = tau == tid;
-            const int j = mine ? my_fill : __ldg(x.filler + tau);
-            const int slot = mine ? my_slot : __ldg(x.hole + tau);
-            for (int r = 0; r < rows; ++r) {
-                float acc = 0.0f;
-#pragma unroll
-                for (int i = 0; i < NMAX; ++i)
-                    if (i < N) {
-                        const uint32_t w =
-                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + (slot >> 3)];
-                        const int code = (int)(((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) - 8;
-                        acc = __fmaf_rn((float)code, mine ? fsc[i] : __ldg(p.s_k + (size_t)i * E + j), acc);
+                const int64_t orow = (t0 + r) * p.out_stride;
+                const int64_t o = orow + 8 * (int64_t)g;
+                store_group<FP32OUT>(p.out, o, acc, mask);
+                uint32_t m = mask;
+                for (int h = hb; m; ++h) {
+                    const int n = __ffs(m) - 1;
+                    m &= m - 1;
+                    float v = 0.0f, f = 0.0f;
+                    const int fcol = __ldg(x.filler + h);
+                    for (int i = 0; i < N; ++i) {
+                        v = __fadd_rn(v, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
+                        const uint32_t w = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + g];
+                        const int code = (int)(((w >> (n * 4)) & 0xFu) ^ 8u) - 8;
+                        f = __fmaf_rn((float)code, __ldg(p.s_k + (size_t)i * E + fcol), f);
                     }
-                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + j, acc);
+                    store_one<FP32OUT>(p.out, o + n, v);
+                    store_one<FP32OUT>(p.out, orow + fcol, f);
+                }
             }
         }
-        // selected features: sum of the BF16 values, devices ascending
-        for (int h = tid; h < k; h += NT) {
-            const int j = (h == tid) ? my_hp : __ldg(x.hp_idx + h);
-            const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
+        TPQ_DMARK(3 + 3 * it);
+        // ---- tail job: selected features at or above L
+        for (int t = tail_t; t < n_tail; t += NT) {
+            const int rank = x.n_holes + t;
+            const int col = (t == tail_t) ? tail_col : __ldg(x.hp_idx + rank);
             for (int r = 0; r < rows; ++r) {
                 float acc = 0.0f;
                 for (int i = 0; i < N; ++i)
-                    acc = __fadd_rn(acc, __uint_as_float((uint32_t)hp[(size_t)i * (lay.hp_stage / 2) + r * k + h] << 16));
-                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + j, acc);
+                    acc = __fadd_rn(acc, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + rank] << 16));
+                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + col, acc);
             }
         }
         __syncwarp();
-        if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
+        if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
+        TPQ_DMARK(4 + 3 * it);
         if (++st == nstage) {
             st = 0;
             parity ^= 1u;
@@ -512,12 +626,11 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
     if (N > 8) return false;
-    if (L8 > (N <= 4 ? 768 : 576)) return false;
+    if (L8 > (N <= 4 ? 768 : 576)) return false;  // consumer threads (register budget per thread)
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
     else if (L8 % 2 == 0) g0 = 2;
-    int G = g0;
-    while (G < 2) G += g0;
+    const int G = g0 < 2 ? 2 : g0;  // 2 or 4 rows per stage, unrolled in the kernel
     if (dr_layout(N, E, k, G, 2).total > (size_t)c->smem_optin) return false;
     const int64_t ngroups = (T + G - 1) / G;
     const int grid = (int)(ngroups < c->sm_count ? ngroups : c->sm_count);
@@ -544,13 +657,20 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
         if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.ngroups, &grid)) {
             pp.q = p;
             pp.x = x;
+#ifdef TPQ_TRACE
+            pp.trace = g_dtrace;
+#endif
             const size_t smem = dr_layout(c->N, c->E, c->k, pp.G, pp.nstage).total;
             const int L8 = (c->E - c->k) / 8;
             int consumers = ((L8 + 31) / 32) * 32;
             if (consumers < 32) consumers = 32;
             const int threads = consumers + 32;
-            cudaError_t e = (c->N <= 4) ? launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st)
-                                        : launch_rows<8, 576>(pp, fp32_out, grid, threads, smem, st);
+            cudaError_t e;
+            if (c->N <= 4)
+                e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, threads, smem, st)
+                                     : launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st);
+            else
+                e = launch_rows<8, 576>(pp, fp32_out, grid, threads, smem, st);
             if (e != cudaSuccess) return e;
             ++*launches;
             return cudaGetLastError();

@@ -251,32 +251,38 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     TPQ_MARK(40);
 
     if (tid >= NT) {
-        // ---------------- producer warp: one lane streams the row groups
-        if (tid == NT) {
-            int st = 0;
-            uint32_t parity = 1;  // parity of the "empty" phase to wait for
-            for (int it = 0;; ++it) {
-                const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-                if (gi >= p.ngroups) break;
+        // ---------------- producer warp: lane 0 waits for the stage and arms its barrier; a contiguous
+        // input is one copy per stage, a strided one is one copy per row, issued by as many lanes at once
+        const int pl = tid - NT;
+        int st = 0;
+        uint32_t parity = 1;  // parity of the "empty" phase to wait for
+        for (int it = 0;; ++it) {
+            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+            if (gi >= p.ngroups) break;
+            const int64_t t0 = gi * G;
+            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+            const uint32_t bar = smem_u32(&full[st]);
+            const uint32_t dst = smem_u32(ring + (size_t)st * stage_bytes);
+            int ok = 1;
+            if (pl == 0) {
                 if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
                     atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
-                    break;
-                }
-                const int64_t t0 = gi * G;
-                const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-                const uint32_t bar = smem_u32(&full[st]);
-                const uint32_t dst = smem_u32(ring + (size_t)st * stage_bytes);
-                mbar_expect_tx(bar, rows * row_bytes);
-                if (p.stride == E) {
-                    bulk_g2s(dst, p.y + t0 * p.stride, rows * row_bytes, bar);
+                    ok = 0;
                 } else {
-                    for (int r = 0; r < rows; ++r)
-                        bulk_g2s(dst + r * row_bytes, p.y + (t0 + r) * p.stride, row_bytes, bar);
+                    mbar_expect_tx(bar, rows * row_bytes);
                 }
-                if (++st == nstage) {
-                    st = 0;
-                    parity ^= 1u;
-                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            if (p.stride == E) {
+                if (pl == 0) bulk_g2s(dst, p.y + t0 * p.stride, rows * row_bytes, bar);
+            } else {
+                for (int r = pl; r < rows; r += 32)
+                    bulk_g2s(dst + r * row_bytes, p.y + (t0 + r) * p.stride, row_bytes, bar);
+            }
+            if (++st == nstage) {
+                st = 0;
+                parity ^= 1u;
             }
         }
         return;
