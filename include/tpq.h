@@ -97,6 +97,28 @@ tpq_status tpq_set_option(tpq_ctx *ctx, tpq_option opt, int value);
 tpq_status tpq_calibrate_ranges(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t n_seq, int64_t S,
                                 int64_t row_stride_elems, void *cuda_stream);
 
+/* The same fold as tpq_calibrate_ranges, for callers that must not allocate.  (The paper has no
+ * counterpart: this is a deployment variant of the call above.)  tpq_calibrate_ranges may grow its
+ * scratch buffer with cudaMalloc / cudaFree, which a caller cannot afford when it runs inside a
+ * serving loop whose device memory is owned by a pool, under a framework that forbids allocation
+ * outside start-up, or at a point where the implicit device synchronisation of cudaFree would stall
+ * other streams.  This variant keeps the per-sequence column extremes in a fixed array that is part
+ * of the library image: TPQ_NOALLOC_SCRATCH_MAX_BYTES (4 MiB) of global memory on every device that
+ * loads the library, held until the process exits.  It calls no cudaMalloc, no cudaFree and no
+ * allocating library routine.
+ *   Limit: 4 * n_seq * E bytes must fit the array, i.e. n_seq * E <= 1 048 576 (e.g. 204 sequences at
+ *   E = 5120) and n_seq <= 65535; larger calls return TPQ_ERR_SIZE and enqueue nothing: fold fewer
+ *   sequences per call (the result does not depend on how the sequences are split over calls).
+ *   The first call on a device looks up the array's device address (cudaGetSymbolAddress); make that
+ *   first call before any stream capture begins.  The device the context was created on must be current.
+ *   All calls, from every context, share the one array per device: two calls whose kernels can overlap
+ *   on the GPU (different streams) race on it; serialise them on one stream or with events.  Nothing
+ *   in the array has to be cleared between calls: every element a call reads it has written first.
+ * Same arguments, results and errors as tpq_calibrate_ranges otherwise. */
+#define TPQ_NOALLOC_SCRATCH_MAX_BYTES (4u << 20)
+tpq_status tpq_calibrate_ranges_noalloc(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t n_seq, int64_t S,
+                                        int64_t row_stride_elems, void *cuda_stream);
+
 /* Section 3 "Selecting High Precision Features": R^(i)_j = 2 max(-m, M),
  * aggregated range Rbar_j = sum_i R^(i)_j (binary32, devices ascending), the
  * k features with the largest Rbar_j (ties: lower index) become the BF16 set;

@@ -35,6 +35,7 @@ SIGNATURES = {
     "tpq_destroy": (c_int, [c_void_p]),
     "tpq_set_option": (c_int, [c_void_p, c_int, c_int]),
     "tpq_calibrate_ranges": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, c_int64, c_void_p]),
+    "tpq_calibrate_ranges_noalloc": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, c_int64, c_void_p]),
     "tpq_select_features": (c_int, [c_void_p, c_int, POINTER(c_int32), POINTER(c_int)]),
     "tpq_set_features": (c_int, [c_void_p, POINTER(c_int32), c_int]),
     "tpq_set_ranges": (c_int, [c_void_p, POINTER(c_float), POINTER(c_float), POINTER(c_int64)]),
@@ -122,6 +123,13 @@ class Tpq:
                          stream: int = 0):
         self._check(lib().tpq_calibrate_ranges(self._h, shard, y_ptr, n_seq, S,
                                                self.E if row_stride is None else row_stride, stream))
+
+    def calibrate_ranges_noalloc(self, shard: int, y_ptr: int, n_seq: int, S: int, row_stride: int | None = None,
+                                 stream: int = 0):
+        """tpq_calibrate_ranges for callers that must not allocate: the scratch is a fixed 4 MiB array
+        inside the library (n_seq * E <= 1 048 576 per call); see include/tpq.h."""
+        self._check(lib().tpq_calibrate_ranges_noalloc(self._h, shard, y_ptr, n_seq, S,
+                                                       self.E if row_stride is None else row_stride, stream))
 
     def select_features(self, k: int = -1) -> np.ndarray:
         out = np.zeros(self.E, np.int32)

@@ -206,3 +206,44 @@ cudaError_t tpq_launch_calibrate(const uint16_t *y, int64_t n_seq, int64_t S, in
     ++*launches;
     return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant of the calibration pass.
+//
+// Same kernels as above; the partial-extremes scratch is this fixed array, resident in the global
+// memory of every device that loads the library until the process exits.  Its address is looked up
+// once per device with cudaGetSymbolAddress (the array's name is only a host-side handle, never a
+// device address) and handed to the kernels like any other scratch pointer.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) int16_t g_calib_static_scratch[TPQ_NOALLOC_SCRATCH_BYTES / sizeof(int16_t)];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];  // device address of the array, per device ordinal (set-up once)
+bool g_static_scratch_ready[kMaxDevices];
+}  // namespace
+
+cudaError_t tpq_static_scratch_address(int device, void **ptr_out)
+{
+    if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!g_static_scratch_ready[device]) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);  // for the CURRENT device
+        if (e != cudaSuccess) return e;
+        g_static_scratch_ptr[device] = ptr;
+        g_static_scratch_ready[device] = true;
+    }
+    *ptr_out = g_static_scratch_ptr[device];
+    return cudaSuccess;
+}
+
+// Largest row-split count (<= the usual choice) whose partial extremes fit the static array; 0 if none.
+int tpq_static_scratch_splits(int64_t n_seq, int64_t S, int E, int sm_count)
+{
+    int ns = pick_splits(n_seq, S, E, sm_count);
+    const size_t per_split = (size_t)2 * (size_t)n_seq * E * sizeof(int16_t);
+    if (per_split == 0 || per_split > (size_t)TPQ_NOALLOC_SCRATCH_BYTES) return 0;
+    const size_t fit = (size_t)TPQ_NOALLOC_SCRATCH_BYTES / per_split;
+    if ((size_t)ns > fit) ns = (int)fit;
+    return ns;
+}

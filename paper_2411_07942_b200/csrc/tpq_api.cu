@@ -203,6 +203,36 @@ tpq_status tpq_calibrate_ranges(tpq_ctx *c, int shard, const void *y, int64_t n_
     return TPQ_OK;
 }
 
+tpq_status tpq_calibrate_ranges_noalloc(tpq_ctx *c, int shard, const void *y, int64_t n_seq, int64_t S, int64_t stride,
+                                        void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (shard < 0 || shard >= c->N) return fail(c, TPQ_ERR_INVALID_ARG, "shard %d out of range [0, %d)", shard, c->N);
+    if (n_seq < 0 || S < 1) return fail(c, TPQ_ERR_INVALID_ARG, "n_seq must be >= 0 and S >= 1");
+    if (n_seq == 0) return TPQ_OK;
+    if (!y) return fail(c, TPQ_ERR_INVALID_ARG, "y is NULL");
+    if (stride < c->E) return fail(c, TPQ_ERR_INVALID_ARG, "row stride %lld < E", (long long)stride);
+    if (reinterpret_cast<uintptr_t>(y) & 1u) return fail(c, TPQ_ERR_ALIGN, "y is not 2-byte aligned");
+    if (n_seq > 65535) return fail(c, TPQ_ERR_SIZE, "at most 65535 sequences per call");
+    const int n_split = tpq_static_scratch_splits(n_seq, S, c->E, c->sm_count);
+    if (n_split < 1)
+        return fail(c, TPQ_ERR_SIZE,
+                    "n_seq * E = %lld exceeds the built-in scratch (%u bytes hold n_seq * E <= %u): "
+                    "fold fewer sequences per call",
+                    (long long)(n_seq * c->E), (unsigned)TPQ_NOALLOC_SCRATCH_BYTES,
+                    (unsigned)(TPQ_NOALLOC_SCRATCH_BYTES / 4));
+    void *scratch = nullptr;
+    cudaError_t e = tpq_static_scratch_address(c->device, &scratch);  // first call on a device: symbol look-up
+    if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetSymbolAddress(static scratch)");
+    float *m = c->t.m + (size_t)shard * c->E, *M = c->t.M + (size_t)shard * c->E;
+    e = tpq_launch_calibrate(static_cast<const uint16_t *>(y), n_seq, S, stride, c->E, m, M, c->counts[shard], c->gamma,
+                             scratch, n_split, static_cast<cudaStream_t>(stream), &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e, "calibration kernels");
+    c->counts[shard] += n_seq;
+    return TPQ_OK;
+}
+
 tpq_status tpq_select_features(tpq_ctx *c, int k, int32_t *hp_out, int *k_out)
 {
     if (!c) return TPQ_ERR_INVALID_ARG;

@@ -64,6 +64,11 @@ cudaError_t tpq_launch_calibrate(const uint16_t *y, int64_t n_seq, int64_t S, in
                                  float *M, int64_t count0, float gamma, void *scratch, int n_split, cudaStream_t st,
                                  int64_t *launches);
 
+// Allocation-free calibration: fixed scratch array inside the library (see calibrate.cu).
+#define TPQ_NOALLOC_SCRATCH_BYTES TPQ_NOALLOC_SCRATCH_MAX_BYTES  /* tpq.h */
+cudaError_t tpq_static_scratch_address(int device, void **ptr_out);
+int tpq_static_scratch_splits(int64_t n_seq, int64_t S, int E, int sm_count);
+
 // Section 3: ranges, aggregate, steps; top-k flags (or flags given); index tables.
 cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_topk_flags(const tpq_tables &t, int E, int k, cudaStream_t st, int64_t *launches);
