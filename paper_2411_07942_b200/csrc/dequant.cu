@@ -76,7 +76,23 @@ __device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
 // code * 16^n exactly, and the step was pre-divided by 16^n (an exact scaling), so
 // fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 5..7 use raw >> 20.
 // Subtractions and FMAs run two at a time (f32x2), one binary32 rounding per element as before.
-__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4])
+// -(2^23 + 8 * 16^pos) for the code pairs (0,1) (2,3) (4,5) (6,7); in constant memory so that the packed
+// subtract can take the pair as an operand instead of rebuilding it in registers
+__constant__ float2 kDecodeBias[4] = {{-8388616.0f, -8388736.0f},      // 16^0, 16^1
+                                      {-8390656.0f, -8421376.0f},      // 16^2, 16^3
+                                      {-8912896.0f, -8388616.0f},      // 16^4, 16^0 (codes 5..7 use raw >> 20)
+                                      {-8388736.0f, -8390656.0f}};     // 16^1, 16^2
+
+// `magic` must hold 0x4B000000 in a REGISTER (see opaque_magic): with both the mask and the exponent as
+// immediates the (x & mask) | magic of every code would take two logic instructions instead of one.
+__device__ __forceinline__ uint32_t opaque_magic()
+{
+    uint32_t m;
+    asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(m));
+    return m;
+}
+
+__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], uint32_t magic)
 {
     const uint32_t xa = raw ^ 0x88888888u;
     const uint32_t xb = xa >> 20;
@@ -84,11 +100,9 @@ __device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], flo
     for (int h = 0; h < 4; ++h) {
         const int n0 = 2 * h, n1 = 2 * h + 1;
         const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
-        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | 0x4B000000u);
-        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | 0x4B000000u);
-        const float c0 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n0))));
-        const float c1 = -(8388608.0f + 8.0f * (float)(1 << (4 * dq_pos(n1))));
-        const float2 d = __fadd2_rn(make_float2(f0, f1), make_float2(c0, c1));
+        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | magic);
+        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | magic);
+        const float2 d = __fadd2_rn(make_float2(f0, f1), kDecodeBias[h]);
         acc[h] = __ffma2_rn(d, sc[h], acc[h]);
     }
 }
@@ -198,6 +212,7 @@ __global__ void __launch_bounds__(128) dequant_strips(const DQParams p, const DX
     if (g >= L8) return;
     const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
     const bool single = p.N <= NC;
+    const uint32_t magic = opaque_magic();
     float2 sc[NC][4];
     if (single) {
 #pragma unroll
@@ -233,7 +248,7 @@ __global__ void __launch_bounds__(128) dequant_strips(const DQParams p, const DX
             for (int r = 0; r < R; ++r)
 #pragma unroll
                 for (int i = 0; i < NC; ++i)
-                    if (t0 + r < p.T && i0 + i < p.N) decode8(w[r][i], sc[i], acc[r]);
+                    if (t0 + r < p.T && i0 + i < p.N) decode8(w[r][i], sc[i], acc[r], magic);
         }
 #pragma unroll
         for (int r = 0; r < R; ++r)
@@ -242,15 +257,25 @@ __global__ void __launch_bounds__(128) dequant_strips(const DQParams p, const DX
 }
 
 // ----------------------------------------------------------------------------------------------
-// Row kernel for N <= 8 devices and E/8 <= MAXT consumer threads.
+// Row kernel for N <= 8 devices and (E-k)/8 <= MAXT main threads.
 //
-// One persistent block per SM; a producer warp streams groups of G rows of all N payloads (code rows
-// and BF16 rows) into a ring of shared-memory stages with 1-D bulk asynchronous copies, completion on
-// "full" mbarriers; consumer warps release a stage through an "empty" mbarrier, so there is no
-// block-wide barrier in the loop.  Thread <-> 8 adjacent output features for every row: its N x 8
-// steps live in registers for the life of the block.  G is a multiple of 4/gcd(4, L/8) so that every
-// stage starts 16-byte aligned in the code stream.
+// One persistent block per SM with three kinds of warps:
+//   producer (1 warp)  streams groups of G rows of all N payloads (a code-row block and a BF16 block per
+//                      device, 2N 1-D bulk asynchronous copies issued by 2N lanes) into a ring of
+//                      shared-memory stages; completion on "full" mbarriers;
+//   main (MAXT/32)     thread <-> 8 adjacent output features = one aligned word per device and row; its
+//                      N x 8 steps live in registers for the life of the block (0 at holes); pure
+//                      decode + 128-bit row stores, two rows at a time, no hole logic at all; arrives on
+//                      "main_done" (release: its stores are ordered before what follows the barrier);
+//   fix-up (4 warps)   after "main_done": one item per selected feature and row -- the sum of the
+//                      devices' BF16 values goes to the selected feature's column (overwriting the 0 the
+//                      main store left at a hole), and, for a hole, the filler feature whose codes the
+//                      hole's slot holds is decoded and stored to the filler's column.
+// Main and fix-up warps release a stage through the "empty" mbarrier; no block-wide barrier in the loop.
+// G is a multiple of 4/gcd(4, L/8) so that every stage starts 16-byte aligned in the code stream.
 // ----------------------------------------------------------------------------------------------
+constexpr int DR_FIXUP_THREADS = 128;
+
 struct DRLayout {
     size_t lp_stage, hp_stage, stage, bars, total;
 };
@@ -261,7 +286,7 @@ __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int ns
     l.hp_stage = (size_t)G * k * 2;
     l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
     l.bars = (size_t)nstage * l.stage;
-    l.total = l.bars + (size_t)nstage * 16;
+    l.total = l.bars + (size_t)nstage * 24;
     return l;
 }
 
@@ -324,43 +349,37 @@ __device__ __forceinline__ long long tpq_dnow()
 #endif
 
 template <int NMAX, int MAXT, bool FP32OUT>
-__global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
+__global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     TPQ_DMARK(0);
     const DQParams &p = pp.q;
     const DXParams &x = pp.x;
     const int tid = threadIdx.x;
-    const int NT = blockDim.x - 32;  // consumer threads
+    const int NT = blockDim.x - DR_FIXUP_THREADS - 32;  // main threads; then the fix-up warps; then the producer warp
     const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;  // G rows per stage, even
     const int L = E - k, L8 = L >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
     uint64_t *empty = full + nstage;
+    uint64_t *main_done = empty + nstage;
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), NT / 32);
+            mbar_init(smem_u32(&empty[s]), (NT + DR_FIXUP_THREADS) / 32);
+            mbar_init(smem_u32(&main_done[s]), NT / 32);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
 
-    // consumer constants: loads issued before the barrier that releases the producer (so that they
+    // main-thread constants: loads issued before the barrier that releases the producer (so that they
     // are not queued behind the bulk copies)
     const int g = tid;
-    const bool live = tid < NT && g < L8;
+    const bool is_main = tid < NT;
+    const bool live = is_main && g < L8;
     const int g_ld = live ? g : 0;
-    uint32_t mask = 0;
-    int hb = 0;
-    if (live) {
-        const uint32_t gd = __ldg(p.grp + g);
-        mask = gd & 0xFFu;
-        hb = (int)(gd >> 8);
-    }
-    // steps of the thread's 8 slots; 0 where the slot's own feature is a selected one (a hole)
-    const int nh = __popc(mask);
     float2 sc[NMAX][4];
 #pragma unroll
     for (int i = 0; i < NMAX; ++i) {
@@ -368,18 +387,12 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
         for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
     }
-    // tail job: the selected features at or above L (ranks n_holes .. k-1; about one per row on
-    // average) are summed by the LAST consumer threads, one feature each
-    const int n_tail = k - x.n_holes;
-    const int tail_t = NT - 1 - tid;
-    int tail_col = 0;
-    if (tid < NT && tail_t < n_tail) tail_col = __ldg(x.hp_idx + x.n_holes + tail_t);
     __syncthreads();
 
-    if (tid >= NT) {
+    if (tid >= NT + DR_FIXUP_THREADS) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
-        // copies of the stage (a code-row block and a BF16 block per device) are issued by 2N lanes at once
-        const int pl = tid - NT;
+        // copies of the stage are issued by 2N lanes at once
+        const int pl = tid - NT - DR_FIXUP_THREADS;
         int st = 0;
         uint32_t parity = 1;  // parity of the "empty" phase to wait for
         for (int it = 0;; ++it) {
@@ -418,41 +431,58 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
         return;
     }
 
-    // ---------------- consumers
-    // Holes are completed warp-cooperatively.  The holes of a warp's 32 groups are consecutive in the
-    // hole order, so lane i takes the warp's i-th hole: it sums the selected feature's BF16 values
-    // (output column hole[], the hole itself) and decodes the filler feature whose codes the hole's
-    // slot holds (output column filler[]).  It stores both after a __syncwarp() that orders them behind
-    // the owner's 128-bit row store, which wrote a placeholder (0) at the hole.  A warp with more than
-    // 32 holes and the ragged last stage take the serial path.
     const int lane = tid & 31;
-    int n_wh, c_rank = 0, c_hole = 0, c_fill = 0;
-    float c_sc[NMAX];
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) c_sc[i] = 0.0f;
-    bool serial;
-    {
-        int tot = nh;
-#pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, d);
-        n_wh = tot;
-        serial = n_wh > 32;
-        const int first = __shfl_sync(0xffffffffu, hb, 0);
-        if (lane < n_wh && !serial) {
-            c_rank = first + lane;
-            c_hole = __ldg(x.hole + c_rank);
-            c_fill = __ldg(x.filler + c_rank);
-#pragma unroll
-            for (int i = 0; i < NMAX; ++i)
-                if (i < N) c_sc[i] = __ldg(p.s_k + (size_t)i * E + c_fill);
-        }
-    }
-    const int c_word = c_hole >> 3;
-    const int c_shift = (c_hole & 7) * 4;
-    TPQ_DMARK(1);
-
     int st = 0;
     uint32_t parity = 0;
+
+    if (!is_main) {
+        // ---------------- fix-up warps
+        const int ft = tid - NT;
+        for (int it = 0;; ++it) {
+            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+            if (gi >= pp.ngroups) break;
+            if (!mbar_wait(smem_u32(&full[st]), parity) || !mbar_wait(smem_u32(&main_done[st]), parity)) {
+                atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
+                break;
+            }
+            const int64_t t0 = gi * G;
+            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+            const uint8_t *stage = smem + (size_t)st * lay.stage;
+            const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
+            const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
+            for (int item = ft; item < rows * k; item += DR_FIXUP_THREADS) {
+                const int r = item / k, h = item - r * k;  // row of the stage, rank of the selected feature
+                const int64_t orow = (t0 + r) * p.out_stride;
+                float hv = 0.0f;
+                for (int i = 0; i < N; ++i)
+                    hv = __fadd_rn(hv, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
+                store_one<FP32OUT>(p.out, orow + __ldg(x.hp_idx + h), hv);
+                if (h < x.n_holes) {  // the hole's slot holds the codes of filler feature h
+                    const int slot = __ldg(x.hole + h), col = __ldg(x.filler + h);
+                    float fv = 0.0f;
+                    for (int i = 0; i < N; ++i) {
+                        const uint32_t w =
+                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + (slot >> 3)];
+                        const float code = __fsub_rn(
+                            __uint_as_float((((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
+                        fv = __fmaf_rn(code, __ldg(p.s_k + (size_t)i * E + col), fv);
+                    }
+                    store_one<FP32OUT>(p.out, orow + col, fv);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
+            if (++st == nstage) {
+                st = 0;
+                parity ^= 1u;
+            }
+        }
+        return;
+    }
+
+    // ---------------- main warps
+    const uint32_t magic = opaque_magic();
+    TPQ_DMARK(1);
     for (int it = 0;; ++it) {
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
         if (gi >= pp.ngroups) break;
@@ -460,109 +490,39 @@ __global__ void __launch_bounds__(MAXT + 32, 1) dequant_rows(const DRParams pp)
             atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
-        TPQ_DMARK(2 + 3 * it);
+        TPQ_DMARK(2 + 2 * it);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
         const uint8_t *stage = smem + (size_t)st * lay.stage;
-        const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
-        const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
-
-        if (!serial && rows == G) {
-            // ---- full stage, two rows at a time, straight-line: 2 x N devices of independent work
-            for (int r0 = 0; r0 < G; r0 += 2) {
-                float2 acc[2][4];
-                float hv[2], fv[2];
+        for (int r0 = 0; r0 < rows; r0 += 2) {
+            const bool two = r0 + 1 < rows;
+            const int r1 = two ? r0 + 1 : r0;  // a ragged last stage decodes its last row twice, stores it once
+            float2 acc[2][4];
 #pragma unroll
-                for (int r = 0; r < 2; ++r) {
+            for (int r = 0; r < 2; ++r)
 #pragma unroll
-                    for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-                    hv[r] = 0.0f;
-                    fv[r] = 0.0f;
-                }
+                for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
 #pragma unroll
-                for (int i = 0; i < NMAX; ++i) {
-                    if (i < N) {  // uniform
-                        const uint32_t *lp = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage);
-                        uint32_t w[2];
-#pragma unroll
-                        for (int r = 0; r < 2; ++r) w[r] = lp[(r0 + r) * L8 + g_ld];
-#pragma unroll
-                        for (int r = 0; r < 2; ++r) decode8(w[r], sc[i], acc[r]);
-                        if (lane < n_wh) {  // "my" hole: the selected feature's value and the filler's code
-#pragma unroll
-                            for (int r = 0; r < 2; ++r) {
-                                const uint32_t hx = hp[i * hp_dev + (r0 + r) * k + c_rank];
-                                const uint32_t cw = lp[(r0 + r) * L8 + c_word];
-                                hv[r] = __fadd_rn(hv[r], __uint_as_float(hx << 16));
-                                const float code = __fsub_rn(
-                                    __uint_as_float((((cw >> c_shift) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
-                                fv[r] = __fmaf_rn(code, c_sc[i], fv[r]);
-                            }
-                        }
-                    }
-                }
-#pragma unroll
-                for (int r = 0; r < 2; ++r)
-                    if (live) store_group<FP32OUT>(p.out, (t0 + r0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
-                if (n_wh) {  // uniform over the warp
-                    __syncwarp();
-                    if (lane < n_wh) {
-#pragma unroll
-                        for (int r = 0; r < 2; ++r) {
-                            const int64_t orow = (t0 + r0 + r) * p.out_stride;
-                            store_one<FP32OUT>(p.out, orow + c_hole, hv[r]);
-                            store_one<FP32OUT>(p.out, orow + c_fill, fv[r]);
-                        }
-                    }
+            for (int i = 0; i < NMAX; ++i) {
+                if (i < N) {  // uniform
+                    const uint32_t *lp = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage);
+                    const uint32_t w0 = lp[r0 * L8 + g_ld];
+                    const uint32_t w1 = lp[r1 * L8 + g_ld];
+                    decode8(w0, sc[i], acc[0], magic);
+                    decode8(w1, sc[i], acc[1], magic);
                 }
             }
-        } else if (live) {
-            // ---- serial path: element-wise; the owner of a hole sums the selected feature's BF16 values
-            // and decodes the filler feature whose codes the hole's slot holds
-            for (int r = 0; r < rows; ++r) {
-                float2 acc[4];
-#pragma unroll
-                for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
-#pragma unroll
-                for (int i = 0; i < NMAX; ++i)
-                    if (i < N)
-                        decode8(reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + g], sc[i],
-                                acc);
-                const int64_t orow = (t0 + r) * p.out_stride;
-                const int64_t o = orow + 8 * (int64_t)g;
-                store_group<FP32OUT>(p.out, o, acc, mask);
-                uint32_t m = mask;
-                for (int h = hb; m; ++h) {
-                    const int n = __ffs(m) - 1;
-                    m &= m - 1;
-                    float v = 0.0f, f = 0.0f;
-                    const int fcol = __ldg(x.filler + h);
-                    for (int i = 0; i < N; ++i) {
-                        v = __fadd_rn(v, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
-                        const uint32_t w = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + g];
-                        const int code = (int)(((w >> (n * 4)) & 0xFu) ^ 8u) - 8;
-                        f = __fmaf_rn((float)code, __ldg(p.s_k + (size_t)i * E + fcol), f);
-                    }
-                    store_one<FP32OUT>(p.out, o + n, v);
-                    store_one<FP32OUT>(p.out, orow + fcol, f);
-                }
-            }
-        }
-        TPQ_DMARK(3 + 3 * it);
-        // ---- tail job: selected features at or above L
-        for (int t = tail_t; t < n_tail; t += NT) {
-            const int rank = x.n_holes + t;
-            const int col = (t == tail_t) ? tail_col : __ldg(x.hp_idx + rank);
-            for (int r = 0; r < rows; ++r) {
-                float acc = 0.0f;
-                for (int i = 0; i < N; ++i)
-                    acc = __fadd_rn(acc, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + rank] << 16));
-                store_one<FP32OUT>(p.out, (t0 + r) * p.out_stride + col, acc);
+            if (live) {
+                store_group<FP32OUT>(p.out, (t0 + r0) * p.out_stride + 8 * (int64_t)g, acc[0], 0u);
+                if (two) store_group<FP32OUT>(p.out, (t0 + r1) * p.out_stride + 8 * (int64_t)g, acc[1], 0u);
             }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
-        TPQ_DMARK(4 + 3 * it);
+        if (lane == 0) {
+            mbar_arrive(smem_u32(&main_done[st]));  // release: the row stores above precede the fix-up stores
+            mbar_arrive(smem_u32(&empty[st]));
+        }
+        TPQ_DMARK(3 + 2 * it);
         if (++st == nstage) {
             st = 0;
             parity ^= 1u;
@@ -664,7 +624,7 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             const int L8 = (c->E - c->k) / 8;
             int consumers = ((L8 + 31) / 32) * 32;
             if (consumers < 32) consumers = 32;
-            const int threads = consumers + 32;
+            const int threads = consumers + DR_FIXUP_THREADS + 32;
             cudaError_t e;
             if (c->N <= 4)
                 e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, threads, smem, st)
