@@ -43,7 +43,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"quantize_tiled": None, "dequant_tiled": None}
+NCU_TRAFFIC_BYTES = {"quantize_tiled": 21027584, "dequant_tiled": 22072320}
 
 
 # ------------------------------------------------------------------ helpers
