@@ -3,7 +3,9 @@
 
 One "step" = one synchronisation of the Llama-2-13B-shaped prefill workload
 (BASELINE config 2): N = 4 simulated tensor-parallel shards, 2048 tokens x 5120
-features of BF16 partial sums each; tpq_quantize_pack once per shard, then one
+features of BF16 partial sums each; the 4 shards are quantised and packed
+(tpq_quantize_pack_batch: one launch, the SMs divided among the shards; the
+per-shard tpq_quantize_pack is timed too, under "extra"), then one
 tpq_dequant_reduce (BF16 output) over the 4 payloads.  The static parameters
 (calibration + feature selection) are computed once before the timed region,
 as in the method (they never change at inference time); their throughput is
@@ -21,6 +23,7 @@ cores on the same workload; there is no other reference implementation.
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import statistics
@@ -43,7 +46,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"quantize_tiled": 21027584, "dequant_tiled": 22072320}
+NCU_TRAFFIC_BYTES = {"quantize_tiled": 21027584, "quantize_tiled_batch": None, "dequant_rows": 22072320}
 
 
 # ------------------------------------------------------------------ helpers
@@ -267,16 +270,19 @@ def main():
         ys = [synth.activations_torch(w, i, T, dev, stream=2 + b, scale=scale) for i in range(N)]
         pls = [torch.empty(P, dtype=torch.uint8, device=dev) for _ in range(N)]
         out = torch.empty((T, E), dtype=torch.bfloat16, device=dev)
-        sets.append((ys, pls, out))
+        yarr = (ctypes.c_void_p * N)(*[y.data_ptr() for y in ys])
+        parr = (ctypes.c_void_p * N)(*[p_.data_ptr() for p_ in pls])
+        sets.append((ys, pls, out, yarr, parr))
     set_bytes = in_bytes + N * P + 2 * T * E
     config["l2"] = (f"rotating {args.sets} buffer sets, {args.sets * set_bytes / 1e6:.0f} MB touched between "
                     f"reuses (> 126 MB L2)")
 
+    # One step: the N simulated ranks' quantize_pack (one batched launch: the SMs are divided among the
+    # N shards, as N devices would work side by side), then the local dequantise + reduce.
     def step(b):
-        ys, pls, out = sets[b % args.sets]
-        for i in range(N):
-            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
-        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+        _, _, out, yarr, parr = sets[b % args.sets]
+        t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh)
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
 
     def barrier():
         if world > 1:
@@ -317,33 +323,38 @@ def main():
         torch.cuda.synchronize()
         return a.elapsed_time(z) / reps
 
-    def q_only(b):
-        ys, pls, _ = sets[b % args.sets]
+    def q_only(b):          # one launch per shard: what each rank of a real deployment calls
+        ys, pls, _, _, _ = sets[b % args.sets]
         for i in range(N):
             t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
 
+    def qb_only(b):         # the N shards in one launch (the step's form)
+        _, _, _, yarr, parr = sets[b % args.sets]
+        t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh)
+
     def d_only(b):
-        _, pls, out = sets[b % args.sets]
-        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+        _, _, out, _, parr = sets[b % args.sets]
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
 
     reps = max(20, min(args.steps, 200))
-    q_ms = time_loop(q_only, reps) / N          # per launch
+    q_ms = time_loop(q_only, reps) / N          # per single-shard launch
+    qb_ms = time_loop(qb_only, reps)            # per batched launch (N shards)
     d_ms = time_loop(d_only, reps)
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
-    ys0, pls0, out0 = sets[0]
+    ys0 = sets[0][0]
     host_in = [torch.empty((T, E), dtype=torch.bfloat16).pin_memory() for _ in range(N)]
     for i in range(N):
         host_in[i].copy_(ys0[i])
     host_out = torch.empty((T, E), dtype=torch.bfloat16).pin_memory()
 
     def e2e_step(b):
-        ys, pls, out = sets[b % args.sets]
+        ys, _, out, yarr, parr = sets[b % args.sets]
         for i in range(N):
             ys[i].copy_(host_in[i], non_blocking=True)
-            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
-        t.dequant_reduce([p.data_ptr() for p in pls], T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+        t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh)
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
         host_out.copy_(out, non_blocking=True)
 
     e2e_reps = max(5, min(args.steps, 30))
@@ -367,20 +378,29 @@ def main():
         return 0
 
     value = units / (ms * 1e-3) / 1e9
-    dom = "quantize_pack" if N * q_ms >= d_ms else "dequant_reduce"
-    dom_ms = q_ms if dom == "quantize_pack" else d_ms
-    achieved = alg[dom] / (dom_ms * 1e-3) / 1e9
+    # dominant kernel of the step: the batched quantize_tiled launch (N shards) or dequant_rows
+    if qb_ms >= d_ms:
+        dom, dom_ms, dom_bytes = "quantize_pack (batched launch, N shards)", qb_ms, N * alg["quantize_pack"]
+        traffic = NCU_TRAFFIC_BYTES["quantize_tiled_batch"]
+    else:
+        dom, dom_ms, dom_bytes = "dequant_reduce", d_ms, alg["dequant_reduce"]
+        traffic = NCU_TRAFFIC_BYTES["dequant_rows"]
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                 "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "algorithmic_bytes_per_launch": alg[dom], "launch_ms": dom_ms,
-                "traffic": NCU_TRAFFIC_BYTES["quantize_tiled" if dom == "quantize_pack" else "dequant_tiled"]}
+                "algorithmic_bytes_per_launch": dom_bytes, "launch_ms": dom_ms, "traffic": traffic}
     extra = {
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
         "payload_bytes_per_shard": int(comm.payload_bytes),
         "comm_bytes_per_rank": {"quantized_allgather": int(comm.quantized_allgather_send),
                                 "bf16_allgather": int(comm.bf16_allgather_send),
                                 "bf16_ring_allreduce": int(comm.bf16_ring_allreduce_send)},
+        "quantize_pack_batch": {"ms_per_launch": qb_ms, "shards_per_launch": N,
+                                "hbm_GBps": N * alg["quantize_pack"] / qb_ms / 1e6,
+                                "frac_of_measured": N * alg["quantize_pack"] / qb_ms / 1e6 / peak,
+                                "frac_of_8000": N * alg["quantize_pack"] / qb_ms / 1e6 / NOMINAL_HBM_GBS,
+                                "input_GBps": in_bytes / qb_ms / 1e6},
         "quantize_pack": {"ms_per_launch": q_ms, "hbm_GBps": alg["quantize_pack"] / q_ms / 1e6,
                           "frac_of_measured": alg["quantize_pack"] / q_ms / 1e6 / peak,
                           "frac_of_8000": alg["quantize_pack"] / q_ms / 1e6 / NOMINAL_HBM_GBS,

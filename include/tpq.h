@@ -182,6 +182,17 @@ tpq_status tpq_comm_bytes(const tpq_ctx *ctx, int64_t T, tpq_comm_report *out);
 tpq_status tpq_quantize_pack(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t T, int64_t row_stride_elems,
                              void *payload_dev, size_t payload_capacity, void *cuda_stream);
 
+/* The same C^(i) for n consecutive devices first_shard .. first_shard+n-1 in ONE launch, for a process
+ * that holds several devices' partial sums on one GPU (the single-GPU simulation of N ranks; in a real
+ * deployment every rank calls tpq_quantize_pack once).  The SMs are divided among the shards; every payload
+ * is byte-identical to what tpq_quantize_pack writes for that shard.
+ *   ys_dev_host / payloads_dev_host : HOST arrays of n DEVICE pointers (inputs [T][E] with the common row
+ *   stride; payloads of payload_capacity bytes each), all 16-byte aligned.
+ * Enqueues on cuda_stream; T == 0 or n == 0 is a no-op.  Errors as tpq_quantize_pack. */
+tpq_status tpq_quantize_pack_batch(tpq_ctx *ctx, int first_shard, int n, const void *const *ys_dev_host, int64_t T,
+                                   int64_t row_stride_elems, void *const *payloads_dev_host, size_t payload_capacity,
+                                   void *cuda_stream);
+
 /* sum_i D^(i) (Figure 2 caption; Section 5 "local reduction"): N payloads ->
  * the synchronised [T][E] output in the original feature order.
  * Low-precision feature: sum_i code_i * s^(i)_j; selected feature: sum_i of

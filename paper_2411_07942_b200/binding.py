@@ -47,6 +47,8 @@ SIGNATURES = {
     "tpq_payload_bytes_for": (c_size_t, [c_int64, c_int64, c_int64]),
     "tpq_comm_bytes": (c_int, [c_void_p, c_int64, POINTER(CommReport)]),
     "tpq_quantize_pack": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, c_void_p, c_size_t, c_void_p]),
+    "tpq_quantize_pack_batch": (c_int, [c_void_p, c_int, c_int, POINTER(c_void_p), c_int64, c_int64, POINTER(c_void_p),
+                                        c_size_t, c_void_p]),
     "tpq_dequant_reduce": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p]),
     "tpq_get_state": (c_int, [c_void_p, c_void_p, POINTER(c_size_t)]),
     "tpq_set_state": (c_int, [c_void_p, c_void_p, c_size_t]),
@@ -187,9 +189,19 @@ class Tpq:
         self._check(lib().tpq_quantize_pack(self._h, shard, y_ptr, T, self.E if row_stride is None else row_stride,
                                             payload_ptr, payload_capacity, stream))
 
+    def quantize_pack_batch(self, first_shard: int, y_ptrs, T: int, payload_ptrs, payload_capacity: int,
+                            row_stride: int | None = None, stream: int = 0):
+        n = len(y_ptrs)
+        assert len(payload_ptrs) == n
+        ya = y_ptrs if isinstance(y_ptrs, ctypes.Array) else (c_void_p * n)(*y_ptrs)
+        pa = payload_ptrs if isinstance(payload_ptrs, ctypes.Array) else (c_void_p * n)(*payload_ptrs)
+        self._check(lib().tpq_quantize_pack_batch(self._h, first_shard, n, ya, T,
+                                                  self.E if row_stride is None else row_stride, pa,
+                                                  payload_capacity, stream))
+
     def dequant_reduce(self, payload_ptrs, T: int, out_ptr: int, out_dtype: int = TPQ_OUT_BF16,
                        out_row_stride: int | None = None, stream: int = 0):
-        arr = (c_void_p * len(payload_ptrs))(*payload_ptrs)
+        arr = payload_ptrs if isinstance(payload_ptrs, ctypes.Array) else (c_void_p * len(payload_ptrs))(*payload_ptrs)
         self._check(lib().tpq_dequant_reduce(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype,
                                              self.E if out_row_stride is None else out_row_stride, stream))
 

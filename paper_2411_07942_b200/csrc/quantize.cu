@@ -74,21 +74,24 @@ constexpr int QP_MAX_GPT = 4;          // groups of 8 features per thread
 constexpr int QP_MAX_CONSUMERS = 992;  // 31 consumer warps + 1 producer warp per block
 constexpr int QP_WAIT_LIMIT = 1 << 22; // bounded mbarrier polling
 
+constexpr int QP_MAX_BATCH = 16;  // devices' shards quantised by one launch (each by its own set of blocks)
+
 struct QPParams {
-    const uint16_t *y;
+    const uint16_t *y[QP_MAX_BATCH];   // one input per shard of the batch
+    uint8_t *payload[QP_MAX_BATCH];    // and its payload
+    int cps;                           // blocks per shard: block b works on shard b / cps
+    int64_t lp_bytes;                  // size of a payload's code section (the BF16 block follows)
     int64_t stride;
     int64_t T;
     int E, k;
     int G;        // rows per stage
     int nstage;
     int64_t ngroups;
-    const float *inv_s;     // this device's [E]
+    const float *inv_s;     // [E] of the batch's first device; device d of the batch at inv_s + d*E
     const uint32_t *grp;    // [E/8]
     const int32_t *filler;  // [n_holes]
     const int32_t *hp_idx;  // [k]
-    uint32_t *lp_out;
     int64_t lp_words;       // words of the code section, padding included
-    uint16_t *hp_out;
     int *status;
 #ifdef TPQ_TRACE
     long long *trace;
@@ -198,6 +201,13 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     TPQ_MARK(0);
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
+    // this block's shard of the batch, its index among the shard's blocks, and the shard's buffers
+    const int sb = blockIdx.x / p.cps;
+    const int bx = blockIdx.x - sb * p.cps;
+    const uint16_t *const y_in = p.y[sb];
+    uint32_t *const lp_out = reinterpret_cast<uint32_t *>(p.payload[sb]);
+    uint16_t *const hp_out = reinterpret_cast<uint16_t *>(p.payload[sb] + p.lp_bytes);
+    const float *const inv_s = p.inv_s + (size_t)sb * p.E;
     const int E = p.E, k = p.k, nstage = p.nstage;  // G rows per stage, unrolled: G independent chains per thread
     const int E8 = E >> 3, L8 = (E - k) >> 3;
     const uint32_t row_bytes = (uint32_t)E * 2u;
@@ -234,8 +244,8 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
             f_sh[a][0] = f_sh[a][1] = 0;
             hmask[a][0] = hmask[a][1] = 0;
             if (g < L8) {
-                const float4 i0 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g));
-                const float4 i1 = __ldg(reinterpret_cast<const float4 *>(p.inv_s + 8 * g + 4));
+                const float4 i0 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g));
+                const float4 i1 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g + 4));
                 const uint32_t gd = __ldg(p.grp + g);
                 inv[a][0] = make_float2(i0.x, i0.y);
                 inv[a][1] = make_float2(i0.z, i0.w);
@@ -257,7 +267,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         int st = 0;
         uint32_t parity = 1;  // parity of the "empty" phase to wait for
         for (int it = 0;; ++it) {
-            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+            const int64_t gi = bx + it * (int64_t)p.cps;
             if (gi >= p.ngroups) break;
             const int64_t t0 = gi * G;
             const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
@@ -275,10 +285,10 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             if (p.stride == E) {
-                if (pl == 0) bulk_g2s(dst, p.y + t0 * p.stride, rows * row_bytes, bar);
+                if (pl == 0) bulk_g2s(dst, y_in + t0 * p.stride, rows * row_bytes, bar);
             } else {
                 for (int r = pl; r < rows; r += 32)
-                    bulk_g2s(dst + r * row_bytes, p.y + (t0 + r) * p.stride, row_bytes, bar);
+                    bulk_g2s(dst + r * row_bytes, y_in + (t0 + r) * p.stride, row_bytes, bar);
             }
             if (++st == nstage) {
                 st = 0;
@@ -317,7 +327,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         if (lane < n_wh[a] && !serial[a]) {
             const int f = __ldg(p.filler + hb_warp + lane);
             w_off[a] = (uint32_t)f * 2u;
-            w_inv[a] = __ldg(p.inv_s + f);
+            w_inv[a] = __ldg(inv_s + f);
         }
         uint32_t m = mask[a];
         keep[a] = 0xFFFFFFFFu;
@@ -333,7 +343,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     int st = 0;
     uint32_t parity = 0;
     for (int it = 0;; ++it) {
-        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
+        const int64_t gi = bx + it * (int64_t)p.cps;
         if (gi >= p.ngroups) break;
         if (!mbar_wait(smem_u32(&full[st]), parity)) {
             atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
@@ -374,7 +384,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                 }
                 if (live) {
 #pragma unroll
-                    for (int r = 0; r < G; ++r) p.lp_out[(t0 + r) * L8 + g] = word[r];
+                    for (int r = 0; r < G; ++r) lp_out[(t0 + r) * L8 + g] = word[r];
                 }
             } else if (live) {
                 // ragged last stage, or a warp on the serial path: every hole patched by its owner
@@ -386,17 +396,17 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                         m &= m - 1;
                         const int f = __ldg(p.filler + hb[a] + h);
                         const uint32_t x = *reinterpret_cast<const uint16_t *>(stage8 + (size_t)r * row_bytes + 2 * f);
-                        const uint32_t q = quant_bits(x, __ldg(p.inv_s + f)) & 0xFu;
+                        const uint32_t q = quant_bits(x, __ldg(inv_s + f)) & 0xFu;
                         word = (word & ~(0xFu << (4 * n))) | (q << (4 * n));
                     }
-                    p.lp_out[(t0 + r) * L8 + g] = word;
+                    lp_out[(t0 + r) * L8 + g] = word;
                 }
             }
             (void)nh;
         }
         for (int h = tid; h < k; h += NT) {
             const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
-            for (int r = 0; r < rows; ++r) p.hp_out[(t0 + r) * k + h] = stage16[r * E + j];
+            for (int r = 0; r < rows; ++r) hp_out[(t0 + r) * k + h] = stage16[r * E + j];
         }
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
@@ -407,9 +417,9 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         }
     }
     // zero padding of the code section (at most 3 words), by the block that owned the last rows
-    if ((p.ngroups - 1) % gridDim.x == blockIdx.x) {
+    if ((p.ngroups - 1) % p.cps == bx) {
         const int64_t valid = p.T * L8;
-        for (int64_t w = valid + tid; w < p.lp_words; w += NT) p.lp_out[w] = 0u;
+        for (int64_t w = valid + tid; w < p.lp_words; w += NT) lp_out[w] = 0u;
     }
 }
 
@@ -447,26 +457,50 @@ cudaError_t tpq_launch_quantize_generic(const tpq_ctx *c, int shard, const uint1
 cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
                                       uint8_t *payload, cudaStream_t st, int64_t *launches)
 {
+    const void *ys[1] = {y};
+    void *pls[1] = {payload};
+    return tpq_launch_quantize_tiled_batch(c, shard, 1, ys, T, stride, pls, st, launches);
+}
+
+cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
+                                            int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches)
+{
+    if (n > QP_MAX_BATCH) {  // more shards than one launch carries: several launches
+        for (int b = 0; b < n; b += QP_MAX_BATCH) {
+            const int nb = n - b < QP_MAX_BATCH ? n - b : QP_MAX_BATCH;
+            cudaError_t e = tpq_launch_quantize_tiled_batch(c, shard0 + b, nb, ys + b, T, stride, payloads + b, st, launches);
+            if (e != cudaSuccess) return e;
+        }
+        return cudaSuccess;
+    }
     const int E = c->E, k = c->k;
     const int E8 = E / 8;
     const int gpt = (E8 + QP_MAX_CONSUMERS - 1) / QP_MAX_CONSUMERS;
     const int nt = ((E8 + gpt - 1) / gpt + 31) / 32 * 32;
-    // rows per stage (= independent chains per thread): small enough that every SM gets work
+    // blocks per shard: the SMs are divided among the shards of the batch (one persistent block per SM)
+    int cps = c->sm_count / n;
+    if (cps < 1) cps = 1;
+    // rows per stage (= independent chains per thread): small enough that every block gets work
     int G = 4;
-    while (G > 1 && ((T + G - 1) / G < 2 * (int64_t)c->sm_count || qp_smem_bytes(E, G, 3) > (size_t)c->smem_optin)) G >>= 1;
+    while (G > 1 && ((T + G - 1) / G < 2 * (int64_t)cps || qp_smem_bytes(E, G, 3) > (size_t)c->smem_optin)) G >>= 1;
     const int64_t ngroups = (T + G - 1) / G;
-    const int64_t grid = ngroups < c->sm_count ? ngroups : c->sm_count;
-    const int64_t per_block = (ngroups + grid - 1) / grid;
+    if (ngroups < cps) cps = (int)ngroups;
+    const int64_t grid = (int64_t)cps * n;
+    const int64_t per_block = (ngroups + cps - 1) / cps;
     int nstage = (int)(per_block < 8 ? per_block : 8);
     if (nstage < 2) nstage = 2;
     while (nstage > 2 && qp_smem_bytes(E, G, nstage) > (size_t)c->smem_optin) --nstage;
 
     QPParams p;
     const int64_t lpb = tpq_lp_bytes_i(T, E, k);
-    p.y = y; p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
-    p.inv_s = c->t.inv_s + (size_t)shard * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
-    p.lp_out = reinterpret_cast<uint32_t *>(payload); p.lp_words = lpb / 4;
-    p.hp_out = reinterpret_cast<uint16_t *>(payload + lpb); p.status = c->t.status;
+    for (int b = 0; b < n; ++b) {
+        p.y[b] = static_cast<const uint16_t *>(ys[b]);
+        p.payload[b] = static_cast<uint8_t *>(payloads[b]);
+    }
+    p.cps = cps; p.lp_bytes = lpb;
+    p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
+    p.inv_s = c->t.inv_s + (size_t)shard0 * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
+    p.lp_words = lpb / 4; p.status = c->t.status;
 #ifdef TPQ_TRACE
     p.trace = g_trace;
 #endif

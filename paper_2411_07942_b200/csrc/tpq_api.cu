@@ -373,6 +373,41 @@ tpq_status tpq_quantize_pack(tpq_ctx *c, int shard, const void *y, int64_t T, in
     return TPQ_OK;
 }
 
+tpq_status tpq_quantize_pack_batch(tpq_ctx *c, int first_shard, int n, const void *const *ys, int64_t T,
+                                   int64_t stride, void *const *payloads, size_t cap, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set: call tpq_select_features or tpq_set_features");
+    if (n < 0 || first_shard < 0 || first_shard + n > c->N)
+        return fail(c, TPQ_ERR_INVALID_ARG, "shards [%d, %d) out of range [0, %d)", first_shard, first_shard + n, c->N);
+    if (T < 0) return fail(c, TPQ_ERR_INVALID_ARG, "T < 0");
+    if (T == 0 || n == 0) return TPQ_OK;
+    if (!ys || !payloads) return fail(c, TPQ_ERR_INVALID_ARG, "NULL pointer array");
+    if (stride < c->E) return fail(c, TPQ_ERR_INVALID_ARG, "row stride %lld < E", (long long)stride);
+    if (cap < tpq_payload_bytes(c, T))
+        return fail(c, TPQ_ERR_SIZE, "payload capacity %zu < %zu", cap, tpq_payload_bytes(c, T));
+    for (int b = 0; b < n; ++b) {
+        if (!ys[b] || !payloads[b]) return fail(c, TPQ_ERR_INVALID_ARG, "NULL buffer for shard %d", first_shard + b);
+        if (!aligned16(ys[b]) || !aligned16(payloads[b]))
+            return fail(c, TPQ_ERR_ALIGN, "y and payload of shard %d must be 16-byte aligned", first_shard + b);
+    }
+    const bool tiled_ok = tpq_quantize_tiled_ok(c, T, stride);
+    if (c->kernel_path == 2 && !tiled_ok) return fail(c, TPQ_ERR_INVALID_ARG, "shape does not admit the tiled kernel");
+    cudaError_t e = cudaSuccess;
+    if (tiled_ok && c->kernel_path != 1) {
+        e = tpq_launch_quantize_tiled_batch(c, first_shard, n, ys, T, stride, payloads, static_cast<cudaStream_t>(stream),
+                                            &c->launches);
+    } else {
+        for (int b = 0; b < n && e == cudaSuccess; ++b)
+            e = tpq_launch_quantize_generic(c, first_shard + b, static_cast<const uint16_t *>(ys[b]), T, stride,
+                                            static_cast<uint8_t *>(payloads[b]), static_cast<cudaStream_t>(stream),
+                                            &c->launches);
+    }
+    if (e != cudaSuccess) return cuda_fail(c, e, "quantize_pack kernel");
+    return TPQ_OK;
+}
+
 tpq_status tpq_dequant_reduce(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
                               tpq_out_dtype dt, int64_t out_stride, void *stream)
 {

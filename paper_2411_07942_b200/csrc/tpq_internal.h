@@ -81,6 +81,9 @@ cudaError_t tpq_launch_quantize_generic(const tpq_ctx *c, int shard, const uint1
 cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
                                       uint8_t *payload, cudaStream_t st, int64_t *launches);
 
+cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
+                                            int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches);
+
 // sum_i D^(i): dequantise + reduce.
 bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int fp32_out);
 cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,

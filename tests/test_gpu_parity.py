@@ -334,3 +334,38 @@ def test_large_config_sampled_rows():
         ok, _ = gu.check_bf16(ob, ref, abs_sum, N)
         assert ok, r
     t.close()
+
+
+@pytest.mark.parametrize("N,T,E,k,path", [(4, 301, 1024, 16, binding.PATH_TILED), (8, 64, 4608, 72, binding.PATH_TILED),
+                                          (3, 17, 130, 2, binding.PATH_AUTO), (16, 40, 512, 8, binding.PATH_TILED),
+                                          (20, 9, 256, 8, binding.PATH_TILED)])
+def test_batched_quantize_equals_per_shard_calls(N, T, E, k, path):
+    """tpq_quantize_pack_batch writes, for every shard, exactly the payload of tpq_quantize_pack (and of the oracle)."""
+    orc = oracle.c()
+    w = _workload(N, T, E, 900 + E + N)
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E)
+    gu.calibrate_both(t, [synth.calibration_np(w, i, scale=scale) for i in range(N)])
+    hp = t.select_features(k)
+    _, inv = t.get_scales()
+    t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+    dev = [gu.dev_bf16(y) for y in ys]
+    P = t.payload_bytes(T)
+    bufs = [gu.guarded(P) for _ in range(N)]
+    t.quantize_pack_batch(0, [d.data_ptr() for d in dev], T, [v.data_ptr() for _, v in bufs], P)
+    torch.cuda.synchronize()
+    assert t.device_status() == 0
+    for i in range(N):
+        whole, view = bufs[i]
+        assert gu.guards_intact(whole, P)
+        assert np.array_equal(view.cpu().numpy(), orc.quantize_pack(ys[i], hp, inv[i])), i
+    # a sub-range of shards
+    if N >= 3:
+        bufs2 = [gu.guarded(P) for _ in range(2)]
+        t.quantize_pack_batch(1, [dev[1].data_ptr(), dev[2].data_ptr()], T, [v.data_ptr() for _, v in bufs2], P)
+        torch.cuda.synchronize()
+        for j in range(2):
+            assert np.array_equal(bufs2[j][1].cpu().numpy(), bufs[1 + j][1].cpu().numpy())
+    assert t.raw("tpq_quantize_pack_batch", N - 1, 2, None, T, E, None, P, None) == binding.TPQ_ERR_INVALID_ARG
+    t.close()
