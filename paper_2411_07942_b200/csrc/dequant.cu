@@ -83,13 +83,20 @@ __constant__ float2 kDecodeBias[4] = {{-8388616.0f, -8388736.0f},      // 16^0, 
                                       {-8912896.0f, -8388616.0f},      // 16^4, 16^0 (codes 5..7 use raw >> 20)
                                       {-8388736.0f, -8390656.0f}};     // 16^1, 16^2
 
-// `magic` must hold 0x4B000000 in a REGISTER (see opaque_magic): with both the mask and the exponent as
-// immediates the (x & mask) | magic of every code would take two logic instructions instead of one.
+// Each code costs ONE logic instruction only if the mask and the exponent pattern are both register
+// operands of an explicit lop3 ((x & mask) | magic, truth table 0xEA): written in C with immediates the
+// compiler emits two.  `magic` holds 0x4B000000 (see opaque_magic).
 __device__ __forceinline__ uint32_t opaque_magic()
 {
     uint32_t m;
     asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(m));
     return m;
+}
+__device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t mask, uint32_t magic)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(x), "r"(mask), "r"(magic));
+    return d;
 }
 
 __device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], uint32_t magic)
@@ -100,8 +107,8 @@ __device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], flo
     for (int h = 0; h < 4; ++h) {
         const int n0 = 2 * h, n1 = 2 * h + 1;
         const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
-        const float f0 = __uint_as_float((x0 & (0xFu << (4 * dq_pos(n0)))) | magic);
-        const float f1 = __uint_as_float((x1 & (0xFu << (4 * dq_pos(n1)))) | magic);
+        const float f0 = __uint_as_float(and_or(x0, 0xFu << (4 * dq_pos(n0)), magic));
+        const float f1 = __uint_as_float(and_or(x1, 0xFu << (4 * dq_pos(n1)), magic));
         const float2 d = __fadd2_rn(make_float2(f0, f1), kDecodeBias[h]);
         acc[h] = __ffma2_rn(d, sc[h], acc[h]);
     }
@@ -482,6 +489,13 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
 
     // ---------------- main warps
     const uint32_t magic = opaque_magic();
+    // 32-bit word indices into shared memory and a per-thread output pointer keep the loop's address
+    // arithmetic short
+    const uint32_t *const smem32 = reinterpret_cast<const uint32_t *>(smem);
+    const int stage_w = (int)(lay.stage >> 2), lp_w = (int)(lay.lp_stage >> 2);
+    constexpr int ESIZE = FP32OUT ? 4 : 2;
+    uint8_t *const out_col = static_cast<uint8_t *>(p.out) + (size_t)8 * g_ld * ESIZE;
+    const int64_t out_row_bytes = p.out_stride * ESIZE;
     TPQ_DMARK(1);
     for (int it = 0;; ++it) {
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
@@ -493,10 +507,12 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
         TPQ_DMARK(2 + 2 * it);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-        const uint8_t *stage = smem + (size_t)st * lay.stage;
+        const uint32_t *const sw = smem32 + st * stage_w + g_ld;  // this thread's word of row 0, device 0
+        uint8_t *orow = out_col + t0 * out_row_bytes;
         for (int r0 = 0; r0 < rows; r0 += 2) {
             const bool two = r0 + 1 < rows;
-            const int r1 = two ? r0 + 1 : r0;  // a ragged last stage decodes its last row twice, stores it once
+            const int d1 = two ? L8 : 0;  // a ragged last stage decodes its last row twice, stores it once
+            const uint32_t *const w = sw + r0 * L8;
             float2 acc[2][4];
 #pragma unroll
             for (int r = 0; r < 2; ++r)
@@ -505,17 +521,17 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
 #pragma unroll
             for (int i = 0; i < NMAX; ++i) {
                 if (i < N) {  // uniform
-                    const uint32_t *lp = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage);
-                    const uint32_t w0 = lp[r0 * L8 + g_ld];
-                    const uint32_t w1 = lp[r1 * L8 + g_ld];
+                    const uint32_t w0 = w[i * lp_w];
+                    const uint32_t w1 = w[i * lp_w + d1];
                     decode8(w0, sc[i], acc[0], magic);
                     decode8(w1, sc[i], acc[1], magic);
                 }
             }
             if (live) {
-                store_group<FP32OUT>(p.out, (t0 + r0) * p.out_stride + 8 * (int64_t)g, acc[0], 0u);
-                if (two) store_group<FP32OUT>(p.out, (t0 + r1) * p.out_stride + 8 * (int64_t)g, acc[1], 0u);
+                store_group<FP32OUT>(orow, 0, acc[0], 0u);
+                if (two) store_group<FP32OUT>(orow + out_row_bytes, 0, acc[1], 0u);
             }
+            orow += 2 * out_row_bytes;
         }
         __syncwarp();
         if (lane == 0) {
@@ -595,7 +611,7 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     const int64_t ngroups = (T + G - 1) / G;
     const int grid = (int)(ngroups < c->sm_count ? ngroups : c->sm_count);
     const int64_t per_block = (ngroups + grid - 1) / grid;
-    int nstage = (int)(per_block < 8 ? per_block : 8);
+    int nstage = (int)(per_block < 4 ? per_block : 4);  // deeper rings measured no faster (often slower)
     if (nstage < 2) nstage = 2;
     while (nstage > 2 && dr_layout(N, E, k, G, nstage).total > (size_t)c->smem_optin) --nstage;
     *G_out = G; *nstage_out = nstage; *ngroups_out = ngroups; *grid_out = grid;
