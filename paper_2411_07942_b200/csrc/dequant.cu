@@ -606,12 +606,15 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
     else if (L8 % 2 == 0) g0 = 2;
-    const int G = g0 < 2 ? 2 : g0;  // 2 or 4 rows per stage, unrolled in the kernel
+    int G = g0 < 2 ? 2 : g0;  // 2 or 4 rows per stage (a multiple of g0), walked two rows at a time
+    // long inputs: 4-row stages amortise the per-stage work (measured faster from about 32 rows per block)
+    if (G == 2 && T >= 32LL * c->sm_count && dr_layout(N, E, k, 4, 3).total <= (size_t)c->smem_optin) G = 4;
     if (dr_layout(N, E, k, G, 2).total > (size_t)c->smem_optin) return false;
     const int64_t ngroups = (T + G - 1) / G;
     const int grid = (int)(ngroups < c->sm_count ? ngroups : c->sm_count);
     const int64_t per_block = (ngroups + grid - 1) / grid;
     int nstage = (int)(per_block < 4 ? per_block : 4);  // deeper rings measured no faster (often slower)
+    if (G == 4 && nstage > 3) nstage = 3;
     if (nstage < 2) nstage = 2;
     while (nstage > 2 && dr_layout(N, E, k, G, nstage).total > (size_t)c->smem_optin) --nstage;
     *G_out = G; *nstage_out = nstage; *ngroups_out = ngroups; *grid_out = grid;
