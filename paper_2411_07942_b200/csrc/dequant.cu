@@ -170,96 +170,157 @@ struct DXParams {           // extras shared by the tiled kernels
 };
 
 // ----------------------------------------------------------------------------------------------
-// Strip kernel (any N): thread <-> 8 adjacent output features, block <-> a strip of 8*blockDim.x
-// features; blocks walk row blocks of R rows with R*NC independent 32-bit loads in flight per thread
-// (a warp reads 128 contiguous bytes).  The steps of NC devices at a time live in registers.
-// Blocks with blockIdx.x == gridDim.x - 1 do the filler and selected features of their rows instead.
+// Panel kernel (any N, any row length).  A 1-D grid of two kinds of blocks:
+//   main blocks   own a panel of CG groups of 8 adjacent code slots and walk chunks of RS*R rows,
+//                 RS = blockDim.x / CG.  Thread <-> (group, R rows): R*4 independent 32-bit loads in flight
+//                 per thread (a warp reads 128 contiguous bytes per device and row).  The panel's steps of
+//                 all N devices IN SLOT ORDER, pre-divided for the in-place decode, live in shared memory
+//                 ([N][CG][8] floats), so the register cost does not grow with N.  A hole's slot carries
+//                 the filler feature's step, so its lane accumulates the filler feature's sum and is
+//                 stored to that feature's column; nothing is stored to a selected feature's column.
+//   HP blocks     (the last n_hp blocks) sum the devices' BF16 blocks: thread <-> 8 consecutive selected
+//                 features of a row, one 16-byte load per device, 8 scattered stores.
+// The two kinds write disjoint columns, so they need no ordering.
 // ----------------------------------------------------------------------------------------------
-template <int NC, int R, bool FP32OUT>
-__global__ void __launch_bounds__(128) dequant_strips(const DQParams p, const DXParams x)
-{
-    const int E8 = p.E >> 3, L8 = (p.E - p.k) >> 3;
-    const int64_t n_rb = (p.T + R - 1) / R;
+constexpr int DP_THREADS = 512;
 
-    if (blockIdx.x == gridDim.x - 1) {
-        // ---- extras: one (row, feature) pair per thread step
-        const int64_t L = p.E - p.k;
-        const int per_row = x.n_holes + p.k;
-        for (int64_t rb = blockIdx.y; rb < n_rb; rb += gridDim.y) {
-            const int64_t t0 = rb * R;
-            const int rows = (int)((p.T - t0 < R) ? p.T - t0 : R);
-            for (int a = threadIdx.x; a < rows * per_row; a += blockDim.x) {
-                const int r = a / per_row, e = a - r * per_row;
-                const int64_t t = t0 + r;
-                float acc = 0.0f;
-                int j;
-                if (e < x.n_holes) {
-                    j = __ldg(x.filler + e);
-                    const int slot = __ldg(x.hole + e);
-                    for (int i = 0; i < p.N; ++i) {
-                        const uint32_t w = reinterpret_cast<const uint32_t *>(p.pl[i])[t * (L >> 3) + (slot >> 3)];
-                        const int code = (int)(((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) - 8;
-                        acc = __fmaf_rn((float)code, __ldg(p.s_k + (size_t)i * p.E + j), acc);
+struct DPParams {
+    DQParams q;
+    const float *s_slot;    // [N][E] slot-order steps
+    const int32_t *lp_idx;  // [E-k] feature of each slot
+    const int32_t *hp_idx;  // [k]
+    int CG, panels, gy, n_hp;
+    int64_t n_chunks;
+};
+
+template <int R, bool FP32OUT>
+__global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
+{
+    extern __shared__ __align__(16) float4 dp_steps[];  // [N][CG][2]
+    const DQParams &p = pp.q;
+    const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
+    const int tid = threadIdx.x;
+    const int n_main = pp.panels * pp.gy;
+
+    if ((int)blockIdx.x >= n_main) {
+        // ---------------- HP blocks
+        const int k8 = k >> 3;
+        const int64_t items = p.T * k8;
+        const int64_t stride = (int64_t)pp.n_hp * DP_THREADS;
+        for (int64_t a = (int64_t)(blockIdx.x - n_main) * DP_THREADS + tid; a < items; a += stride) {
+            const int64_t t = a / k8;
+            const int h8 = (int)(a - t * k8);
+            const int64_t off = p.lp_bytes + (t * k + 8 * h8) * 2;
+            float2 acc[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
+            for (int i0 = 0; i0 < N; i0 += 8) {
+                uint4 v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i0 + i < N) v[i] = __ldcs(reinterpret_cast<const uint4 *>(p.pl[i0 + i] + off));
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (i0 + i < N) {
+                        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                        for (int h = 0; h < 4; ++h)
+                            acc[h] = __fadd2_rn(acc[h], make_float2(__uint_as_float(w[h] << 16),
+                                                                    __uint_as_float(w[h] & 0xFFFF0000u)));
                     }
-                } else {
-                    const int h = e - x.n_holes;
-                    j = __ldg(x.hp_idx + h);
-                    for (int i = 0; i < p.N; ++i) {
-                        const uint16_t v = reinterpret_cast<const uint16_t *>(p.pl[i] + p.lp_bytes)[t * p.k + h];
-                        acc = __fadd_rn(acc, __uint_as_float((uint32_t)v << 16));
-                    }
-                }
-                store_one<FP32OUT>(p.out, t * p.out_stride + j, acc);
             }
+            const int4 c0 = __ldg(reinterpret_cast<const int4 *>(pp.hp_idx + 8 * h8));
+            const int4 c1 = __ldg(reinterpret_cast<const int4 *>(pp.hp_idx + 8 * h8) + 1);
+            const int64_t orow = t * p.out_stride;
+            store_one<FP32OUT>(p.out, orow + c0.x, acc[0].x);
+            store_one<FP32OUT>(p.out, orow + c0.y, acc[0].y);
+            store_one<FP32OUT>(p.out, orow + c0.z, acc[1].x);
+            store_one<FP32OUT>(p.out, orow + c0.w, acc[1].y);
+            store_one<FP32OUT>(p.out, orow + c1.x, acc[2].x);
+            store_one<FP32OUT>(p.out, orow + c1.y, acc[2].y);
+            store_one<FP32OUT>(p.out, orow + c1.z, acc[3].x);
+            store_one<FP32OUT>(p.out, orow + c1.w, acc[3].y);
         }
         return;
     }
 
-    const int g = blockIdx.x * blockDim.x + threadIdx.x;
-    if (g >= L8) return;
-    const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
-    const bool single = p.N <= NC;
-    const uint32_t magic = opaque_magic();
-    float2 sc[NC][4];
-    if (single) {
+    // ---------------- main blocks
+    const int CG = pp.CG;
+    const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
+    const int cg = tid & (CG - 1), rs = tid / CG, RS = DP_THREADS / CG;
+    const int g = panel * CG + cg;
+    const bool live = g < L8;
+    const int g_ld = live ? g : L8 - 1;
+
+    for (int a = tid; a < N * CG; a += DP_THREADS) {
+        const int i = a / CG, gg = panel * CG + (a & (CG - 1));
+        float2 s4[4];
 #pragma unroll
-        for (int i = 0; i < NC; ++i) {
-#pragma unroll
-            for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
-            if (i < p.N) load_steps(p.s_k + (size_t)i * p.E, g, sc[i]);
-        }
+        for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
+        if (gg < L8) load_steps(pp.s_slot + (size_t)i * E, gg, s4);
+        dp_steps[2 * a] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
+        dp_steps[2 * a + 1] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
     }
-    for (int64_t rb = blockIdx.y; rb < n_rb; rb += gridDim.y) {
-        const int64_t t0 = rb * R;
+    const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
+    const uint32_t magic = opaque_magic();
+    __syncthreads();
+
+    const int rows_chunk = RS * R;
+    const float4 *const my_steps = dp_steps + 2 * cg;
+
+    for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
+        const int64_t t0 = ch * rows_chunk + rs * R;
+        int64_t off[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int64_t t = (t0 + r < p.T) ? t0 + r : p.T - 1;  // rows past the end are decoded again, not stored
+            off[r] = t * L8 + g_ld;
+        }
         float2 acc[R][4];
 #pragma unroll
         for (int r = 0; r < R; ++r)
 #pragma unroll
             for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-        for (int i0 = 0; i0 < p.N; i0 += NC) {
-            if (!single) {
+        for (int i0 = 0; i0 < N; i0 += 4) {
+            uint32_t w[4][R];
 #pragma unroll
-                for (int i = 0; i < NC; ++i)
-                    if (i0 + i < p.N) load_steps(p.s_k + (size_t)(i0 + i) * p.E, g, sc[i]);
-            }
-            uint32_t w[R][NC];
+            for (int i = 0; i < 4; ++i)
+                if (i0 + i < N) {
+                    const uint32_t *const base = reinterpret_cast<const uint32_t *>(p.pl[i0 + i]);
 #pragma unroll
-            for (int r = 0; r < R; ++r)
-#pragma unroll
-                for (int i = 0; i < NC; ++i) {
-                    w[r][i] = 0x88888888u;  // all codes zero... (unused when out of range)
-                    if (t0 + r < p.T && i0 + i < p.N)
-                        w[r][i] = __ldcs(reinterpret_cast<const uint32_t *>(p.pl[i0 + i]) + (t0 + r) * L8 + g);
+                    for (int r = 0; r < R; ++r) w[i][r] = __ldcs(base + off[r]);
                 }
 #pragma unroll
-            for (int r = 0; r < R; ++r)
+            for (int i = 0; i < 4; ++i)
+                if (i0 + i < N) {
+                    const float4 a = my_steps[(size_t)(i0 + i) * CG * 2], b = my_steps[(size_t)(i0 + i) * CG * 2 + 1];
+                    const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
+                                          make_float2(b.z, b.w)};
 #pragma unroll
-                for (int i = 0; i < NC; ++i)
-                    if (t0 + r < p.T && i0 + i < p.N) decode8(w[r][i], sc[i], acc[r], magic);
+                    for (int r = 0; r < R; ++r) decode8(w[i][r], sc, acc[r], magic);
+                }
         }
+        if (live) {
+            if (mask == 0) {
 #pragma unroll
-        for (int r = 0; r < R; ++r)
-            if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], mask);
+                for (int r = 0; r < R; ++r)
+                    if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
+            } else {
+                // lane n of a hole's slot holds the sum of the filler feature lp_idx[8g+n]
+                int col[8];
+#pragma unroll
+                for (int n = 0; n < 8; ++n) col[n] = (mask & (1u << n)) ? __ldg(pp.lp_idx + 8 * g + n) : 8 * g + n;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    if (t0 + r < p.T) {
+                        const int64_t orow = (t0 + r) * p.out_stride;
+                        const float a8[8] = {acc[r][0].x, acc[r][0].y, acc[r][1].x, acc[r][1].y,
+                                             acc[r][2].x, acc[r][2].y, acc[r][3].x, acc[r][3].y};
+#pragma unroll
+                        for (int n = 0; n < 8; ++n) store_one<FP32OUT>(p.out, orow + col[n], a8[n]);
+                    }
+            }
+        }
     }
 }
 
@@ -621,6 +682,61 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     return true;
 }
 
+// Panel kernel geometry: CG groups per panel so that the steps fit comfortably in shared memory; rows
+// per thread R = 4 unless the input is too short to give every SM a block that way; one full wave of
+// blocks, a few of them for the BF16 block (its share of the bytes, with some margin), the others
+// walking their share of the row chunks.
+template <int R, bool FP32OUT>
+cudaError_t launch_panels_r(const tpq_ctx *c, DPParams &pp, int64_t T, cudaStream_t st)
+{
+    const int CG = pp.CG, N = c->N, E = c->E, k = c->k;
+    const size_t smem = (size_t)N * CG * 32;
+    const int RS = DP_THREADS / CG;
+    cudaError_t e = cudaFuncSetAttribute(dequant_panels<R, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 1;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dequant_panels<R, FP32OUT>, DP_THREADS, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const int total = c->sm_count * per_sm;
+    pp.n_chunks = (T + RS * R - 1) / (RS * R);
+    int n_hp = 0;
+    if (k > 0) {
+        const double share = 1.5 * (2.0 * k * N) / (N * ((E - k) * 0.5 + 2.0 * k) + 2.0 * E);
+        n_hp = (int)(total * share + 0.5);
+        const int64_t need = (T * (k / 8) + DP_THREADS - 1) / DP_THREADS;
+        if (n_hp > need) n_hp = (int)need;
+        if (n_hp < 1) n_hp = 1;
+    }
+    int64_t gy = (total - n_hp) / pp.panels;
+    if (gy > pp.n_chunks) gy = pp.n_chunks;
+    if (gy < 1) gy = 1;
+    pp.gy = (int)gy;
+    pp.n_hp = n_hp;
+    dequant_panels<R, FP32OUT><<<(unsigned)(pp.panels * gy + n_hp), DP_THREADS, smem, st>>>(pp);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_panels(const tpq_ctx *c, const DQParams &p, int64_t T, int fp32_out, cudaStream_t st,
+                          int64_t *launches)
+{
+    const int L8 = (c->E - c->k) / 8;
+    DPParams pp;
+    pp.q = p;
+    pp.s_slot = c->t.s_slot; pp.lp_idx = c->t.lp_idx; pp.hp_idx = c->t.hp_idx;
+    int CG = 128;
+    while (CG > 32 && (size_t)c->N * CG * 32 > (size_t)96 * 1024) CG >>= 1;
+    pp.CG = CG;
+    pp.panels = (L8 + CG - 1) / CG;
+    const int RS = DP_THREADS / CG;
+    const bool r4 = (T + RS * 4 - 1) / (RS * 4) * pp.panels >= c->sm_count;
+    cudaError_t e;
+    if (r4) e = fp32_out ? launch_panels_r<4, true>(c, pp, T, st) : launch_panels_r<4, false>(c, pp, T, st);
+    else    e = fp32_out ? launch_panels_r<1, true>(c, pp, T, st) : launch_panels_r<1, false>(c, pp, T, st);
+    if (e == cudaSuccess) ++*launches;
+    return e;
+}
+
 }  // namespace
 
 cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out, int fp32_out,
@@ -655,22 +771,5 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             return cudaGetLastError();
         }
     }
-    const int L8 = (c->E - c->k) / 8;
-    const int strips = (L8 + 127) / 128;
-    constexpr int R = 4;
-    const int64_t n_rb = (T + R - 1) / R;
-    int64_t gy = ((int64_t)c->sm_count * 4 + strips - 1) / strips;
-    if (gy > n_rb) gy = n_rb;
-    if (gy > 65535) gy = 65535;
-    if (gy < 1) gy = 1;
-    dim3 grid(strips + 1, (unsigned)gy), block(128);   // the last x-block does the filler / selected features
-    if (c->N <= 4) {
-        if (fp32_out) dequant_strips<4, R, true><<<grid, block, 0, st>>>(p, x);
-        else          dequant_strips<4, R, false><<<grid, block, 0, st>>>(p, x);
-    } else {
-        if (fp32_out) dequant_strips<8, R, true><<<grid, block, 0, st>>>(p, x);
-        else          dequant_strips<8, R, false><<<grid, block, 0, st>>>(p, x);
-    }
-    ++*launches;
-    return cudaGetLastError();
+    return launch_panels(c, p, T, fp32_out, st, launches);
 }

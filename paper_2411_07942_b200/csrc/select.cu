@@ -51,7 +51,8 @@ __global__ void __launch_bounds__(256) topk_flags_kernel(const float *__restrict
 }
 
 // One block: exclusive scan of the flags -> selected list, hole / filler lists, slot order,
-// per-feature slots, the dequantiser's zeroed-step copy and the per-8-feature group descriptors.
+// per-feature slots, the dequantiser's zeroed-step and slot-order step copies and the per-8-feature
+// group descriptors.
 __global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E, int k)
 {
     __shared__ int warp_sums[32];
@@ -102,7 +103,9 @@ __global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E
     __syncthreads();
     for (int j = tid; j < E; j += 1024) {
         const int f = t.flag[j];
-        if (j < L) t.lp_idx[j] = f ? t.filler[t.hpre[j]] : j;
+        const int src = (j < L) ? (f ? t.filler[t.hpre[j]] : j) : -1;  // feature held by slot j
+        if (j < L) t.lp_idx[j] = src;
+        for (int i = 0; i < N; ++i) t.s_slot[(size_t)i * E + j] = (src >= 0) ? t.s[(size_t)i * E + src] : 0.0f;
         if (f)
             t.pos[j] = -(t.hpre[j] + 1);
         else

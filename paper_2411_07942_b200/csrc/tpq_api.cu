@@ -45,7 +45,7 @@ cudaError_t dalloc(T **p, size_t n)
 void free_tables(tpq_tables &t)
 {
     cudaFree(t.m); cudaFree(t.M); cudaFree(t.R); cudaFree(t.Rbar); cudaFree(t.s); cudaFree(t.inv_s);
-    cudaFree(t.s_k); cudaFree(t.flag); cudaFree(t.hpre); cudaFree(t.pos); cudaFree(t.hp_idx);
+    cudaFree(t.s_k); cudaFree(t.s_slot); cudaFree(t.flag); cudaFree(t.hpre); cudaFree(t.pos); cudaFree(t.hp_idx);
     cudaFree(t.lp_idx); cudaFree(t.hole); cudaFree(t.filler); cudaFree(t.grp); cudaFree(t.status);
     memset(&t, 0, sizeof t);
 }
@@ -129,6 +129,7 @@ tpq_status tpq_create(tpq_ctx **out, int n_shards, int n_features, int bits, flo
     if (e == cudaSuccess) e = dalloc(&t.s, NE);
     if (e == cudaSuccess) e = dalloc(&t.inv_s, NE);
     if (e == cudaSuccess) e = dalloc(&t.s_k, NE);
+    if (e == cudaSuccess) e = dalloc(&t.s_slot, NE);
     if (e == cudaSuccess) e = dalloc(&t.flag, E);
     if (e == cudaSuccess) e = dalloc(&t.hpre, E);
     if (e == cudaSuccess) e = dalloc(&t.pos, E);

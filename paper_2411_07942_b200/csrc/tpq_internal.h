@@ -15,6 +15,7 @@ struct tpq_tables {
     float *Rbar;         // [E]    aggregated range
     float *s, *inv_s;    // [N][E] Int4 step and its reciprocal
     float *s_k;          // [N][E] step with 0 at selected features (dequantiser's copy)
+    float *s_slot;       // [N][E] step of the feature held by code slot c (slot order; 0 for c >= E-k)
     uint8_t *flag;       // [E]    1 = selected (kept in BF16)
     int32_t *hpre;       // [E]    number of selected features before j
     int32_t *pos;        // [E]    >= 0: code slot of feature j; < 0: -(h+1), h = rank among selected
