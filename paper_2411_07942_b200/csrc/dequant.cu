@@ -169,20 +169,63 @@ struct DXParams {           // extras shared by the tiled kernels
     int *status;
 };
 
+// ---- mbarrier / bulk-copy primitives shared by the panel and row kernels
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (int i = 0; i < DR_WAIT_LIMIT; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 // ----------------------------------------------------------------------------------------------
 // Panel kernel (any N, any row length).  A 1-D grid of two kinds of blocks:
-//   main blocks   own a panel of CG groups of 8 adjacent code slots and walk chunks of RS*R rows,
-//                 RS = blockDim.x / CG.  Thread <-> (group, R rows): R*4 independent 32-bit loads in flight
-//                 per thread (a warp reads 128 contiguous bytes per device and row).  The panel's steps of
-//                 all N devices IN SLOT ORDER, pre-divided for the in-place decode, live in shared memory
-//                 ([N][CG][8] floats), so the register cost does not grow with N.  A hole's slot carries
-//                 the filler feature's step, so its lane accumulates the filler feature's sum and is
-//                 stored to that feature's column; nothing is stored to a selected feature's column.
+//   main blocks   own a panel of CG groups of 8 adjacent code slots and walk chunks of RC = RS*DP_R rows,
+//                 RS = DP_THREADS / CG.  Thread <-> (group, DP_R rows).  A chunk is taken DP_NB devices at a
+//                 time ("step"); the DP_NB*DP_R code words a thread needs for a step are fetched by the
+//                 thread itself with 4-byte asynchronous copies into its own column of a shared-memory ring,
+//                 DP_STAGES-1 steps ahead of their use, so no thread waits on another and no register is
+//                 held by a load in flight (works for any row pitch: only 4-byte alignment is needed).
+//                 The panel's steps of all N devices IN SLOT ORDER, pre-divided for the in-place decode,
+//                 live in shared memory ([N][CG][8] floats), so the register cost does not grow with N.  A
+//                 hole's slot carries the filler feature's step, so its lane accumulates the filler
+//                 feature's sum and is stored to that feature's column; nothing is stored to a selected
+//                 feature's column.
 //   HP blocks     (the last n_hp blocks) sum the devices' BF16 blocks: thread <-> 8 consecutive selected
 //                 features of a row, one 16-byte load per device, 8 scattered stores.
 // The two kinds write disjoint columns, so they need no ordering.
 // ----------------------------------------------------------------------------------------------
 constexpr int DP_THREADS = 512;
+constexpr int DP_R = 4;       // rows per thread
+constexpr int DP_NB = 4;      // devices per step
+constexpr int DP_STAGES = 4;  // ring depth (steps)
 
 struct DPParams {
     DQParams q;
@@ -193,10 +236,27 @@ struct DPParams {
     int64_t n_chunks;
 };
 
-template <int R, bool FP32OUT>
-__global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
+__host__ __device__ inline size_t dp_steps_bytes(int N, int CG) { return (size_t)N * CG * 32; }
+__host__ __device__ inline size_t dp_smem_bytes(int N, int CG)
 {
-    extern __shared__ __align__(16) float4 dp_steps[];  // [N][CG][2]
+    return dp_steps_bytes(N, CG) + (size_t)DP_STAGES * DP_NB * DP_R * DP_THREADS * 4;
+}
+
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
+}
+
+template <bool FP32OUT>
+__global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams pp)
+{
+    extern __shared__ __align__(128) uint8_t dp_smem[];
     const DQParams &p = pp.q;
     const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
     const int tid = threadIdx.x;
@@ -246,11 +306,46 @@ __global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
 
     // ---------------- main blocks
     const int CG = pp.CG;
+    const int RS = DP_THREADS / CG, RC = RS * DP_R;
+    float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][CG][2]
     const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
-    const int cg = tid & (CG - 1), rs = tid / CG, RS = DP_THREADS / CG;
+    const int cg = tid & (CG - 1), rs = tid / CG;
     const int g = panel * CG + cg;
     const bool live = g < L8;
     const int g_ld = live ? g : L8 - 1;
+
+    // ring: word (stage, slot, thread), slot = device-in-step * DP_R + row; a thread only touches its own column
+    uint32_t *const ring = reinterpret_cast<uint32_t *>(dp_smem + dp_steps_bytes(N, CG)) + tid;
+    const uint32_t ring_s = smem_u32(ring);
+    constexpr int SLOTS = DP_NB * DP_R;
+    const int nbatch = (N + DP_NB - 1) / DP_NB;
+
+    // issue side of the pipeline: step (chunk ich, device batch ib) into stage ist
+    int64_t ich = by;
+    int ib = 0, ist = 0;
+    auto issue = [&]() {
+        if (ich < pp.n_chunks) {
+            const int64_t t0 = ich * RC + rs * DP_R;
+            const int i0 = ib * DP_NB;
+#pragma unroll
+            for (int r = 0; r < DP_R; ++r) {
+                const int64_t t = (t0 + r < p.T) ? t0 + r : p.T - 1;  // rows past the end are decoded again, not stored
+                const int64_t off = (t * L8 + g_ld) * 4;
+#pragma unroll
+                for (int i = 0; i < DP_NB; ++i)
+                    if (i0 + i < N)
+                        cp_async4(ring_s + (uint32_t)((ist * SLOTS + i * DP_R + r) * DP_THREADS * 4), p.pl[i0 + i] + off);
+            }
+            if (++ib == nbatch) {
+                ib = 0;
+                ich += pp.gy;
+            }
+            if (++ist == DP_STAGES) ist = 0;
+        }
+        cp_async_commit();  // (possibly empty: keeps the group count in step with the consumer)
+    };
+#pragma unroll
+    for (int s = 0; s < DP_STAGES - 1; ++s) issue();
 
     for (int a = tid; a < N * CG; a += DP_THREADS) {
         const int i = a / CG, gg = panel * CG + (a & (CG - 1));
@@ -265,45 +360,39 @@ __global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
     const uint32_t magic = opaque_magic();
     __syncthreads();
 
-    const int rows_chunk = RS * R;
     const float4 *const my_steps = dp_steps + 2 * cg;
-
+    int st = 0;
     for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
-        const int64_t t0 = ch * rows_chunk + rs * R;
-        int64_t off[R];
+        const int64_t t0 = ch * RC + rs * DP_R;
+        float2 acc[DP_R][4];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const int64_t t = (t0 + r < p.T) ? t0 + r : p.T - 1;  // rows past the end are decoded again, not stored
-            off[r] = t * L8 + g_ld;
-        }
-        float2 acc[R][4];
-#pragma unroll
-        for (int r = 0; r < R; ++r)
+        for (int r = 0; r < DP_R; ++r)
 #pragma unroll
             for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-        for (int i0 = 0; i0 < N; i0 += 4) {
-            uint32_t w[4][R];
+        for (int i0 = 0; i0 < N; i0 += DP_NB) {
+            issue();
+            cp_async_wait<DP_STAGES - 1>();  // this step's words have landed (the thread's own copies)
+            const uint32_t *const sw = ring + st * SLOTS * DP_THREADS;
+            uint32_t w[DP_NB][DP_R];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                if (i0 + i < N) {
-                    const uint32_t *const base = reinterpret_cast<const uint32_t *>(p.pl[i0 + i]);
+            for (int i = 0; i < DP_NB; ++i)
 #pragma unroll
-                    for (int r = 0; r < R; ++r) w[i][r] = __ldcs(base + off[r]);
-                }
+                for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * DP_R + r) * DP_THREADS];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < DP_NB; ++i)
                 if (i0 + i < N) {
                     const float4 a = my_steps[(size_t)(i0 + i) * CG * 2], b = my_steps[(size_t)(i0 + i) * CG * 2 + 1];
                     const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                           make_float2(b.z, b.w)};
 #pragma unroll
-                    for (int r = 0; r < R; ++r) decode8(w[i][r], sc, acc[r], magic);
+                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic);
                 }
+            if (++st == DP_STAGES) st = 0;
         }
         if (live) {
             if (mask == 0) {
 #pragma unroll
-                for (int r = 0; r < R; ++r)
+                for (int r = 0; r < DP_R; ++r)
                     if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
             } else {
                 // lane n of a hole's slot holds the sum of the filler feature lp_idx[8g+n]
@@ -311,7 +400,7 @@ __global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
 #pragma unroll
                 for (int n = 0; n < 8; ++n) col[n] = (mask & (1u << n)) ? __ldg(pp.lp_idx + 8 * g + n) : 8 * g + n;
 #pragma unroll
-                for (int r = 0; r < R; ++r)
+                for (int r = 0; r < DP_R; ++r)
                     if (t0 + r < p.T) {
                         const int64_t orow = (t0 + r) * p.out_stride;
                         const float a8[8] = {acc[r][0].x, acc[r][0].y, acc[r][1].x, acc[r][1].y,
@@ -322,6 +411,7 @@ __global__ void __launch_bounds__(DP_THREADS) dequant_panels(const DPParams pp)
             }
         }
     }
+    cp_async_wait<0>();
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -356,41 +446,6 @@ __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int ns
     l.bars = (size_t)nstage * l.stage;
     l.total = l.bars + (size_t)nstage * 24;
     return l;
-}
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (int i = 0; i < DR_WAIT_LIMIT; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
 }
 
 struct DRParams {
@@ -682,59 +737,43 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     return true;
 }
 
-// Panel kernel geometry: CG groups per panel so that the steps fit comfortably in shared memory; rows
-// per thread R = 4 unless the input is too short to give every SM a block that way; one full wave of
-// blocks, a few of them for the BF16 block (its share of the bytes, with some margin), the others
-// walking their share of the row chunks.
-template <int R, bool FP32OUT>
-cudaError_t launch_panels_r(const tpq_ctx *c, DPParams &pp, int64_t T, cudaStream_t st)
+// Panel kernel geometry: the widest panel (CG groups) whose steps fit in shared memory beside the ring;
+// one block per SM, a few of them for the BF16 block (its share of the bytes, with some margin), the
+// others walking their share of the row chunks.  Returns false if the shape does not admit it.
+bool panels_plan(const tpq_ctx *c, int64_t T, DPParams &pp)
 {
-    const int CG = pp.CG, N = c->N, E = c->E, k = c->k;
-    const size_t smem = (size_t)N * CG * 32;
-    const int RS = DP_THREADS / CG;
-    cudaError_t e = cudaFuncSetAttribute(dequant_panels<R, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    int per_sm = 1;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, dequant_panels<R, FP32OUT>, DP_THREADS, smem);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    const int total = c->sm_count * per_sm;
-    pp.n_chunks = (T + RS * R - 1) / (RS * R);
+    const int N = c->N, E = c->E, k = c->k, L8 = (E - k) / 8;
+    int CG = 128;
+    while (CG >= 32 && dp_smem_bytes(N, CG) > (size_t)c->smem_optin) CG >>= 1;
+    if (CG < 32) return false;
+    pp.CG = CG;
+    pp.panels = (L8 + CG - 1) / CG;
+    const int RC = DP_THREADS / CG * DP_R;
+    pp.n_chunks = (T + RC - 1) / RC;
     int n_hp = 0;
     if (k > 0) {
         const double share = 1.5 * (2.0 * k * N) / (N * ((E - k) * 0.5 + 2.0 * k) + 2.0 * E);
-        n_hp = (int)(total * share + 0.5);
+        n_hp = (int)(c->sm_count * share + 0.5);
         const int64_t need = (T * (k / 8) + DP_THREADS - 1) / DP_THREADS;
         if (n_hp > need) n_hp = (int)need;
         if (n_hp < 1) n_hp = 1;
     }
-    int64_t gy = (total - n_hp) / pp.panels;
+    int64_t gy = (c->sm_count - n_hp) / pp.panels;
     if (gy > pp.n_chunks) gy = pp.n_chunks;
     if (gy < 1) gy = 1;
     pp.gy = (int)gy;
     pp.n_hp = n_hp;
-    dequant_panels<R, FP32OUT><<<(unsigned)(pp.panels * gy + n_hp), DP_THREADS, smem, st>>>(pp);
-    return cudaGetLastError();
+    return true;
 }
 
-cudaError_t launch_panels(const tpq_ctx *c, const DQParams &p, int64_t T, int fp32_out, cudaStream_t st,
-                          int64_t *launches)
+template <bool FP32OUT>
+cudaError_t launch_panels(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
 {
-    const int L8 = (c->E - c->k) / 8;
-    DPParams pp;
-    pp.q = p;
-    pp.s_slot = c->t.s_slot; pp.lp_idx = c->t.lp_idx; pp.hp_idx = c->t.hp_idx;
-    int CG = 128;
-    while (CG > 32 && (size_t)c->N * CG * 32 > (size_t)96 * 1024) CG >>= 1;
-    pp.CG = CG;
-    pp.panels = (L8 + CG - 1) / CG;
-    const int RS = DP_THREADS / CG;
-    const bool r4 = (T + RS * 4 - 1) / (RS * 4) * pp.panels >= c->sm_count;
-    cudaError_t e;
-    if (r4) e = fp32_out ? launch_panels_r<4, true>(c, pp, T, st) : launch_panels_r<4, false>(c, pp, T, st);
-    else    e = fp32_out ? launch_panels_r<1, true>(c, pp, T, st) : launch_panels_r<1, false>(c, pp, T, st);
-    if (e == cudaSuccess) ++*launches;
-    return e;
+    const size_t smem = dp_smem_bytes(c->N, pp.CG);
+    cudaError_t e = cudaFuncSetAttribute(dequant_panels<FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dequant_panels<FP32OUT><<<(unsigned)(pp.panels * pp.gy + pp.n_hp), DP_THREADS, smem, st>>>(pp);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -771,5 +810,11 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             return cudaGetLastError();
         }
     }
-    return launch_panels(c, p, T, fp32_out, st, launches);
+    DPParams dp;
+    if (!panels_plan(c, T, dp)) return tpq_launch_dequant_generic(c, payloads, T, out, fp32_out, out_stride, st, launches);
+    dp.q = p;
+    dp.s_slot = c->t.s_slot; dp.lp_idx = c->t.lp_idx; dp.hp_idx = c->t.hp_idx;
+    const cudaError_t e = fp32_out ? launch_panels<true>(c, dp, st) : launch_panels<false>(c, dp, st);
+    if (e == cudaSuccess) ++*launches;
+    return e;
 }
