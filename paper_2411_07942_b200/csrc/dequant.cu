@@ -99,7 +99,8 @@ __device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t mask, uint32_t m
     return d;
 }
 
-__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], uint32_t magic)
+__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], uint32_t magic,
+                                        const float2 (&bias)[4] = kDecodeBias)
 {
     const uint32_t xa = raw ^ 0x88888888u;
     const uint32_t xb = xa >> 20;
@@ -109,7 +110,7 @@ __device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], flo
         const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
         const float f0 = __uint_as_float(and_or(x0, 0xFu << (4 * dq_pos(n0)), magic));
         const float f1 = __uint_as_float(and_or(x1, 0xFu << (4 * dq_pos(n1)), magic));
-        const float2 d = __fadd2_rn(make_float2(f0, f1), kDecodeBias[h]);
+        const float2 d = __fadd2_rn(make_float2(f0, f1), bias[h]);
         acc[h] = __ffma2_rn(d, sc[h], acc[h]);
     }
 }
@@ -206,45 +207,53 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
 }
 
 // ----------------------------------------------------------------------------------------------
-// Panel kernel (any N, any row length).  A 1-D grid of two kinds of blocks:
-//   main blocks   own a panel of CG groups of 8 adjacent code slots and walk chunks of RC = RS*DP_R rows,
-//                 RS = DP_THREADS / CG.  Thread <-> (group, DP_R rows).  A chunk is taken DP_NB devices at a
-//                 time ("step"); the DP_NB*DP_R code words a thread needs for a step are fetched by the
-//                 thread itself with 4-byte asynchronous copies into its own column of a shared-memory ring,
-//                 DP_STAGES-1 steps ahead of their use, so no thread waits on another and no register is
-//                 held by a load in flight (works for any row pitch: only 4-byte alignment is needed).
-//                 The panel's steps of all N devices IN SLOT ORDER, pre-divided for the in-place decode,
-//                 live in shared memory ([N][CG][8] floats), so the register cost does not grow with N.  A
-//                 hole's slot carries the filler feature's step, so its lane accumulates the filler
-//                 feature's sum and is stored to that feature's column; nothing is stored to a selected
-//                 feature's column.
-//   HP blocks     (the last n_hp blocks) sum the devices' BF16 blocks: thread <-> 8 consecutive selected
-//                 features of a row, one 16-byte load per device, 8 scattered stores.
-// The two kinds write disjoint columns, so they need no ordering.
+// Panel kernel (any N, any row length).  A block owns a panel of CG groups of 8 adjacent code slots and
+// walks chunks of RC = RS*DP_R rows, RS = DP_THREADS / CG; thread <-> (group, DP_R rows).  A chunk is taken
+// DP_NB devices at a time ("step").  The code words of a step -- one segment of CG words per (device, row),
+// widened to a 16-byte aligned start -- are fetched by all threads together with 16-byte asynchronous
+// copies into a ring of shared-memory stages, DP_STAGES-1 steps ahead of their use; one block barrier per
+// step makes a landed stage visible and frees the stage consumed before it.  (A chunk starts on a 16-byte
+// boundary of the code stream because RC is a multiple of 4, so the shift of a row inside its segment
+// depends only on the row's place in the chunk.)  The panel's steps of all N devices IN SLOT ORDER,
+// pre-divided for the in-place decode, live in shared memory ([N][2][CG] float4), so the register cost does
+// not grow with N.  A hole's slot carries the filler feature's step, so its lane accumulates the filler
+// feature's sum and is stored to that feature's column; nothing is stored to a selected feature's column.
+// After its chunks every block sums its share of the devices' BF16 blocks: thread <-> 8 consecutive
+// selected features of a row, one 16-byte load per device, 8 scattered stores.  Code lanes and BF16 sums
+// write disjoint columns, so they need no ordering.
 // ----------------------------------------------------------------------------------------------
-constexpr int DP_THREADS = 512;
-constexpr int DP_R = 4;       // rows per thread
-constexpr int DP_NB = 4;      // devices per step
-constexpr int DP_STAGES = 4;  // ring depth (steps)
+#ifndef TPQ_DP_THREADS
+#define TPQ_DP_THREADS 512
+#define TPQ_DP_NB 4
+#define TPQ_DP_STAGES 4
+#endif
+constexpr int DP_THREADS = TPQ_DP_THREADS;
+constexpr int DP_R = 4;                   // rows per thread (a multiple of 4: see above)
+constexpr int DP_NB = TPQ_DP_NB;          // devices per step
+constexpr int DP_STAGES = TPQ_DP_STAGES;  // ring depth (steps)
 
 struct DPParams {
     DQParams q;
     const float *s_slot;    // [N][E] slot-order steps
     const int32_t *lp_idx;  // [E-k] feature of each slot
     const int32_t *hp_idx;  // [k]
-    int CG, panels, gy, n_hp;
+    int CG, panels, gy;
     int64_t n_chunks;
 };
 
 __host__ __device__ inline size_t dp_steps_bytes(int N, int CG) { return (size_t)N * CG * 32; }
+__host__ __device__ inline size_t dp_stage_bytes(int CG)
+{
+    return (size_t)DP_NB * (DP_THREADS / CG * DP_R) * (CG / 4 + 1) * 16;
+}
 __host__ __device__ inline size_t dp_smem_bytes(int N, int CG)
 {
-    return dp_steps_bytes(N, CG) + (size_t)DP_STAGES * DP_NB * DP_R * DP_THREADS * 4;
+    return dp_steps_bytes(N, CG) + (size_t)DP_STAGES * dp_stage_bytes(CG);
 }
 
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src)
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src)
 {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
@@ -253,94 +262,108 @@ __device__ __forceinline__ void cp_async_wait()
     asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
 }
 
+// the BF16 block: thread <-> 8 consecutive selected features of a row; items first, first + stride, ...
 template <bool FP32OUT>
+__device__ __forceinline__ void dp_sum_bf16_block(const DQParams &p, const int32_t *hp_idx, int64_t first, int64_t stride)
+{
+    const int N = p.N, k = p.k;
+    const int k8 = k >> 3;
+    const int64_t items = p.T * k8;
+    for (int64_t a = first; a < items; a += stride) {
+        const int64_t t = a / k8;
+        const int h8 = (int)(a - t * k8);
+        const int64_t off = p.lp_bytes + (t * k + 8 * h8) * 2;
+        float2 acc[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
+        for (int i0 = 0; i0 < N; i0 += 8) {
+            uint4 v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i0 + i < N) v[i] = __ldcs(reinterpret_cast<const uint4 *>(p.pl[i0 + i] + off));
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (i0 + i < N) {
+                    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                    for (int h = 0; h < 4; ++h)
+                        acc[h] = __fadd2_rn(acc[h], make_float2(__uint_as_float(w[h] << 16),
+                                                                __uint_as_float(w[h] & 0xFFFF0000u)));
+                }
+        }
+        const int4 c0 = __ldg(reinterpret_cast<const int4 *>(hp_idx + 8 * h8));
+        const int4 c1 = __ldg(reinterpret_cast<const int4 *>(hp_idx + 8 * h8) + 1);
+        const int64_t orow = t * p.out_stride;
+        store_one<FP32OUT>(p.out, orow + c0.x, acc[0].x);
+        store_one<FP32OUT>(p.out, orow + c0.y, acc[0].y);
+        store_one<FP32OUT>(p.out, orow + c0.z, acc[1].x);
+        store_one<FP32OUT>(p.out, orow + c0.w, acc[1].y);
+        store_one<FP32OUT>(p.out, orow + c1.x, acc[2].x);
+        store_one<FP32OUT>(p.out, orow + c1.y, acc[2].y);
+        store_one<FP32OUT>(p.out, orow + c1.z, acc[3].x);
+        store_one<FP32OUT>(p.out, orow + c1.w, acc[3].y);
+    }
+}
+
+template <int CG, bool FP32OUT>
 __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams pp)
 {
     extern __shared__ __align__(128) uint8_t dp_smem[];
+    constexpr int RS = DP_THREADS / CG, RC = RS * DP_R;
+    constexpr int SEGC = CG / 4 + 1;          // 16-byte pieces per segment
+    constexpr int SEGW = SEGC * 4;            // words per segment
+    constexpr int PIECES = DP_NB * RC * SEGC; // pieces per step
+    constexpr int NCP = (PIECES + DP_THREADS - 1) / DP_THREADS;
+    constexpr uint32_t STAGE_BYTES = PIECES * 16;
+    static_assert(RC % 4 == 0, "a chunk must start on a 16-byte boundary of the code stream");
+
     const DQParams &p = pp.q;
     const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
     const int tid = threadIdx.x;
-    const int n_main = pp.panels * pp.gy;
-
-    if ((int)blockIdx.x >= n_main) {
-        // ---------------- HP blocks
-        const int k8 = k >> 3;
-        const int64_t items = p.T * k8;
-        const int64_t stride = (int64_t)pp.n_hp * DP_THREADS;
-        for (int64_t a = (int64_t)(blockIdx.x - n_main) * DP_THREADS + tid; a < items; a += stride) {
-            const int64_t t = a / k8;
-            const int h8 = (int)(a - t * k8);
-            const int64_t off = p.lp_bytes + (t * k + 8 * h8) * 2;
-            float2 acc[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
-            for (int i0 = 0; i0 < N; i0 += 8) {
-                uint4 v[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i0 + i < N) v[i] = __ldcs(reinterpret_cast<const uint4 *>(p.pl[i0 + i] + off));
-#pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (i0 + i < N) {
-                        const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-#pragma unroll
-                        for (int h = 0; h < 4; ++h)
-                            acc[h] = __fadd2_rn(acc[h], make_float2(__uint_as_float(w[h] << 16),
-                                                                    __uint_as_float(w[h] & 0xFFFF0000u)));
-                    }
-            }
-            const int4 c0 = __ldg(reinterpret_cast<const int4 *>(pp.hp_idx + 8 * h8));
-            const int4 c1 = __ldg(reinterpret_cast<const int4 *>(pp.hp_idx + 8 * h8) + 1);
-            const int64_t orow = t * p.out_stride;
-            store_one<FP32OUT>(p.out, orow + c0.x, acc[0].x);
-            store_one<FP32OUT>(p.out, orow + c0.y, acc[0].y);
-            store_one<FP32OUT>(p.out, orow + c0.z, acc[1].x);
-            store_one<FP32OUT>(p.out, orow + c0.w, acc[1].y);
-            store_one<FP32OUT>(p.out, orow + c1.x, acc[2].x);
-            store_one<FP32OUT>(p.out, orow + c1.y, acc[2].y);
-            store_one<FP32OUT>(p.out, orow + c1.z, acc[3].x);
-            store_one<FP32OUT>(p.out, orow + c1.w, acc[3].y);
-        }
-        return;
-    }
-
-    // ---------------- main blocks
-    const int CG = pp.CG;
-    const int RS = DP_THREADS / CG, RC = RS * DP_R;
-    float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][CG][2]
+    float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][2][CG]
     const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
     const int cg = tid & (CG - 1), rs = tid / CG;
     const int g = panel * CG + cg;
     const bool live = g < L8;
-    const int g_ld = live ? g : L8 - 1;
-
-    // ring: word (stage, slot, thread), slot = device-in-step * DP_R + row; a thread only touches its own column
-    uint32_t *const ring = reinterpret_cast<uint32_t *>(dp_smem + dp_steps_bytes(N, CG)) + tid;
-    const uint32_t ring_s = smem_u32(ring);
-    constexpr int SLOTS = DP_NB * DP_R;
     const int nbatch = (N + DP_NB - 1) / DP_NB;
+    const int64_t chunk_bytes = (int64_t)RC * L8 * 4;  // code bytes of one device in a chunk of rows
+    uint8_t *const ring = dp_smem + dp_steps_bytes(N, CG);
+    const uint32_t ring_s = smem_u32(ring);
 
-    // issue side of the pipeline: step (chunk ich, device batch ib) into stage ist
+    // copy side: piece c = tid + j * DP_THREADS of a step is piece `within` of segment (device i, row) and
+    // lands at byte 16 c of the stage; its source offset inside the chunk does not depend on the chunk
+    uint32_t cp_goff[NCP];  // source byte offset inside the device's chunk
+    int cp_dev[NCP];        // device within the step; -1: no such piece
+#pragma unroll
+    for (int j = 0; j < NCP; ++j) {
+        const int c = tid + j * DP_THREADS;
+        const int seg = c / SEGC, within = c - seg * SEGC;
+        const int i = seg / RC, row = seg - i * RC;
+        cp_dev[j] = (c < PIECES) ? i : -1;
+        cp_goff[j] = (((uint32_t)row * (uint32_t)L8 + (uint32_t)panel * CG) * 4u & ~15u) + (uint32_t)within * 16u;
+    }
     int64_t ich = by;
-    int ib = 0, ist = 0;
+    int ib = 0;
+    uint32_t idst = ring_s + (uint32_t)tid * 16u;
     auto issue = [&]() {
         if (ich < pp.n_chunks) {
-            const int64_t t0 = ich * RC + rs * DP_R;
+            const int64_t cbase = ich * chunk_bytes;
+            const int64_t left = p.lp_bytes - cbase;  // bytes of the code section from the chunk's start on
+            const uint32_t lim = (uint32_t)(left < (int64_t)0x7FFFFFF0 ? left : (int64_t)0x7FFFFFF0);
             const int i0 = ib * DP_NB;
 #pragma unroll
-            for (int r = 0; r < DP_R; ++r) {
-                const int64_t t = (t0 + r < p.T) ? t0 + r : p.T - 1;  // rows past the end are decoded again, not stored
-                const int64_t off = (t * L8 + g_ld) * 4;
-#pragma unroll
-                for (int i = 0; i < DP_NB; ++i)
-                    if (i0 + i < N)
-                        cp_async4(ring_s + (uint32_t)((ist * SLOTS + i * DP_R + r) * DP_THREADS * 4), p.pl[i0 + i] + off);
+            for (int j = 0; j < NCP; ++j) {
+                // pieces past the end of the code section (rows past the end, the last panel's overhang) and
+                // devices past N are skipped; what they would have filled is never stored
+                if (cp_dev[j] >= 0 && i0 + cp_dev[j] < N && cp_goff[j] + 16u <= lim)
+                    cp_async16(idst + (uint32_t)(j * DP_THREADS * 16), p.pl[i0 + cp_dev[j]] + cbase + cp_goff[j]);
             }
             if (++ib == nbatch) {
                 ib = 0;
                 ich += pp.gy;
             }
-            if (++ist == DP_STAGES) ist = 0;
+            idst += STAGE_BYTES;
+            if (idst == ring_s + (uint32_t)tid * 16u + DP_STAGES * STAGE_BYTES) idst = ring_s + (uint32_t)tid * 16u;
         }
         cp_async_commit();  // (possibly empty: keeps the group count in step with the consumer)
     };
@@ -348,20 +371,33 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
     for (int s = 0; s < DP_STAGES - 1; ++s) issue();
 
     for (int a = tid; a < N * CG; a += DP_THREADS) {
-        const int i = a / CG, gg = panel * CG + (a & (CG - 1));
+        const int i = a / CG, c = a & (CG - 1), gg = panel * CG + c;
         float2 s4[4];
 #pragma unroll
         for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
         if (gg < L8) load_steps(pp.s_slot + (size_t)i * E, gg, s4);
-        dp_steps[2 * a] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
-        dp_steps[2 * a + 1] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
+        dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
+        dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
     }
     const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
     const uint32_t magic = opaque_magic();
-    __syncthreads();
+    float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        bias[h] = kDecodeBias[h];
+        asm volatile("" : "+f"(bias[h].x), "+f"(bias[h].y));
+    }
 
-    const float4 *const my_steps = dp_steps + 2 * cg;
-    int st = 0;
+    // consume side: word of (device i of the step, this thread's row r) inside a stage
+    int wofs[DP_R];
+#pragma unroll
+    for (int r = 0; r < DP_R; ++r) {
+        const int rowc = rs * DP_R + r;
+        wofs[r] = rowc * SEGW + (int)(((uint32_t)rowc * (uint32_t)L8 + (uint32_t)panel * CG) & 3u) + (live ? cg : 0);
+    }
+    const float4 *const my_steps = dp_steps + cg;
+    const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring);
+    const uint32_t *sw = ring_w;
     for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
         const int64_t t0 = ch * RC + rs * DP_R;
         float2 acc[DP_R][4];
@@ -369,25 +405,38 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
         for (int r = 0; r < DP_R; ++r)
 #pragma unroll
             for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-        for (int i0 = 0; i0 < N; i0 += DP_NB) {
+        const float4 *st4 = my_steps;
+        for (int i0 = 0; i0 < N; i0 += DP_NB, st4 += DP_NB * 2 * CG) {
+            cp_async_wait<DP_STAGES - 2>();  // this thread's pieces of the step have landed ...
+            __syncthreads();                 // ... and everybody's; the stage consumed last is free
             issue();
-            cp_async_wait<DP_STAGES - 1>();  // this step's words have landed (the thread's own copies)
-            const uint32_t *const sw = ring + st * SLOTS * DP_THREADS;
             uint32_t w[DP_NB][DP_R];
 #pragma unroll
             for (int i = 0; i < DP_NB; ++i)
 #pragma unroll
-                for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * DP_R + r) * DP_THREADS];
+                for (int r = 0; r < DP_R; ++r) w[i][r] = sw[i * RC * SEGW + wofs[r]];
+            sw += STAGE_BYTES / 4;
+            if (sw == ring_w + DP_STAGES * (STAGE_BYTES / 4)) sw = ring_w;
+            if (i0 + DP_NB <= N) {
 #pragma unroll
-            for (int i = 0; i < DP_NB; ++i)
-                if (i0 + i < N) {
-                    const float4 a = my_steps[(size_t)(i0 + i) * CG * 2], b = my_steps[(size_t)(i0 + i) * CG * 2 + 1];
+                for (int i = 0; i < DP_NB; ++i) {
+                    const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
                     const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                           make_float2(b.z, b.w)};
 #pragma unroll
-                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic);
+                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
                 }
-            if (++st == DP_STAGES) st = 0;
+            } else {
+#pragma unroll
+                for (int i = 0; i < DP_NB; ++i)
+                    if (i0 + i < N) {
+                        const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
+                        const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
+                                              make_float2(b.z, b.w)};
+#pragma unroll
+                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                    }
+            }
         }
         if (live) {
             if (mask == 0) {
@@ -412,6 +461,9 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
         }
     }
     cp_async_wait<0>();
+
+    // every block's share of the BF16 block
+    dp_sum_bf16_block<FP32OUT>(p, pp.hp_idx, (int64_t)blockIdx.x * DP_THREADS + tid, (int64_t)gridDim.x * DP_THREADS);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -750,30 +802,31 @@ bool panels_plan(const tpq_ctx *c, int64_t T, DPParams &pp)
     pp.panels = (L8 + CG - 1) / CG;
     const int RC = DP_THREADS / CG * DP_R;
     pp.n_chunks = (T + RC - 1) / RC;
-    int n_hp = 0;
-    if (k > 0) {
-        const double share = 1.5 * (2.0 * k * N) / (N * ((E - k) * 0.5 + 2.0 * k) + 2.0 * E);
-        n_hp = (int)(c->sm_count * share + 0.5);
-        const int64_t need = (T * (k / 8) + DP_THREADS - 1) / DP_THREADS;
-        if (n_hp > need) n_hp = (int)need;
-        if (n_hp < 1) n_hp = 1;
-    }
-    int64_t gy = (c->sm_count - n_hp) / pp.panels;
+    int64_t gy = c->sm_count / pp.panels;
     if (gy > pp.n_chunks) gy = pp.n_chunks;
     if (gy < 1) gy = 1;
     pp.gy = (int)gy;
-    pp.n_hp = n_hp;
     return true;
+}
+
+template <int CG, bool FP32OUT>
+cudaError_t launch_panels_cg(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
+{
+    const size_t smem = dp_smem_bytes(c->N, CG);
+    cudaError_t e = cudaFuncSetAttribute(dequant_panels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dequant_panels<CG, FP32OUT><<<(unsigned)(pp.panels * pp.gy), DP_THREADS, smem, st>>>(pp);
+    return cudaGetLastError();
 }
 
 template <bool FP32OUT>
 cudaError_t launch_panels(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
 {
-    const size_t smem = dp_smem_bytes(c->N, pp.CG);
-    cudaError_t e = cudaFuncSetAttribute(dequant_panels<FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    dequant_panels<FP32OUT><<<(unsigned)(pp.panels * pp.gy + pp.n_hp), DP_THREADS, smem, st>>>(pp);
-    return cudaGetLastError();
+    switch (pp.CG) {
+    case 128: return launch_panels_cg<128, FP32OUT>(c, pp, st);
+    case 64: return launch_panels_cg<64, FP32OUT>(c, pp, st);
+    default: return launch_panels_cg<32, FP32OUT>(c, pp, st);
+    }
 }
 
 }  // namespace
