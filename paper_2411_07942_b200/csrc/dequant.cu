@@ -4,7 +4,10 @@
 //
 // Accumulation is binary32, devices in ascending order: acc = fma(code_i, s_i, acc) for a
 // low-precision feature, acc = fl(acc + y_i) for a selected one; one final rounding for BF16.
+#include <cuda.h>  // CUtensorMap and the encode function's type (reached through the runtime, no libcuda link)
 #include <cuda_bf16.h>
+
+#include <new>
 
 #include "tpq_internal.h"
 
@@ -305,6 +308,32 @@ __device__ __forceinline__ void dp_sum_bf16_block(const DQParams &p, const int32
     }
 }
 
+// a thread's DP_R rows of sums -> the output; lane n of a hole's slot holds the sum of the filler feature
+// lp_idx[8g+n] and goes to that feature's column
+template <bool FP32OUT>
+__device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *lp_idx, int64_t t0, int g, uint32_t mask,
+                                              const float2 (&acc)[DP_R][4])
+{
+    if (mask == 0) {
+#pragma unroll
+        for (int r = 0; r < DP_R; ++r)
+            if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
+    } else {
+        int col[8];
+#pragma unroll
+        for (int n = 0; n < 8; ++n) col[n] = (mask & (1u << n)) ? __ldg(lp_idx + 8 * g + n) : 8 * g + n;
+#pragma unroll
+        for (int r = 0; r < DP_R; ++r)
+            if (t0 + r < p.T) {
+                const int64_t orow = (t0 + r) * p.out_stride;
+                const float a8[8] = {acc[r][0].x, acc[r][0].y, acc[r][1].x, acc[r][1].y,
+                                     acc[r][2].x, acc[r][2].y, acc[r][3].x, acc[r][3].y};
+#pragma unroll
+                for (int n = 0; n < 8; ++n) store_one<FP32OUT>(p.out, orow + col[n], a8[n]);
+            }
+    }
+}
+
 template <int CG, bool FP32OUT>
 __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams pp)
 {
@@ -438,32 +467,188 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                     }
             }
         }
-        if (live) {
-            if (mask == 0) {
-#pragma unroll
-                for (int r = 0; r < DP_R; ++r)
-                    if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
-            } else {
-                // lane n of a hole's slot holds the sum of the filler feature lp_idx[8g+n]
-                int col[8];
-#pragma unroll
-                for (int n = 0; n < 8; ++n) col[n] = (mask & (1u << n)) ? __ldg(pp.lp_idx + 8 * g + n) : 8 * g + n;
-#pragma unroll
-                for (int r = 0; r < DP_R; ++r)
-                    if (t0 + r < p.T) {
-                        const int64_t orow = (t0 + r) * p.out_stride;
-                        const float a8[8] = {acc[r][0].x, acc[r][0].y, acc[r][1].x, acc[r][1].y,
-                                             acc[r][2].x, acc[r][2].y, acc[r][3].x, acc[r][3].y};
-#pragma unroll
-                        for (int n = 0; n < 8; ++n) store_one<FP32OUT>(p.out, orow + col[n], a8[n]);
-                    }
-            }
-        }
+        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, mask, acc);
     }
     cp_async_wait<0>();
 
     // every block's share of the BF16 block
     dp_sum_bf16_block<FP32OUT>(p, pp.hp_idx, (int64_t)blockIdx.x * DP_THREADS + tid, (int64_t)gridDim.x * DP_THREADS);
+}
+
+// ----------------------------------------------------------------------------------------------
+// Tensor-map panel kernel (N <= DT_MAX_DEV devices, row pitch a multiple of 16 bytes).
+//
+// Same division of work as the panel kernel above, but the code words arrive through the tensor copy
+// engine: each device's code section is a 2-D tensor of 32-bit words ((E-k)/8 words x T rows), and one
+// tiled copy per device and step brings a box of CG words x RC rows into a shared-memory stage, signalling
+// a "full" mbarrier.  A producer warp (one elected lane) issues the copies; main warps free a stage through
+// the "empty" mbarrier as soon as its words are in registers.  Rows past T and words past the row end are
+// zero-filled by the copy engine (their sums are never stored).  Every wait is bounded: on expiry the
+// kernel sets the status word and returns.
+// ----------------------------------------------------------------------------------------------
+constexpr int DT_MAX_DEV = 16;
+constexpr int DT_MAIN = 512;
+constexpr int DT_THREADS = DT_MAIN + 32;
+constexpr int DT_NB = 4;      // devices per stage
+
+struct alignas(64) DTMaps {
+    CUtensorMap m[DT_MAX_DEV];
+};
+
+struct DTParams {
+    DPParams d;
+    int nstage;
+    int *status;
+};
+
+__host__ __device__ inline size_t dt_stage_bytes() { return (size_t)DT_NB * DT_MAIN * DP_R * 4; }  // CG*RC = DT_MAIN*DP_R words per device
+__host__ __device__ inline size_t dt_smem_bytes(int N, int CG, int nstage)
+{
+    return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes() + (size_t)nstage * 16;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+template <int CG, bool FP32OUT>
+__global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams tp, const __grid_constant__ DTMaps maps)
+{
+    extern __shared__ __align__(128) uint8_t dp_smem[];
+    constexpr int RS = DT_MAIN / CG, RC = RS * DP_R;
+    constexpr uint32_t BOX_BYTES = (uint32_t)CG * RC * 4;
+    constexpr uint32_t STAGE_BYTES = DT_NB * BOX_BYTES;
+    const DPParams &pp = tp.d;
+    const DQParams &p = pp.q;
+    const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
+    const int tid = threadIdx.x, nstage = tp.nstage;
+    float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][2][CG]
+    uint8_t *const ring = dp_smem + dp_steps_bytes(N, CG);
+    uint64_t *full = reinterpret_cast<uint64_t *>(ring + (size_t)nstage * STAGE_BYTES);
+    uint64_t *empty = full + nstage;
+    const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
+
+    if (tid == 0) {
+        for (int s = 0; s < nstage; ++s) {
+            mbar_init(smem_u32(&full[s]), 1);
+            mbar_init(smem_u32(&empty[s]), DT_MAIN / 32);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    // the panel's steps (loads issued before the barrier that releases the producer)
+    for (int a = tid; a < N * CG; a += DT_THREADS) {
+        const int i = a / CG, c = a & (CG - 1), gg = panel * CG + c;
+        float2 s4[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
+        if (gg < L8) load_steps(pp.s_slot + (size_t)i * E, gg, s4);
+        dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
+        dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
+    }
+    const int cg = tid & (CG - 1), rs = tid / CG;
+    const int g = panel * CG + cg;
+    const bool live = tid < DT_MAIN && g < L8;
+    const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
+    __syncthreads();
+
+    if (tid >= DT_MAIN) {
+        // ---------------- producer warp: one lane issues everything
+        if (tid == DT_MAIN) {
+            int st = 0, it = 0;
+            uint32_t parity = 1;
+            for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
+                for (int i0 = 0; i0 < N; i0 += DT_NB, ++it) {
+                    const int nb = (N - i0 < DT_NB) ? N - i0 : DT_NB;
+                    const uint32_t bar = smem_u32(&full[st]);
+                    if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
+                        atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
+                        return;
+                    }
+                    mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
+                    const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
+                    for (int i = 0; i < nb; ++i)
+                        tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
+                    if (++st == nstage) {
+                        st = 0;
+                        parity ^= 1u;
+                    }
+                }
+            }
+        }
+        return;
+    }
+
+    // ---------------- main warps
+    const uint32_t magic = opaque_magic();
+    const int lane = tid & 31;
+    float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
+#pragma unroll
+    for (int h = 0; h < 4; ++h) {
+        bias[h] = kDecodeBias[h];
+        asm volatile("" : "+f"(bias[h].x), "+f"(bias[h].y));
+    }
+    const float4 *const my_steps = dp_steps + cg;
+    const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R) * CG + cg;
+    int st = 0;
+    uint32_t parity = 0;
+    bool ok = true;
+    for (int64_t ch = by; ch < pp.n_chunks && ok; ch += pp.gy) {
+        const int64_t t0 = ch * RC + rs * DP_R;
+        float2 acc[DP_R][4];
+#pragma unroll
+        for (int r = 0; r < DP_R; ++r)
+#pragma unroll
+            for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
+        const float4 *st4 = my_steps;
+        for (int i0 = 0; i0 < N; i0 += DT_NB, st4 += DT_NB * 2 * CG) {
+            if (!mbar_wait(smem_u32(&full[st]), parity)) {
+                atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
+                ok = false;
+                break;
+            }
+            const uint32_t *const sw = ring_w + (size_t)st * (STAGE_BYTES / 4);
+            uint32_t w[DT_NB][DP_R];
+#pragma unroll
+            for (int i = 0; i < DT_NB; ++i)
+#pragma unroll
+                for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * RC + r) * CG];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&empty[st]));  // the stage's words are in registers
+            if (++st == nstage) {
+                st = 0;
+                parity ^= 1u;
+            }
+            if (i0 + DT_NB <= N) {
+#pragma unroll
+                for (int i = 0; i < DT_NB; ++i) {
+                    const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
+                    const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
+                                          make_float2(b.z, b.w)};
+#pragma unroll
+                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < DT_NB; ++i)
+                    if (i0 + i < N) {
+                        const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
+                        const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
+                                              make_float2(b.z, b.w)};
+#pragma unroll
+                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                    }
+            }
+        }
+        if (ok && live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, mask, acc);
+    }
+
+    // every block's share of the BF16 block (main threads)
+    dp_sum_bf16_block<FP32OUT>(p, pp.hp_idx, (int64_t)blockIdx.x * DT_MAIN + tid, (int64_t)gridDim.x * DT_MAIN);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -829,6 +1014,122 @@ cudaError_t launch_panels(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
     }
 }
 
+// ---- tensor maps of the payloads' code sections
+typedef CUresult (*tpq_encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                        const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+tpq_encode_tiled_fn encode_tiled_fn()
+{
+    static tpq_encode_tiled_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<tpq_encode_tiled_fn>(sym);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+// A payload's map depends on its address and on the shape; encoding costs about a microsecond of host time,
+// so the maps of recently seen payloads are kept (callers reuse their communication buffers).
+struct DTCacheEntry {
+    const void *ptr;
+    int64_t T;
+    int L8, CG, RC;
+    CUtensorMap map;
+};
+struct DTCache {
+    static constexpr int CAP = 256;
+    int n = 0, next = 0;
+    DTCacheEntry e[CAP];
+};
+
+bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC, CUtensorMap *out)
+{
+    if (!c->dq_cache) c->dq_cache = new (std::nothrow) DTCache();
+    DTCache *cache = static_cast<DTCache *>(c->dq_cache);
+    if (cache)
+        for (int j = 0; j < cache->n; ++j) {
+            const DTCacheEntry &e = cache->e[j];
+            if (e.ptr == ptr && e.T == T && e.L8 == L8 && e.CG == CG && e.RC == RC) {
+                *out = e.map;
+                return true;
+            }
+        }
+    tpq_encode_tiled_fn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)L8, (cuuint64_t)T};
+    const cuuint64_t strides[1] = {(cuuint64_t)L8 * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)CG, (cuuint32_t)RC};
+    const cuuint32_t estr[2] = {1, 1};
+    CUtensorMap m;
+    if (fn(&m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    if (cache) {
+        DTCacheEntry &e = cache->e[cache->next];
+        e.ptr = ptr; e.T = T; e.L8 = L8; e.CG = CG; e.RC = RC; e.map = m;
+        cache->next = (cache->next + 1) % DTCache::CAP;
+        if (cache->n < DTCache::CAP) ++cache->n;
+    }
+    *out = m;
+    return true;
+}
+
+// Tensor-map panel kernel geometry; false if the shape (or the driver) does not admit it.
+bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &tp, DTMaps &maps)
+{
+    const int N = c->N, E = c->E, k = c->k, L8 = (E - k) / 8;
+    if (N > DT_MAX_DEV || L8 % 4 != 0 || T > 0x7FFFFFF0LL) return false;
+    int CG = 128;
+    while (CG >= 32 && dt_smem_bytes(N, CG, 2) > (size_t)c->smem_optin) CG >>= 1;
+    if (CG < 32) return false;
+    const int RC = DT_MAIN / CG * DP_R;
+    DPParams &pp = tp.d;
+    pp.CG = CG;
+    pp.panels = (L8 + CG - 1) / CG;
+    pp.n_chunks = (T + RC - 1) / RC;
+    if (pp.n_chunks * pp.panels < c->sm_count) return false;  // short inputs: the copy kernel starts faster
+    int64_t gy = c->sm_count / pp.panels;
+    if (gy > pp.n_chunks) gy = pp.n_chunks;
+    if (gy < 1) gy = 1;
+    pp.gy = (int)gy;
+    int nstage = 6;
+    while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
+    tp.nstage = nstage;
+    tp.status = c->t.status;
+    for (int i = 0; i < N; ++i)
+        if (!payload_map(c, payloads[i], T, L8, CG, RC, &maps.m[i])) return false;
+    return true;
+}
+
+template <int CG, bool FP32OUT>
+cudaError_t launch_tpanels_cg(const tpq_ctx *c, const DTParams &tp, const DTMaps &maps, cudaStream_t st)
+{
+    const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage);
+    cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    dequant_tpanels<CG, FP32OUT><<<(unsigned)(tp.d.panels * tp.d.gy), DT_THREADS, smem, st>>>(tp, maps);
+    return cudaGetLastError();
+}
+
+template <bool FP32OUT>
+cudaError_t launch_tpanels(const tpq_ctx *c, const DTParams &tp, const DTMaps &maps, cudaStream_t st)
+{
+    switch (tp.d.CG) {
+    case 128: return launch_tpanels_cg<128, FP32OUT>(c, tp, maps, st);
+    case 64: return launch_tpanels_cg<64, FP32OUT>(c, tp, maps, st);
+    default: return launch_tpanels_cg<32, FP32OUT>(c, tp, maps, st);
+    }
+}
+
 }  // namespace
 
 cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out, int fp32_out,
@@ -863,6 +1164,17 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             return cudaGetLastError();
         }
     }
+    {
+        DTParams tp;
+        DTMaps maps;
+        if (tpanels_plan(const_cast<tpq_ctx *>(c), payloads, T, tp, maps)) {
+            tp.d.q = p;
+            tp.d.s_slot = c->t.s_slot; tp.d.lp_idx = c->t.lp_idx; tp.d.hp_idx = c->t.hp_idx;
+            const cudaError_t e = fp32_out ? launch_tpanels<true>(c, tp, maps, st) : launch_tpanels<false>(c, tp, maps, st);
+            if (e == cudaSuccess) ++*launches;
+            return e;
+        }
+    }
     DPParams dp;
     if (!panels_plan(c, T, dp)) return tpq_launch_dequant_generic(c, payloads, T, out, fp32_out, out_stride, st, launches);
     dp.q = p;
@@ -870,4 +1182,10 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
     const cudaError_t e = fp32_out ? launch_panels<true>(c, dp, st) : launch_panels<false>(c, dp, st);
     if (e == cudaSuccess) ++*launches;
     return e;
+}
+
+void tpq_dequant_release(tpq_ctx *c)
+{
+    delete static_cast<DTCache *>(c->dq_cache);
+    c->dq_cache = nullptr;
 }

@@ -158,6 +158,7 @@ tpq_status tpq_destroy(tpq_ctx *c)
     cudaDeviceSynchronize();
     free_tables(c->t);
     cudaFree(c->scratch);
+    tpq_dequant_release(c);
     delete c;
     return TPQ_OK;
 }

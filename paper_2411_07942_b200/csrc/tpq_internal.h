@@ -41,6 +41,7 @@ struct tpq_ctx {
     void *scratch;      // calibration partial extremes
     size_t scratch_bytes;
     int64_t launches;
+    void *dq_cache;     // tensor maps of recently used payloads (dequant.cu)
     char err[512];
 };
 
@@ -87,6 +88,7 @@ cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n,
 
 // sum_i D^(i): dequantise + reduce.
 bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int fp32_out);
+void tpq_dequant_release(tpq_ctx *c);  // frees dq_cache
 cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,
                                        int fp32_out, int64_t out_stride, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,
