@@ -497,14 +497,15 @@ struct alignas(64) DTMaps {
 
 struct DTParams {
     DPParams d;
-    int nstage;
+    int nstage, n_holes;
+    const int32_t *filler;  // [n_holes] feature whose codes sit in hole tau's slot
     int *status;
 };
 
 __host__ __device__ inline size_t dt_stage_bytes() { return (size_t)DT_NB * DT_MAIN * DP_R * 4; }  // CG*RC = DT_MAIN*DP_R words per device
 __host__ __device__ inline size_t dt_smem_bytes(int N, int CG, int nstage)
 {
-    return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes() + (size_t)nstage * 16;
+    return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes() + (size_t)nstage * 16;  // steps, ring, mbarriers
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
@@ -594,18 +595,62 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     }
     const float4 *const my_steps = dp_steps + cg;
     const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R) * CG + cg;
+
+    // Selected features completed by this block ("items", one per row and rank): the panel's holes, ranks
+    // [hs, he); the last panel also takes the selected features at or above E-k, ranks [n_holes, k).
+    // Main threads store all 8 lanes of every group; a hole's lane holds the sum of the filler feature whose
+    // codes sit in the hole's slot.  After a block barrier (which orders the two stores to the hole's
+    // column) the item thread moves that value to the filler feature's column and writes the selected
+    // feature's own sum -- the devices' BF16 values added in ascending order -- over it.
+    const int n_holes = tp.n_holes;
+    const int hs = (int)(__ldg(p.grp + panel * CG) >> 8);
+    const int he = (panel == pp.panels - 1) ? k : (int)(__ldg(p.grp + (panel + 1) * CG) >> 8);
+    const int n_it = he - hs;                           // items per row
+    const int items = RC * n_it;
+    const int my_r = (tid < items) ? tid / n_it : 0;    // this thread's first item: row of the chunk, rank
+    const int my_h = (tid < items) ? hs + (tid - my_r * n_it) : 0;
+    const int my_col = (tid < items) ? __ldg(pp.hp_idx + my_h) : 0;
+    const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(tp.filler + my_h) : -1;
+
+    auto item_done = [&](int64_t t, int sel_col, int filler_col, float v) {
+        const int64_t orow = t * p.out_stride;
+        if (filler_col >= 0) {
+            if (FP32OUT)
+                static_cast<float *>(p.out)[orow + filler_col] = __ldcg(static_cast<const float *>(p.out) + orow + sel_col);
+            else
+                static_cast<uint16_t *>(p.out)[orow + filler_col] =
+                    __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
+        }
+        store_one<FP32OUT>(p.out, orow + sel_col, v);
+    };
+
     int st = 0;
     uint32_t parity = 0;
     bool ok = true;
     for (int64_t ch = by; ch < pp.n_chunks && ok; ch += pp.gy) {
-        const int64_t t0 = ch * RC + rs * DP_R;
+        const int64_t tc = ch * RC;
+        const int64_t t0 = tc + rs * DP_R;
         float2 acc[DP_R][4];
 #pragma unroll
         for (int r = 0; r < DP_R; ++r)
 #pragma unroll
             for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
+        const bool it_on = tid < items && tc + my_r < p.T;
+        const int64_t it_off = p.lp_bytes + ((tc + my_r) * k + my_h) * 2;
+        float hv = 0.0f;
+        uint16_t hvv[DT_NB] = {};
         const float4 *st4 = my_steps;
         for (int i0 = 0; i0 < N; i0 += DT_NB, st4 += DT_NB * 2 * CG) {
+            if (it_on) {
+                // add the values loaded a step ago (ascending device order), then load this step's
+                if (i0 > 0) {
+#pragma unroll
+                    for (int i = 0; i < DT_NB; ++i) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+                }
+#pragma unroll
+                for (int i = 0; i < DT_NB; ++i)
+                    if (i0 + i < N) hvv[i] = __ldcs(reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + it_off));
+            }
             if (!mbar_wait(smem_u32(&full[st]), parity)) {
                 atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
                 ok = false;
@@ -644,11 +689,29 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                     }
             }
         }
-        if (ok && live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, mask, acc);
+        if (!ok) break;
+        if (it_on) {  // the last step's values (a partial batch has N % DT_NB of them)
+            const int nl = N - (N - 1) / DT_NB * DT_NB;
+#pragma unroll
+            for (int i = 0; i < DT_NB; ++i)
+                if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+        }
+        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+        if (n_it > 0) {
+            asm volatile("bar.sync 1, %0;" ::"n"(DT_MAIN) : "memory");  // the chunk's rows are stored
+            if (it_on) item_done(tc + my_r, my_col, my_fcol, hv);
+            // panels with more items than threads (many selected features in one panel): the rest, unpipelined
+            for (int a = tid + DT_MAIN; a < items; a += DT_MAIN) {
+                const int r = a / n_it, h = hs + (a - r * n_it);
+                if (tc + r >= p.T) break;
+                const int64_t off = p.lp_bytes + ((tc + r) * k + h) * 2;
+                float v = 0.0f;
+                for (int i = 0; i < N; ++i)
+                    v = __fadd_rn(v, __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const uint16_t *>(p.pl[i] + off)) << 16));
+                item_done(tc + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(tp.filler + h) : -1, v);
+            }
+        }
     }
-
-    // every block's share of the BF16 block (main threads)
-    dp_sum_bf16_block<FP32OUT>(p, pp.hp_idx, (int64_t)blockIdx.x * DT_MAIN + tid, (int64_t)gridDim.x * DT_MAIN);
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -1105,6 +1168,8 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
     tp.nstage = nstage;
     tp.status = c->t.status;
+    tp.n_holes = c->n_holes;
+    tp.filler = c->t.filler;
     for (int i = 0; i < N; ++i)
         if (!payload_map(c, payloads[i], T, L8, CG, RC, &maps.m[i])) return false;
     return true;
