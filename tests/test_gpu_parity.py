@@ -67,6 +67,57 @@ def test_tiled_path_shapes(N, T, E, k, pad):
     _full_pipeline(_workload(N, T, E, 7 * E + T), k, binding.PATH_TILED, stride_pad=pad)
 
 
+@pytest.mark.parametrize("N,T,E,k", [(10, 2390, 1024, 32), (16, 1203, 2048, 32), (9, 2401, 1024, 0), (13, 2369, 1024, 64),
+                                     (2, 1195, 8192, 128)])
+def test_tensor_map_panel_kernel_shapes(N, T, E, k):
+    """Shapes that dequant_reduce serves with tiled tensor copies (more than 8 devices or long rows, 16-byte
+    row pitch, i.e. E - k a multiple of 32, and at least 148 row chunks x panels): device counts that are not a multiple of the 4 devices
+    per stage, ragged last chunk, partial last panel, no selected feature at all."""
+    _full_pipeline(_workload(N, T, E, 11 * E + T, calib=(2, 8)), k, binding.PATH_TILED)
+
+
+@pytest.mark.parametrize("N,T,E,k", [(9, 100, 1040, 8), (12, 37, 5120, 80), (33, 21, 1024, 16), (64, 9, 512, 8),
+                                     (9, 300, 4608, 72)])
+def test_copy_ring_panel_kernel_shapes(N, T, E, k):
+    """Shapes served by the asynchronous-copy panel kernel: row pitch not a multiple of 16 bytes, more than
+    16 devices (narrower panels), short inputs."""
+    _full_pipeline(_workload(N, T, E, 13 * E + T, calib=(2, 8)), k, binding.PATH_TILED)
+
+
+def test_panel_kernels_equal_generic_on_clustered_feature_sets():
+    """The panel kernels on arbitrary feature sets: several holes in one group, whole groups, more selected
+    features in a panel than the block has threads, selected features at the very end, nearly everything
+    selected.  N = 9 keeps the row kernel out; T = 2400 reaches the tensor-map kernel, T = 50 the copy ring."""
+    N, E = 9, 1024
+    rng = np.random.default_rng(5)
+    sets = [                                             # sizes are multiples of 32: 16-byte row pitch
+        list(range(0, 32)),
+        list(range(0, 31)) + [1023],
+        list(range(3, 3 + 32)),
+        sorted(rng.permutation(E)[:128].tolist()),
+        sorted(rng.permutation(E)[:512].tolist()),
+        list(range(E - 32, E)),
+        list(range(32, E)),
+        [5, 6, 7, 8, 9, 10] + list(range(100, 340, 10)) + [1000, 1001],
+        list(range(0, 8)),                               # (these two: pitch not a multiple of 16 bytes)
+        list(range(3, 3 + 24)),
+    ]
+    for T in (2400, 50):
+        w = _workload(N, T, E, 31 + T, calib=(2, 8))
+        scale = synth.column_scales(w)
+        cal = [synth.calibration_np(w, i, scale=scale) for i in range(N)]
+        ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+        for hp in sets:
+            t = binding.Tpq(N, E)
+            gu.calibrate_both(t, cal)
+            t.set_features(hp)
+            a = gu.run_sync(t, ys, path=binding.PATH_GENERIC)
+            b = gu.run_sync(t, ys, path=binding.PATH_TILED)
+            for x, y in zip(a, b):
+                assert np.array_equal(x, y)
+            t.close()
+
+
 def test_tiled_equals_generic_on_clustered_feature_sets():
     """Arbitrary feature sets (the paper's random-selection baseline and worse):
     runs of adjacent selected features, whole groups of 8, first and last feature."""
