@@ -351,6 +351,33 @@ def main():
     q_ms = time_loop(q_only, reps) / N          # per single-shard launch
     qb_ms = time_loop(qb_only, reps)            # per batched launch (N shards)
     d_ms = time_loop(d_only, reps)
+    # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
+    # what the launch path costs, relevant for the decode-sized workloads
+    graph_ms = None
+    try:
+        gs = torch.cuda.Stream()
+        gs.wait_stream(stream)
+        gsh = gs.cuda_stream
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=gs):
+            for b in range(args.sets):
+                _, _, out, yarr, parr = sets[b]
+                t.quantize_pack_batch(0, yarr, T, parr, P, stream=gsh)
+                t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=gsh)
+        with torch.cuda.stream(gs):
+            for _ in range(3):
+                graph.replay()
+            ga, gz = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            greps = max(5, min(args.steps, 2000) // args.sets)
+            ga.record(gs)
+            for _ in range(greps):
+                graph.replay()
+            gz.record(gs)
+        torch.cuda.synchronize()
+        graph_ms = ga.elapsed_time(gz) / (greps * args.sets)
+    except Exception as exc:  # measurement only: the step itself does not depend on graphs
+        graph_ms = f"unavailable: {type(exc).__name__}: {exc}"[:200]
+        torch.cuda.synchronize()
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
@@ -405,6 +432,7 @@ def main():
                 "algorithmic_bytes_per_launch": dom_bytes, "launch_ms": dom_ms, "traffic": traffic}
     extra = {
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
+        "step_cuda_graph_replay_ms": graph_ms,
         "payload_bytes_per_shard": int(comm.payload_bytes),
         "comm_bytes_per_rank": {"quantized_allgather": int(comm.quantized_allgather_send),
                                 "bf16_allgather": int(comm.bf16_allgather_send),
