@@ -555,7 +555,9 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     const int g = panel * CG + cg;
     const bool live = tid < DT_MAIN && g < L8;
     const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
+    tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
     __syncthreads();
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
     if (tid >= DT_MAIN) {
         // ---------------- producer warp: one lane issues everything
@@ -810,7 +812,9 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
         for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
     }
+    tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
     __syncthreads();
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
     if (tid >= NT + DR_FIXUP_THREADS) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
@@ -1004,10 +1008,10 @@ cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads,
     cudaError_t e;
     if (fp32_out) {
         e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) dequant_rows<NMAX, MAXT, true><<<grid, threads, smem, st>>>(pp);
+        if (e == cudaSuccess) e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, true>, dim3(grid), dim3(threads), smem, st, pp);
     } else {
         e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) dequant_rows<NMAX, MAXT, false><<<grid, threads, smem, st>>>(pp);
+        if (e == cudaSuccess) e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, false>, dim3(grid), dim3(threads), smem, st, pp);
     }
     return e;
 }
@@ -1181,8 +1185,8 @@ cudaError_t launch_tpanels_cg(const tpq_ctx *c, const DTParams &tp, const DTMaps
     const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage);
     cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dequant_tpanels<CG, FP32OUT><<<(unsigned)(tp.d.panels * tp.d.gy), DT_THREADS, smem, st>>>(tp, maps);
-    return cudaGetLastError();
+    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3((unsigned)(tp.d.panels * tp.d.gy)), dim3(DT_THREADS), smem, st, tp,
+                          maps);
 }
 
 template <bool FP32OUT>

@@ -257,7 +257,9 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         }
         if (tid < k) my_hp = __ldg(p.hp_idx + tid);
     }
+    tpq_grid_dep_wait();    // the input and the payload buffer may still be in use by the kernel ahead
     __syncthreads();
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
     TPQ_MARK(40);
 
     if (tid >= NT) {
@@ -511,7 +513,7 @@ cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n,
     do {                                                                                                             \
         e = cudaFuncSetAttribute(quantize_tiled<GPT, GG, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
                                  (int)smem);                                                                         \
-        if (e == cudaSuccess) quantize_tiled<GPT, GG, TB><<<(unsigned)grid, nt + 32, smem, st>>>(p);                 \
+        if (e == cudaSuccess) e = tpq_launch_pdl(quantize_tiled<GPT, GG, TB>, dim3((unsigned)grid), dim3(nt + 32), smem, st, p); \
     } while (0)
 #define TPQ_QP_LAUNCH_G(GPT, TB)                          \
     do {                                                  \

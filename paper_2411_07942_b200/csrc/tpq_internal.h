@@ -93,3 +93,28 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
                                        int fp32_out, int64_t out_stride, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out,
                                      int fp32_out, int64_t out_stride, cudaStream_t st, int64_t *launches);
+
+// ---- programmatic dependent launch: a kernel launched this way may start (and run its prologue: barrier
+// set-up, loads of the context's tables, which no kernel in flight writes) before the kernel ahead of it in
+// the stream has drained; it must execute tpq_grid_dep_wait() before it touches memory that earlier work in
+// the stream may still read or write.
+#ifdef __CUDACC__
+__device__ __forceinline__ void tpq_grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void tpq_grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t tpq_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
