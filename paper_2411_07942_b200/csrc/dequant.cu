@@ -220,10 +220,10 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
 // depends only on the row's place in the chunk.)  The panel's steps of all N devices IN SLOT ORDER,
 // pre-divided for the in-place decode, live in shared memory ([N][2][CG] float4), so the register cost does
 // not grow with N.  A hole's slot carries the filler feature's step, so its lane accumulates the filler
-// feature's sum and is stored to that feature's column; nothing is stored to a selected feature's column.
-// After its chunks every block sums its share of the devices' BF16 blocks: thread <-> 8 consecutive
-// selected features of a row, one 16-byte load per device, 8 scattered stores.  Code lanes and BF16 sums
-// write disjoint columns, so they need no ordering.
+// feature's sum; every group is stored whole (8 lanes, one 128-bit store).  Item threads (one per row of the
+// chunk and selected feature of the panel) add the devices' BF16 values in ascending order, a step's values
+// loaded one step before they are used; after the next block barrier they move the filler's sum from the
+// hole's column to the filler feature's own column and write the selected feature's sum over it.
 // ----------------------------------------------------------------------------------------------
 #ifndef TPQ_DP_THREADS
 #define TPQ_DP_THREADS 512
@@ -240,6 +240,8 @@ struct DPParams {
     const float *s_slot;    // [N][E] slot-order steps
     const int32_t *lp_idx;  // [E-k] feature of each slot
     const int32_t *hp_idx;  // [k]
+    const int32_t *filler;  // [n_holes] feature whose codes sit in hole tau's slot
+    int n_holes;
     int CG, panels, gy;
     int64_t n_chunks;
 };
@@ -263,49 +265,6 @@ template <int PENDING>
 __device__ __forceinline__ void cp_async_wait()
 {
     asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory");
-}
-
-// the BF16 block: thread <-> 8 consecutive selected features of a row; items first, first + stride, ...
-template <bool FP32OUT>
-__device__ __forceinline__ void dp_sum_bf16_block(const DQParams &p, const int32_t *hp_idx, int64_t first, int64_t stride)
-{
-    const int N = p.N, k = p.k;
-    const int k8 = k >> 3;
-    const int64_t items = p.T * k8;
-    for (int64_t a = first; a < items; a += stride) {
-        const int64_t t = a / k8;
-        const int h8 = (int)(a - t * k8);
-        const int64_t off = p.lp_bytes + (t * k + 8 * h8) * 2;
-        float2 acc[4];
-#pragma unroll
-        for (int h = 0; h < 4; ++h) acc[h] = make_float2(0.0f, 0.0f);
-        for (int i0 = 0; i0 < N; i0 += 8) {
-            uint4 v[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i0 + i < N) v[i] = __ldcs(reinterpret_cast<const uint4 *>(p.pl[i0 + i] + off));
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (i0 + i < N) {
-                    const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-#pragma unroll
-                    for (int h = 0; h < 4; ++h)
-                        acc[h] = __fadd2_rn(acc[h], make_float2(__uint_as_float(w[h] << 16),
-                                                                __uint_as_float(w[h] & 0xFFFF0000u)));
-                }
-        }
-        const int4 c0 = __ldg(reinterpret_cast<const int4 *>(hp_idx + 8 * h8));
-        const int4 c1 = __ldg(reinterpret_cast<const int4 *>(hp_idx + 8 * h8) + 1);
-        const int64_t orow = t * p.out_stride;
-        store_one<FP32OUT>(p.out, orow + c0.x, acc[0].x);
-        store_one<FP32OUT>(p.out, orow + c0.y, acc[0].y);
-        store_one<FP32OUT>(p.out, orow + c0.z, acc[1].x);
-        store_one<FP32OUT>(p.out, orow + c0.w, acc[1].y);
-        store_one<FP32OUT>(p.out, orow + c1.x, acc[2].x);
-        store_one<FP32OUT>(p.out, orow + c1.y, acc[2].y);
-        store_one<FP32OUT>(p.out, orow + c1.z, acc[3].x);
-        store_one<FP32OUT>(p.out, orow + c1.w, acc[3].y);
-    }
 }
 
 // a thread's DP_R rows of sums -> the output; lane n of a hole's slot holds the sum of the filler feature
@@ -408,7 +367,6 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
         dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
         dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
     }
-    const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
     const uint32_t magic = opaque_magic();
     float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
 #pragma unroll
@@ -427,8 +385,58 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
     const float4 *const my_steps = dp_steps + cg;
     const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring);
     const uint32_t *sw = ring_w;
+
+    // Selected features completed by this block ("items", one per row and rank): the panel's holes, ranks
+    // [hs, he); the last panel also takes the selected features at or above E-k, ranks [n_holes, k).
+    // Threads store all 8 lanes of every group; a hole's lane holds the sum of the filler feature whose
+    // codes sit in the hole's slot.  After the next block barrier (which orders the two stores to the hole's
+    // column) the item thread moves that value to the filler feature's column and writes the selected
+    // feature's own sum -- the devices' BF16 values added in ascending order -- over it.
+    const int n_holes = pp.n_holes;
+    const int hs = (int)(__ldg(p.grp + panel * CG) >> 8);
+    const int he = (panel == pp.panels - 1) ? k : (int)(__ldg(p.grp + (panel + 1) * CG) >> 8);
+    const int n_it = he - hs;                           // items per row
+    const int items = RC * n_it;
+    const int my_r = (tid < items) ? tid / n_it : 0;    // this thread's first item: row of the chunk, rank
+    const int my_h = (tid < items) ? hs + (tid - my_r * n_it) : 0;
+    const int my_col = (tid < items) ? __ldg(pp.hp_idx + my_h) : 0;
+    const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(pp.filler + my_h) : -1;
+    auto item_done = [&](int64_t t, int sel_col, int filler_col, float v) {
+        const int64_t orow = t * p.out_stride;
+        if (filler_col >= 0) {
+            if (FP32OUT)
+                static_cast<float *>(p.out)[orow + filler_col] = __ldcg(static_cast<const float *>(p.out) + orow + sel_col);
+            else
+                static_cast<uint16_t *>(p.out)[orow + filler_col] =
+                    __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
+        }
+        store_one<FP32OUT>(p.out, orow + sel_col, v);
+    };
+    // the items of the chunk whose first row is tcp: this thread's pipelined one (sum v) and, in panels with
+    // more items than threads, the rest
+    auto fixup = [&](int64_t tcp, bool on, float v) {
+        if (on) item_done(tcp + my_r, my_col, my_fcol, v);
+        for (int a = tid + DP_THREADS; a < items; a += DP_THREADS) {
+            const int r = a / n_it, h = hs + (a - r * n_it);
+            if (tcp + r >= p.T) break;
+            const int64_t off = p.lp_bytes + ((tcp + r) * k + h) * 2;
+            float u = 0.0f;
+            for (int i = 0; i < N; ++i)
+                u = __fadd_rn(u, __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const uint16_t *>(p.pl[i] + off)) << 16));
+            item_done(tcp + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(pp.filler + h) : -1, u);
+        }
+    };
+    bool pend = false, pend_on = false;
+    float pend_v = 0.0f;
+    int64_t pend_tc = 0;
+
     for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
-        const int64_t t0 = ch * RC + rs * DP_R;
+        const int64_t tc = ch * RC;
+        const int64_t t0 = tc + rs * DP_R;
+        const bool it_on = tid < items && tc + my_r < p.T;
+        const int64_t it_off = p.lp_bytes + ((tc + my_r) * k + my_h) * 2;
+        float hv = 0.0f;
+        uint16_t hvv[DP_NB] = {};
         float2 acc[DP_R][4];
 #pragma unroll
         for (int r = 0; r < DP_R; ++r)
@@ -439,6 +447,20 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
             cp_async_wait<DP_STAGES - 2>();  // this thread's pieces of the step have landed ...
             __syncthreads();                 // ... and everybody's; the stage consumed last is free
             issue();
+            if (pend) {  // (first step of a chunk) the barrier above is also behind the previous chunk's row stores
+                if (n_it > 0) fixup(pend_tc, pend_on, pend_v);
+                pend = false;
+            }
+            if (it_on) {
+                // add the values loaded a step ago (ascending device order), then load this step's
+                if (i0 > 0) {
+#pragma unroll
+                    for (int i = 0; i < DP_NB; ++i) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+                }
+#pragma unroll
+                for (int i = 0; i < DP_NB; ++i)
+                    if (i0 + i < N) hvv[i] = __ldcs(reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + it_off));
+            }
             uint32_t w[DP_NB][DP_R];
 #pragma unroll
             for (int i = 0; i < DP_NB; ++i)
@@ -467,12 +489,23 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                     }
             }
         }
-        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, mask, acc);
+        if (it_on) {  // the last step's values (a partial batch has N % DP_NB of them)
+            const int nl = N - (N - 1) / DP_NB * DP_NB;
+#pragma unroll
+            for (int i = 0; i < DP_NB; ++i)
+                if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+        }
+        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+        pend = true;
+        pend_on = it_on;
+        pend_v = hv;
+        pend_tc = tc;
     }
     cp_async_wait<0>();
-
-    // every block's share of the BF16 block
-    dp_sum_bf16_block<FP32OUT>(p, pp.hp_idx, (int64_t)blockIdx.x * DP_THREADS + tid, (int64_t)gridDim.x * DP_THREADS);
+    if (pend) {
+        __syncthreads();
+        if (n_it > 0) fixup(pend_tc, pend_on, pend_v);
+    }
 }
 
 // ----------------------------------------------------------------------------------------------
@@ -497,8 +530,7 @@ struct alignas(64) DTMaps {
 
 struct DTParams {
     DPParams d;
-    int nstage, n_holes;
-    const int32_t *filler;  // [n_holes] feature whose codes sit in hole tau's slot
+    int nstage;
     int *status;
 };
 
@@ -604,7 +636,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     // codes sit in the hole's slot.  After a block barrier (which orders the two stores to the hole's
     // column) the item thread moves that value to the filler feature's column and writes the selected
     // feature's own sum -- the devices' BF16 values added in ascending order -- over it.
-    const int n_holes = tp.n_holes;
+    const int n_holes = pp.n_holes;
     const int hs = (int)(__ldg(p.grp + panel * CG) >> 8);
     const int he = (panel == pp.panels - 1) ? k : (int)(__ldg(p.grp + (panel + 1) * CG) >> 8);
     const int n_it = he - hs;                           // items per row
@@ -612,7 +644,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     const int my_r = (tid < items) ? tid / n_it : 0;    // this thread's first item: row of the chunk, rank
     const int my_h = (tid < items) ? hs + (tid - my_r * n_it) : 0;
     const int my_col = (tid < items) ? __ldg(pp.hp_idx + my_h) : 0;
-    const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(tp.filler + my_h) : -1;
+    const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(pp.filler + my_h) : -1;
 
     auto item_done = [&](int64_t t, int sel_col, int filler_col, float v) {
         const int64_t orow = t * p.out_stride;
@@ -710,7 +742,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                 float v = 0.0f;
                 for (int i = 0; i < N; ++i)
                     v = __fadd_rn(v, __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const uint16_t *>(p.pl[i] + off)) << 16));
-                item_done(tc + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(tp.filler + h) : -1, v);
+                item_done(tc + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(pp.filler + h) : -1, v);
             }
         }
     }
@@ -1172,8 +1204,6 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
     tp.nstage = nstage;
     tp.status = c->t.status;
-    tp.n_holes = c->n_holes;
-    tp.filler = c->t.filler;
     for (int i = 0; i < N; ++i)
         if (!payload_map(c, payloads[i], T, L8, CG, RC, &maps.m[i])) return false;
     return true;
@@ -1239,6 +1269,7 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
         if (tpanels_plan(const_cast<tpq_ctx *>(c), payloads, T, tp, maps)) {
             tp.d.q = p;
             tp.d.s_slot = c->t.s_slot; tp.d.lp_idx = c->t.lp_idx; tp.d.hp_idx = c->t.hp_idx;
+            tp.d.filler = c->t.filler; tp.d.n_holes = c->n_holes;
             const cudaError_t e = fp32_out ? launch_tpanels<true>(c, tp, maps, st) : launch_tpanels<false>(c, tp, maps, st);
             if (e == cudaSuccess) ++*launches;
             return e;
@@ -1248,6 +1279,7 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
     if (!panels_plan(c, T, dp)) return tpq_launch_dequant_generic(c, payloads, T, out, fp32_out, out_stride, st, launches);
     dp.q = p;
     dp.s_slot = c->t.s_slot; dp.lp_idx = c->t.lp_idx; dp.hp_idx = c->t.hp_idx;
+    dp.filler = c->t.filler; dp.n_holes = c->n_holes;
     const cudaError_t e = fp32_out ? launch_panels<true>(c, dp, st) : launch_panels<false>(c, dp, st);
     if (e == cudaSuccess) ++*launches;
     return e;
