@@ -355,6 +355,8 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
         }
         cp_async_commit();  // (possibly empty: keeps the group count in step with the consumer)
     };
+    tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 #pragma unroll
     for (int s = 0; s < DP_STAGES - 1; ++s) issue();
 
@@ -749,7 +751,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 }
 
 // ----------------------------------------------------------------------------------------------
-// Row kernel for N <= 8 devices and (E-k)/8 <= MAXT main threads.
+// Row kernel for N <= 4 devices, (E-k)/8 <= MAXT main threads and long inputs.
 //
 // One persistent block per SM with three kinds of warps:
 //   producer (1 warp)  streams groups of G rows of all N payloads (a code-row block and a BF16 block per
@@ -1053,8 +1055,10 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
 {
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
-    if (N > 8) return false;
-    if (L8 > (N <= 4 ? 768 : 576)) return false;  // consumer threads (register budget per thread)
+    // measured against the panel kernels: the row kernel wins only with few devices and at least about ten
+    // rows per SM (the panel kernels start faster and scale better with N)
+    if (N > 4 || T < 10LL * c->sm_count) return false;
+    if (L8 > 768) return false;  // consumer threads (register budget per thread)
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
     else if (L8 % 2 == 0) g0 = 2;
@@ -1099,8 +1103,7 @@ cudaError_t launch_panels_cg(const tpq_ctx *c, const DPParams &pp, cudaStream_t 
     const size_t smem = dp_smem_bytes(c->N, CG);
     cudaError_t e = cudaFuncSetAttribute(dequant_panels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    dequant_panels<CG, FP32OUT><<<(unsigned)(pp.panels * pp.gy), DP_THREADS, smem, st>>>(pp);
-    return cudaGetLastError();
+    return tpq_launch_pdl(dequant_panels<CG, FP32OUT>, dim3((unsigned)(pp.panels * pp.gy)), dim3(DP_THREADS), smem, st, pp);
 }
 
 template <bool FP32OUT>
@@ -1253,11 +1256,8 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             if (consumers < 32) consumers = 32;
             const int threads = consumers + DR_FIXUP_THREADS + 32;
             cudaError_t e;
-            if (c->N <= 4)
-                e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, threads, smem, st)
-                                     : launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st);
-            else
-                e = launch_rows<8, 576>(pp, fp32_out, grid, threads, smem, st);
+            e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, threads, smem, st)
+                                 : launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st);
             if (e != cudaSuccess) return e;
             ++*launches;
             return cudaGetLastError();

@@ -118,6 +118,34 @@ def test_panel_kernels_equal_generic_on_clustered_feature_sets():
             t.close()
 
 
+@pytest.mark.parametrize("N,T,E,k,pad", [(4, 1501, 5120, 80, 0), (2, 1999, 1024, 16, 8), (3, 1600, 4608, 72, 0),
+                                         (1, 1481, 256, 8, 0), (4, 1537, 512, 0, 0), (2, 1490, 6144, 96, 0)])
+def test_row_kernel_shapes(N, T, E, k, pad):
+    """Shapes that dequant_reduce serves with the row kernel (at most 4 devices, at least ten rows per SM):
+    ragged last stage, odd rows-per-stage alignment classes of (E-k)/8, strided input, no selected feature."""
+    _full_pipeline(_workload(N, T, E, 17 * E + T, calib=(2, 8)), k, binding.PATH_TILED, stride_pad=pad)
+
+
+def test_row_kernel_equals_generic_on_clustered_feature_sets():
+    N, T, E = 3, 1500, 512
+    w = _workload(N, T, E, 78, calib=(2, 8))
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, scale=scale) for i in range(N)]
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+    rng = np.random.default_rng(2)
+    sets = [list(range(0, 8)), list(range(0, 15)) + [511], list(range(3, 3 + 24)),
+            sorted(rng.permutation(E)[:64].tolist()), list(range(E - 8, E)), list(range(8, E))]
+    for hp in sets:
+        t = binding.Tpq(N, E)
+        gu.calibrate_both(t, cal)
+        t.set_features(hp)
+        a = gu.run_sync(t, ys, path=binding.PATH_GENERIC)
+        b = gu.run_sync(t, ys, path=binding.PATH_TILED)
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+        t.close()
+
+
 def test_tiled_equals_generic_on_clustered_feature_sets():
     """Arbitrary feature sets (the paper's random-selection baseline and worse):
     runs of adjacent selected features, whole groups of 8, first and last feature."""
