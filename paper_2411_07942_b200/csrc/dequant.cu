@@ -561,11 +561,16 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     const DQParams &p = pp.q;
     const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
     const int tid = threadIdx.x, nstage = tp.nstage;
+    const int lane = tid & 31;
     float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][2][CG]
     uint8_t *const ring = dp_smem + dp_steps_bytes(N, CG);
     uint64_t *full = reinterpret_cast<uint64_t *>(ring + (size_t)nstage * STAGE_BYTES);
     uint64_t *empty = full + nstage;
-    const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
+
+    // Work items are (panel, chunk) pairs, panel-major; the blocks take equal contiguous runs of them, so a
+    // block works on one panel, or on the end of one and the start of the next ("segments").
+    const int64_t total = (int64_t)pp.panels * pp.n_chunks;
+    const int64_t f0 = total * blockIdx.x / gridDim.x, f1 = total * (blockIdx.x + 1) / gridDim.x;
 
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
@@ -575,54 +580,8 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    // the panel's steps (loads issued before the barrier that releases the producer)
-    for (int a = tid; a < N * CG; a += DT_THREADS) {
-        const int i = a / CG, c = a & (CG - 1), gg = panel * CG + c;
-        float2 s4[4];
-#pragma unroll
-        for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
-        if (gg < L8) load_steps(pp.s_slot + (size_t)i * E, gg, s4);
-        dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
-        dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
-    }
     const int cg = tid & (CG - 1), rs = tid / CG;
-    const int g = panel * CG + cg;
-    const bool live = tid < DT_MAIN && g < L8;
-    const uint32_t mask = live ? (__ldg(p.grp + g) & 0xFFu) : 0u;
-    tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
-    __syncthreads();
-    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
-
-    if (tid >= DT_MAIN) {
-        // ---------------- producer warp: one lane issues everything
-        if (tid == DT_MAIN) {
-            int st = 0, it = 0;
-            uint32_t parity = 1;
-            for (int64_t ch = by; ch < pp.n_chunks; ch += pp.gy) {
-                for (int i0 = 0; i0 < N; i0 += DT_NB, ++it) {
-                    const int nb = (N - i0 < DT_NB) ? N - i0 : DT_NB;
-                    const uint32_t bar = smem_u32(&full[st]);
-                    if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
-                        atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
-                        return;
-                    }
-                    mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
-                    const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
-                    for (int i = 0; i < nb; ++i)
-                        tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
-                    if (++st == nstage) {
-                        st = 0;
-                        parity ^= 1u;
-                    }
-                }
-            }
-        }
-        return;
-    }
-
-    // ---------------- main warps
     const uint32_t magic = opaque_magic();
-    const int lane = tid & 31;
     float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
@@ -631,122 +590,170 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     }
     const float4 *const my_steps = dp_steps + cg;
     const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R) * CG + cg;
+    // ring state: the producer lane and the main warps walk the same sequence of stages across segments
+    int st = 0, it = 0;
+    uint32_t parity = (tid >= DT_MAIN) ? 1u : 0u;  // producer: parity of the "empty" phase to wait for
 
-    // Selected features completed by this block ("items", one per row and rank): the panel's holes, ranks
-    // [hs, he); the last panel also takes the selected features at or above E-k, ranks [n_holes, k).
-    // Main threads store all 8 lanes of every group; a hole's lane holds the sum of the filler feature whose
-    // codes sit in the hole's slot.  After a block barrier (which orders the two stores to the hole's
-    // column) the item thread moves that value to the filler feature's column and writes the selected
-    // feature's own sum -- the devices' BF16 values added in ascending order -- over it.
-    const int n_holes = pp.n_holes;
-    const int hs = (int)(__ldg(p.grp + panel * CG) >> 8);
-    const int he = (panel == pp.panels - 1) ? k : (int)(__ldg(p.grp + (panel + 1) * CG) >> 8);
-    const int n_it = he - hs;                           // items per row
-    const int items = RC * n_it;
-    const int my_r = (tid < items) ? tid / n_it : 0;    // this thread's first item: row of the chunk, rank
-    const int my_h = (tid < items) ? hs + (tid - my_r * n_it) : 0;
-    const int my_col = (tid < items) ? __ldg(pp.hp_idx + my_h) : 0;
-    const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(pp.filler + my_h) : -1;
-
-    auto item_done = [&](int64_t t, int sel_col, int filler_col, float v) {
-        const int64_t orow = t * p.out_stride;
-        if (filler_col >= 0) {
-            if (FP32OUT)
-                static_cast<float *>(p.out)[orow + filler_col] = __ldcg(static_cast<const float *>(p.out) + orow + sel_col);
-            else
-                static_cast<uint16_t *>(p.out)[orow + filler_col] =
-                    __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
+    for (int64_t f = f0; f < f1;) {
+        const int panel = (int)(f / pp.n_chunks);
+        const int64_t chb = f - (int64_t)panel * pp.n_chunks;
+        const int64_t che = (pp.n_chunks - chb < f1 - f) ? pp.n_chunks : chb + (f1 - f);
+        __syncthreads();  // (the previous segment's steps are no longer read; first time: the barriers exist)
+        // the panel's steps (loads issued before the barrier that releases the producer)
+        for (int a = tid; a < N * CG; a += DT_THREADS) {
+            const int i = a / CG, c = a & (CG - 1), gg = panel * CG + c;
+            float2 s4[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
+            if (gg < L8) load_steps(pp.s_slot + (size_t)i * E, gg, s4);
+            dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
+            dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
         }
-        store_one<FP32OUT>(p.out, orow + sel_col, v);
-    };
+        const int g = panel * CG + cg;
+        const bool live = tid < DT_MAIN && g < L8;
+        if (f == f0) tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
+        __syncthreads();
+        if (f == f0) tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
-    int st = 0;
-    uint32_t parity = 0;
-    bool ok = true;
-    for (int64_t ch = by; ch < pp.n_chunks && ok; ch += pp.gy) {
-        const int64_t tc = ch * RC;
-        const int64_t t0 = tc + rs * DP_R;
-        float2 acc[DP_R][4];
-#pragma unroll
-        for (int r = 0; r < DP_R; ++r)
-#pragma unroll
-            for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-        const bool it_on = tid < items && tc + my_r < p.T;
-        const int64_t it_off = p.lp_bytes + ((tc + my_r) * k + my_h) * 2;
-        float hv = 0.0f;
-        uint16_t hvv[DT_NB] = {};
-        const float4 *st4 = my_steps;
-        for (int i0 = 0; i0 < N; i0 += DT_NB, st4 += DT_NB * 2 * CG) {
-            if (it_on) {
-                // add the values loaded a step ago (ascending device order), then load this step's
-                if (i0 > 0) {
-#pragma unroll
-                    for (int i = 0; i < DT_NB; ++i) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+        if (tid >= DT_MAIN) {
+            // ---------------- producer warp: one lane issues everything
+            if (tid == DT_MAIN) {
+                for (int64_t ch = chb; ch < che; ++ch) {
+                    for (int i0 = 0; i0 < N; i0 += DT_NB, ++it) {
+                        const int nb = (N - i0 < DT_NB) ? N - i0 : DT_NB;
+                        const uint32_t bar = smem_u32(&full[st]);
+                        if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
+                            atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
+                            return;
+                        }
+                        mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
+                        const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
+                        for (int i = 0; i < nb; ++i)
+                            tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
+                        if (++st == nstage) {
+                            st = 0;
+                            parity ^= 1u;
+                        }
+                    }
                 }
+            }
+            f += che - chb;
+            continue;
+        }
+
+        // ---------------- main warps
+        // Selected features completed for this panel ("items", one per row and rank): the panel's holes,
+        // ranks [hs, he); the last panel also takes the selected features at or above E-k, ranks [n_holes, k).
+        // Main threads store all 8 lanes of every group; a hole's lane holds the sum of the filler feature
+        // whose codes sit in the hole's slot.  After a barrier among the main warps (which orders the two
+        // stores to the hole's column) the item thread moves that value to the filler feature's column and
+        // writes the selected feature's own sum -- the devices' BF16 values added in ascending order -- over it.
+        const int n_holes = pp.n_holes;
+        const int hs = (int)(__ldg(p.grp + panel * CG) >> 8);
+        const int he = (panel == pp.panels - 1) ? k : (int)(__ldg(p.grp + (panel + 1) * CG) >> 8);
+        const int n_it = he - hs;                           // items per row
+        const int items = RC * n_it;
+        const int my_r = (tid < items) ? tid / n_it : 0;    // this thread's first item: row of the chunk, rank
+        const int my_h = (tid < items) ? hs + (tid - my_r * n_it) : 0;
+        const int my_col = (tid < items) ? __ldg(pp.hp_idx + my_h) : 0;
+        const int my_fcol = (tid < items && my_h < n_holes) ? __ldg(pp.filler + my_h) : -1;
+        auto item_done = [&](int64_t t, int sel_col, int filler_col, float v) {
+            const int64_t orow = t * p.out_stride;
+            if (filler_col >= 0) {
+                if (FP32OUT)
+                    static_cast<float *>(p.out)[orow + filler_col] =
+                        __ldcg(static_cast<const float *>(p.out) + orow + sel_col);
+                else
+                    static_cast<uint16_t *>(p.out)[orow + filler_col] =
+                        __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
+            }
+            store_one<FP32OUT>(p.out, orow + sel_col, v);
+        };
+
+        for (int64_t ch = chb; ch < che; ++ch) {
+            const int64_t tc = ch * RC;
+            const int64_t t0 = tc + rs * DP_R;
+            float2 acc[DP_R][4];
+#pragma unroll
+            for (int r = 0; r < DP_R; ++r)
+#pragma unroll
+                for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
+            const bool it_on = tid < items && tc + my_r < p.T;
+            const int64_t it_off = p.lp_bytes + ((tc + my_r) * k + my_h) * 2;
+            float hv = 0.0f;
+            uint16_t hvv[DT_NB] = {};
+            const float4 *st4 = my_steps;
+            for (int i0 = 0; i0 < N; i0 += DT_NB, st4 += DT_NB * 2 * CG) {
+                if (it_on) {
+                    // add the values loaded a step ago (ascending device order), then load this step's
+                    if (i0 > 0) {
+#pragma unroll
+                        for (int i = 0; i < DT_NB; ++i) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+                    }
+#pragma unroll
+                    for (int i = 0; i < DT_NB; ++i)
+                        if (i0 + i < N) hvv[i] = __ldcs(reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + it_off));
+                }
+                if (!mbar_wait(smem_u32(&full[st]), parity)) {
+                    atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
+                    return;
+                }
+                const uint32_t *const sw = ring_w + (size_t)st * (STAGE_BYTES / 4);
+                uint32_t w[DT_NB][DP_R];
 #pragma unroll
                 for (int i = 0; i < DT_NB; ++i)
-                    if (i0 + i < N) hvv[i] = __ldcs(reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + it_off));
-            }
-            if (!mbar_wait(smem_u32(&full[st]), parity)) {
-                atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
-                ok = false;
-                break;
-            }
-            const uint32_t *const sw = ring_w + (size_t)st * (STAGE_BYTES / 4);
-            uint32_t w[DT_NB][DP_R];
 #pragma unroll
-            for (int i = 0; i < DT_NB; ++i)
-#pragma unroll
-                for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * RC + r) * CG];
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&empty[st]));  // the stage's words are in registers
-            if (++st == nstage) {
-                st = 0;
-                parity ^= 1u;
-            }
-            if (i0 + DT_NB <= N) {
-#pragma unroll
-                for (int i = 0; i < DT_NB; ++i) {
-                    const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
-                    const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
-                                          make_float2(b.z, b.w)};
-#pragma unroll
-                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                    for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * RC + r) * CG];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&empty[st]));  // the stage's words are in registers
+                if (++st == nstage) {
+                    st = 0;
+                    parity ^= 1u;
                 }
-            } else {
+                if (i0 + DT_NB <= N) {
 #pragma unroll
-                for (int i = 0; i < DT_NB; ++i)
-                    if (i0 + i < N) {
+                    for (int i = 0; i < DT_NB; ++i) {
                         const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
                         const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                               make_float2(b.z, b.w)};
 #pragma unroll
                         for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
                     }
-            }
-        }
-        if (!ok) break;
-        if (it_on) {  // the last step's values (a partial batch has N % DT_NB of them)
-            const int nl = N - (N - 1) / DT_NB * DT_NB;
+                } else {
 #pragma unroll
-            for (int i = 0; i < DT_NB; ++i)
-                if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
-        }
-        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
-        if (n_it > 0) {
-            asm volatile("bar.sync 1, %0;" ::"n"(DT_MAIN) : "memory");  // the chunk's rows are stored
-            if (it_on) item_done(tc + my_r, my_col, my_fcol, hv);
-            // panels with more items than threads (many selected features in one panel): the rest, unpipelined
-            for (int a = tid + DT_MAIN; a < items; a += DT_MAIN) {
-                const int r = a / n_it, h = hs + (a - r * n_it);
-                if (tc + r >= p.T) break;
-                const int64_t off = p.lp_bytes + ((tc + r) * k + h) * 2;
-                float v = 0.0f;
-                for (int i = 0; i < N; ++i)
-                    v = __fadd_rn(v, __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const uint16_t *>(p.pl[i] + off)) << 16));
-                item_done(tc + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(pp.filler + h) : -1, v);
+                    for (int i = 0; i < DT_NB; ++i)
+                        if (i0 + i < N) {
+                            const float4 a = st4[(2 * i) * CG], b = st4[(2 * i + 1) * CG];
+                            const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
+                                                  make_float2(b.z, b.w)};
+#pragma unroll
+                            for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                        }
+                }
+            }
+            if (it_on) {  // the last step's values (a partial batch has N % DT_NB of them)
+                const int nl = N - (N - 1) / DT_NB * DT_NB;
+#pragma unroll
+                for (int i = 0; i < DT_NB; ++i)
+                    if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
+            }
+            if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+            if (n_it > 0) {
+                asm volatile("bar.sync 1, %0;" ::"n"(DT_MAIN) : "memory");  // the chunk's rows are stored
+                if (it_on) item_done(tc + my_r, my_col, my_fcol, hv);
+                // panels with more items than threads (many selected features in one panel): the rest, unpipelined
+                for (int a = tid + DT_MAIN; a < items; a += DT_MAIN) {
+                    const int r = a / n_it, h = hs + (a - r * n_it);
+                    if (tc + r >= p.T) break;
+                    const int64_t off = p.lp_bytes + ((tc + r) * k + h) * 2;
+                    float v = 0.0f;
+                    for (int i = 0; i < N; ++i)
+                        v = __fadd_rn(v, __uint_as_float((uint32_t)__ldcs(reinterpret_cast<const uint16_t *>(p.pl[i] + off)) << 16));
+                    item_done(tc + r, __ldg(pp.hp_idx + h), h < n_holes ? __ldg(pp.filler + h) : -1, v);
+                }
             }
         }
+        f += che - chb;
     }
 }
 
@@ -1199,10 +1206,7 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     pp.panels = (L8 + CG - 1) / CG;
     pp.n_chunks = (T + RC - 1) / RC;
     if (pp.n_chunks * pp.panels < c->sm_count) return false;  // short inputs: the copy kernel starts faster
-    int64_t gy = c->sm_count / pp.panels;
-    if (gy > pp.n_chunks) gy = pp.n_chunks;
-    if (gy < 1) gy = 1;
-    pp.gy = (int)gy;
+    pp.gy = 0;  // (unused: the blocks take equal runs of (panel, chunk) pairs)
     int nstage = 6;
     while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
     tp.nstage = nstage;
@@ -1218,8 +1222,7 @@ cudaError_t launch_tpanels_cg(const tpq_ctx *c, const DTParams &tp, const DTMaps
     const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage);
     cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3((unsigned)(tp.d.panels * tp.d.gy)), dim3(DT_THREADS), smem, st, tp,
-                          maps);
+    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3((unsigned)c->sm_count), dim3(DT_THREADS), smem, st, tp, maps);
 }
 
 template <bool FP32OUT>
