@@ -64,6 +64,17 @@ class COracle:
         L.tpqo_dequant_reduce.argtypes = [ctypes.POINTER(u8p), i64, i64, i64, i32p, i64, f32p,
                                           ctypes.POINTER(ctypes.c_double), f32p]
         L.tpqo_round_bf16_f32.argtypes = [f32p, i64, u16p]
+        ci = ctypes.c_int
+        L.tpqo_params_b.argtypes = [f32p, i64, ci, f32p, f32p]
+        L.tpqo_lp_bytes_b.argtypes = [i64, i64, i64, ci]
+        L.tpqo_lp_bytes_b.restype = i64
+        L.tpqo_payload_bytes_b.argtypes = [i64, i64, i64, ci]
+        L.tpqo_payload_bytes_b.restype = i64
+        L.tpqo_quantize_one_b.argtypes = [ctypes.c_uint16, f32, ci]
+        L.tpqo_quantize_one_b.restype = ctypes.c_int
+        L.tpqo_quantize_pack_b.argtypes = [u16p, i64, i64, i64, i32p, i64, f32p, ci, u8p]
+        L.tpqo_dequant_reduce_b.argtypes = [ctypes.POINTER(u8p), i64, i64, i64, i32p, i64, f32p, ci,
+                                            ctypes.POINTER(ctypes.c_double), f32p]
 
     def num_threads(self) -> int:
         return int(self.lib.tpqo_num_threads())
@@ -107,20 +118,28 @@ class COracle:
         self.lib.tpqo_select(_ptr(Rbar, ctypes.c_float), Rbar.shape[0], k, _ptr(out, ctypes.c_int32))
         return out[:k].copy()
 
-    def params(self, R: np.ndarray):
+    def params(self, R: np.ndarray, bits: int = 4):
         R = np.ascontiguousarray(R, dtype=np.float32)
         s = np.empty_like(R)
         inv_s = np.empty_like(R)
-        self.lib.tpqo_params(_ptr(R, ctypes.c_float), R.size, _ptr(s, ctypes.c_float),
-                             _ptr(inv_s, ctypes.c_float))
+        if bits == 4:
+            self.lib.tpqo_params(_ptr(R, ctypes.c_float), R.size, _ptr(s, ctypes.c_float),
+                                 _ptr(inv_s, ctypes.c_float))
+        else:
+            self.lib.tpqo_params_b(_ptr(R, ctypes.c_float), R.size, bits, _ptr(s, ctypes.c_float),
+                                   _ptr(inv_s, ctypes.c_float))
         return s, inv_s
 
     # ---- payload
-    def lp_bytes(self, T: int, E: int, k: int) -> int:
-        return int(self.lib.tpqo_lp_bytes(T, E, k))
+    def lp_bytes(self, T: int, E: int, k: int, bits: int = 4) -> int:
+        if bits == 4:
+            return int(self.lib.tpqo_lp_bytes(T, E, k))
+        return int(self.lib.tpqo_lp_bytes_b(T, E, k, bits))
 
-    def payload_bytes(self, T: int, E: int, k: int) -> int:
-        return int(self.lib.tpqo_payload_bytes(T, E, k))
+    def payload_bytes(self, T: int, E: int, k: int, bits: int = 4) -> int:
+        if bits == 4:
+            return int(self.lib.tpqo_payload_bytes(T, E, k))
+        return int(self.lib.tpqo_payload_bytes_b(T, E, k, bits))
 
     def lp_index(self, E: int, hp_idx) -> np.ndarray:
         """Feature held by each code slot (the payload's slot order)."""
@@ -131,24 +150,30 @@ class COracle:
         self.lib.tpqo_slot_order(E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(out, ctypes.c_int32))
         return out[: E - k].copy()
 
-    def quantize_one(self, x_bits: int, inv_s: float) -> int:
-        return int(self.lib.tpqo_quantize_one(ctypes.c_uint16(int(x_bits)), ctypes.c_float(inv_s)))
+    def quantize_one(self, x_bits: int, inv_s: float, bits: int = 4) -> int:
+        if bits == 4:
+            return int(self.lib.tpqo_quantize_one(ctypes.c_uint16(int(x_bits)), ctypes.c_float(inv_s)))
+        return int(self.lib.tpqo_quantize_one_b(ctypes.c_uint16(int(x_bits)), ctypes.c_float(inv_s), bits))
 
-    def quantize_pack(self, y_bits: np.ndarray, hp_idx: np.ndarray, inv_s: np.ndarray) -> np.ndarray:
+    def quantize_pack(self, y_bits: np.ndarray, hp_idx: np.ndarray, inv_s: np.ndarray, bits: int = 4) -> np.ndarray:
         y = np.ascontiguousarray(y_bits, dtype=np.uint16)
         T, E = y.shape
         hp = np.ascontiguousarray(hp_idx, dtype=np.int32)
         k = hp.shape[0]
         inv = np.ascontiguousarray(inv_s, dtype=np.float32)
         assert inv.shape == (E,)
-        out = np.empty(self.payload_bytes(T, E, k), np.uint8)
+        out = np.empty(self.payload_bytes(T, E, k, bits), np.uint8)
         hp_arg = hp if k else np.zeros(1, np.int32)
-        self.lib.tpqo_quantize_pack(_ptr(y, ctypes.c_uint16), T, E, E, _ptr(hp_arg, ctypes.c_int32), k,
-                                    _ptr(inv, ctypes.c_float), _ptr(out, ctypes.c_uint8))
+        if bits == 4:
+            self.lib.tpqo_quantize_pack(_ptr(y, ctypes.c_uint16), T, E, E, _ptr(hp_arg, ctypes.c_int32), k,
+                                        _ptr(inv, ctypes.c_float), _ptr(out, ctypes.c_uint8))
+        else:
+            self.lib.tpqo_quantize_pack_b(_ptr(y, ctypes.c_uint16), T, E, E, _ptr(hp_arg, ctypes.c_int32), k,
+                                          _ptr(inv, ctypes.c_float), bits, _ptr(out, ctypes.c_uint8))
         return out
 
     def dequant_reduce(self, payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray,
-                       want_chain32: bool = True):
+                       want_chain32: bool = True, bits: int = 4):
         N = len(payloads)
         hp = np.ascontiguousarray(hp_idx, dtype=np.int32)
         k = hp.shape[0]
@@ -156,15 +181,20 @@ class COracle:
         assert s.shape == (N, E)
         pls = [np.ascontiguousarray(p, dtype=np.uint8) for p in payloads]
         for p in pls:
-            assert p.size == self.payload_bytes(T, E, k)
+            assert p.size == self.payload_bytes(T, E, k, bits)
         u8p = ctypes.POINTER(ctypes.c_uint8)
         arr = (u8p * N)(*[_ptr(p, ctypes.c_uint8) for p in pls])
         ref = np.empty((T, E), np.float64)
         chain = np.empty((T, E), np.float32) if want_chain32 else None
         hp_arg = hp if k else np.zeros(1, np.int32)
-        self.lib.tpqo_dequant_reduce(arr, N, T, E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(s, ctypes.c_float),
-                                     _ptr(ref, ctypes.c_double),
-                                     _ptr(chain, ctypes.c_float) if want_chain32 else None)
+        if bits == 4:
+            self.lib.tpqo_dequant_reduce(arr, N, T, E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(s, ctypes.c_float),
+                                         _ptr(ref, ctypes.c_double),
+                                         _ptr(chain, ctypes.c_float) if want_chain32 else None)
+        else:
+            self.lib.tpqo_dequant_reduce_b(arr, N, T, E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(s, ctypes.c_float),
+                                           bits, _ptr(ref, ctypes.c_double),
+                                           _ptr(chain, ctypes.c_float) if want_chain32 else None)
         return ref, chain
 
     def round_bf16(self, x: np.ndarray) -> np.ndarray:

@@ -100,9 +100,10 @@ def select(Rbar: np.ndarray, k: int) -> np.ndarray:
     return np.array(sorted(order[:k]), dtype=np.int32)
 
 
-def params(R: np.ndarray):
-    """Step s = R/15 floored at 2^-23, and the reciprocal the quantiser uses."""
-    s = (np.asarray(R, dtype=F32) / LEVELS_MINUS_ONE).astype(F32)
+def params(R: np.ndarray, bits: int = 4):
+    """Step s = R/(2^bits - 1) (R/15 for Int4) floored at 2^-23, and the reciprocal the quantiser uses."""
+    levels = LEVELS_MINUS_ONE if bits == 4 else F32((1 << bits) - 1)
+    s = (np.asarray(R, dtype=F32) / levels).astype(F32)
     s = np.where(s >= S_FLOOR, s, S_FLOOR).astype(F32)
     inv_s = (F32(1.0) / s).astype(F32)
     return s, inv_s
@@ -125,67 +126,67 @@ def lp_index(E: int, hp_idx: np.ndarray) -> np.ndarray:
     return order
 
 
-def quantize_codes(y_bits: np.ndarray, inv_s: np.ndarray) -> np.ndarray:
-    """Symmetric Int4 codes in [-8, 7]: product rounded to float32, clamped,
-    then rounded half-to-even (np.rint)."""
+def quantize_codes(y_bits: np.ndarray, inv_s: np.ndarray, bits: int = 4) -> np.ndarray:
+    """Symmetric codes in [-2^(bits-1), 2^(bits-1) - 1] ([-8, 7] for Int4): product rounded to
+    float32, clamped, then rounded half-to-even (np.rint)."""
+    q_min = Q_MIN if bits == 4 else F32(-(1 << (bits - 1)))
+    q_max = Q_MAX if bits == 4 else F32((1 << (bits - 1)) - 1)
     with np.errstate(over="ignore"):
         u = (widen(y_bits) * np.asarray(inv_s, dtype=F32)).astype(F32)
-    u = np.minimum(np.maximum(u, Q_MIN), Q_MAX)
-    return np.rint(u).astype(np.int8)
+    u = np.minimum(np.maximum(u, q_min), q_max)
+    return np.rint(u).astype(np.int16)
 
 
-def lp_bytes(T: int, E: int, k: int) -> int:
-    nib = T * (E - k)
-    return ((nib + 1) // 2 + 15) // 16 * 16
+def lp_bytes(T: int, E: int, k: int, bits: int = 4) -> int:
+    nbits = T * (E - k) * bits
+    return ((nbits + 7) // 8 + 15) // 16 * 16
 
 
-def payload_bytes(T: int, E: int, k: int) -> int:
-    return lp_bytes(T, E, k) + 2 * T * k
+def payload_bytes(T: int, E: int, k: int, bits: int = 4) -> int:
+    return lp_bytes(T, E, k, bits) + 2 * T * k
 
 
-def bits_per_value(T: int, E: int, k: int) -> float:
-    return 8.0 * payload_bytes(T, E, k) / (T * E)
+def bits_per_value(T: int, E: int, k: int, bits: int = 4) -> float:
+    return 8.0 * payload_bytes(T, E, k, bits) / (T * E)
 
 
-def quantize_pack(y_bits: np.ndarray, hp_idx: np.ndarray, inv_s: np.ndarray) -> np.ndarray:
-    """One device's [T, E] BF16 partial sums -> payload bytes."""
+def quantize_pack(y_bits: np.ndarray, hp_idx: np.ndarray, inv_s: np.ndarray, bits: int = 4) -> np.ndarray:
+    """One device's [T, E] BF16 partial sums -> payload bytes.  The codes form one little-endian bit
+    stream: bit b of code p is bit p*bits + b of the stream (for Int4: low nibble first)."""
     T, E = y_bits.shape
     k = len(hp_idx)
     lp = lp_index(E, hp_idx)
-    codes = quantize_codes(y_bits[:, lp], inv_s[lp])            # [T, E-k]
-    nib = (codes.astype(np.int16) & 0xF).astype(np.uint8).reshape(-1)
-    if nib.size % 2:
-        nib = np.concatenate([nib, np.zeros(1, np.uint8)])
-    packed = nib[0::2] | (nib[1::2] << 4)
-    out = np.zeros(payload_bytes(T, E, k), dtype=np.uint8)
+    codes = quantize_codes(y_bits[:, lp], inv_s[lp], bits).reshape(-1)          # [T (E-k)]
+    u = (codes.astype(np.int32) & ((1 << bits) - 1)).astype(np.uint32)
+    bitplanes = ((u[:, None] >> np.arange(bits, dtype=np.uint32)[None, :]) & 1).astype(np.uint8)   # [n, bits]
+    packed = np.packbits(bitplanes.reshape(-1), bitorder="little")
+    out = np.zeros(payload_bytes(T, E, k, bits), dtype=np.uint8)
     out[: packed.size] = packed
     hp = np.ascontiguousarray(y_bits[:, np.asarray(hp_idx, dtype=np.int64)])
-    out[lp_bytes(T, E, k):] = hp.view(np.uint8).reshape(-1)
+    out[lp_bytes(T, E, k, bits):] = hp.view(np.uint8).reshape(-1)
     return out
 
 
-def unpack(payload: np.ndarray, T: int, E: int, k: int):
-    """Payload -> (codes [T, E-k] int8, hp [T, k] BF16 bits)."""
+def unpack(payload: np.ndarray, T: int, E: int, k: int, bits: int = 4):
+    """Payload -> (codes [T, E-k] int16, hp [T, k] BF16 bits)."""
     L = E - k
-    nb = lp_bytes(T, E, k)
-    b = payload[:nb]
-    nib = np.empty(nb * 2, dtype=np.uint8)
-    nib[0::2] = b & 0xF
-    nib[1::2] = b >> 4
-    nib = nib[: T * L].astype(np.int8)
-    codes = np.where(nib >= 8, nib - 16, nib).astype(np.int8).reshape(T, L)
+    nb = lp_bytes(T, E, k, bits)
+    stream = np.unpackbits(np.asarray(payload[:nb], dtype=np.uint8), bitorder="little")[: T * L * bits]
+    planes = stream.reshape(T * L, bits).astype(np.int32)
+    u = (planes << np.arange(bits, dtype=np.int32)[None, :]).sum(axis=1)
+    codes = np.where(u >= (1 << (bits - 1)), u - (1 << bits), u).astype(np.int16).reshape(T, L)
     hp = payload[nb:].view(np.uint16).reshape(T, k) if k else np.zeros((T, 0), np.uint16)
     return codes, hp
 
 
 # ------------------------------------------------------------------ decompression + sum
-def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray):
+def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray, bits: int = 4):
     """Sum over devices of the dequantised payloads, in float64, original feature order."""
     k = len(hp_idx)
     lp = lp_index(E, hp_idx)
     out = np.zeros((T, E), dtype=np.float64)
     for i, p in enumerate(payloads):
-        codes, hp = unpack(np.asarray(p, dtype=np.uint8), T, E, k)
+        codes, hp = unpack(np.asarray(p, dtype=np.uint8), T, E, k, bits)
         out[:, lp] += codes.astype(np.float64) * s[i, lp].astype(np.float64)[None, :]
         if k:
             out[:, np.asarray(hp_idx, dtype=np.int64)] += widen(hp).astype(np.float64)

@@ -37,6 +37,16 @@
 #include <stdlib.h>
 #include <string.h>
 
+/* code widths other than 4 (definitions below, beside their Int4 forms) */
+void tpqo_params_b(const float *R, int64_t n, int bits, float *s, float *inv_s);
+int64_t tpqo_lp_bytes_b(int64_t T, int64_t E, int64_t k, int bits);
+int64_t tpqo_payload_bytes_b(int64_t T, int64_t E, int64_t k, int bits);
+int tpqo_quantize_one_b(uint16_t x_bf16, float inv_s, int bits);
+void tpqo_quantize_pack_b(const uint16_t *y, int64_t T, int64_t E, int64_t stride, const int32_t *hp_idx, int64_t k,
+                          const float *inv_s, int bits, uint8_t *payload);
+void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T, int64_t E, const int32_t *hp_idx,
+                           int64_t k, const float *s, int bits, double *ref64, float *chain32);
+
 #ifdef _OPENMP
 #include <omp.h>
 #endif
@@ -185,11 +195,16 @@ int64_t tpqo_default_k(int64_t E) { return E / 64; }
  * "Int4" and gives the range).  Reading: step s = R / (2^4 - 1), zero-point 0,
  * codes -8..7; a degenerate range is floored at s = 2^-23 so that 1/s is
  * finite; the quantiser multiplies by the stored reciprocal fl(1/s). */
-void tpqo_params(const float *R, int64_t n, float *s, float *inv_s)
+void tpqo_params(const float *R, int64_t n, float *s, float *inv_s) { tpqo_params_b(R, n, 4, s, inv_s); }
+
+/* The same at another code width b (Section 4 / Figure 3 evaluate the method "at lower and higher
+ * precision"): step s = R / (2^b - 1), codes -2^(b-1) .. 2^(b-1)-1. */
+void tpqo_params_b(const float *R, int64_t n, int bits, float *s, float *inv_s)
 {
     const float floor_s = 1.1920928955078125e-07f; /* 2^-23 */
+    const float levels = (float)((1 << bits) - 1);
     for (int64_t a = 0; a < n; ++a) {
-        volatile float v = R[a] / 15.0f;
+        volatile float v = R[a] / levels;
         if (!(v >= floor_s)) v = floor_s;
         s[a] = v;
         volatile float r = 1.0f / v;
@@ -227,31 +242,41 @@ void tpqo_slot_order(int64_t E, const int32_t *hp_idx, int64_t k, int32_t *slot_
     free(sel);
 }
 
-int64_t tpqo_lp_bytes(int64_t T, int64_t E, int64_t k)
+int64_t tpqo_lp_bytes(int64_t T, int64_t E, int64_t k) { return tpqo_lp_bytes_b(T, E, k, 4); }
+
+int64_t tpqo_payload_bytes(int64_t T, int64_t E, int64_t k) { return tpqo_payload_bytes_b(T, E, k, 4); }
+
+/* Width b: T(E-k) codes of b bits each, one flat little-endian bit stream (code p occupies bits
+ * [p b, p b + b) of the stream, bit 0 = least significant bit of byte 0), padded to 16 bytes. */
+int64_t tpqo_lp_bytes_b(int64_t T, int64_t E, int64_t k, int bits)
 {
-    int64_t nib = T * (E - k);
-    int64_t bytes = (nib + 1) / 2;
+    int64_t nbits = T * (E - k) * bits;
+    int64_t bytes = (nbits + 7) / 8;
     return (bytes + 15) / 16 * 16;
 }
 
-int64_t tpqo_payload_bytes(int64_t T, int64_t E, int64_t k)
+int64_t tpqo_payload_bytes_b(int64_t T, int64_t E, int64_t k, int bits)
 {
-    return tpqo_lp_bytes(T, E, k) + 2 * T * k;
+    return tpqo_lp_bytes_b(T, E, k, bits) + 2 * T * k;
 }
 
 /* ------------------------------------------------------- compression C^(i) */
 
 /* One symmetric Int4 code: u = fl(x * inv_s); clamp to [-8, 7]; round half to
  * even.  Two roundings (the product, then the integer), never a fused one. */
-int tpqo_quantize_one(uint16_t x_bf16, float inv_s)
+int tpqo_quantize_one(uint16_t x_bf16, float inv_s) { return tpqo_quantize_one_b(x_bf16, inv_s, 4); }
+
+/* Width b: clamp to [-2^(b-1), 2^(b-1) - 1]. */
+int tpqo_quantize_one_b(uint16_t x_bf16, float inv_s, int bits)
 {
+    const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
     volatile float u = bf16_widen(x_bf16) * inv_s;
     float v = u;
-    if (v < -8.0f) v = -8.0f;
-    if (v > 7.0f) v = 7.0f;
+    if (v < lo) v = lo;
+    if (v > hi) v = hi;
     /* round half to even without relying on the floating-point environment */
     float fl = floorf(v);
-    float d = v - fl;                 /* exact for |v| <= 8 */
+    float d = v - fl;                 /* exact for |v| <= 128 */
     int q = (int)fl;
     if (d > 0.5f || (d == 0.5f && (q & 1))) q += 1;
     return q;
@@ -264,15 +289,23 @@ void tpqo_quantize_pack(const uint16_t *y, int64_t T, int64_t E, int64_t stride,
                         const int32_t *hp_idx, int64_t k, const float *inv_s,
                         uint8_t *payload)
 {
+    tpqo_quantize_pack_b(y, T, E, stride, hp_idx, k, inv_s, 4, payload);
+}
+
+void tpqo_quantize_pack_b(const uint16_t *y, int64_t T, int64_t E, int64_t stride,
+                          const int32_t *hp_idx, int64_t k, const float *inv_s, int bits,
+                          uint8_t *payload)
+{
     int64_t L = E - k;
-    int64_t lp_bytes = tpqo_lp_bytes(T, E, k);
+    int64_t lp_bytes = tpqo_lp_bytes_b(T, E, k, bits);
+    const unsigned cmask = (1u << bits) - 1u;
     int32_t *lp_idx = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L > 0 ? L : 1));
     tpqo_slot_order(E, hp_idx, k, lp_idx);      /* lp_idx[c] = feature held by slot c */
     memset(payload, 0, (size_t)lp_bytes);
     uint16_t *hp = (uint16_t *)(payload + lp_bytes);
-    /* rows are independent; codes of two rows can share a byte only when L is
-     * odd, so rows are paired up for the threads in that case. */
-    int64_t rows_per_chunk = (L % 2) ? 2 : 1;
+    /* rows are independent; 8 rows of codes always end on a byte boundary, so
+     * the threads take 8 rows at a time and never share a byte. */
+    int64_t rows_per_chunk = 8;
     int64_t n_chunks = (T + rows_per_chunk - 1) / rows_per_chunk;
 #pragma omp parallel for schedule(static)
     for (int64_t ch = 0; ch < n_chunks; ++ch) {
@@ -281,11 +314,11 @@ void tpqo_quantize_pack(const uint16_t *y, int64_t T, int64_t E, int64_t stride,
         for (int64_t t = t0; t < t1; ++t) {
             for (int64_t c = 0; c < L; ++c) {
                 int64_t j = lp_idx[c];
-                int q = tpqo_quantize_one(y[t * stride + j], inv_s[j]);
-                int64_t p = t * L + c;
-                uint8_t nib = (uint8_t)(q & 0xF);
-                if (p & 1) payload[p >> 1] |= (uint8_t)(nib << 4);
-                else       payload[p >> 1] |= nib;
+                int q = tpqo_quantize_one_b(y[t * stride + j], inv_s[j], bits);
+                int64_t bit = (t * L + c) * bits;          /* first bit of the code in the stream */
+                unsigned u = ((unsigned)q & cmask) << (bit & 7);   /* at most 15 bits: spans <= 2 bytes */
+                payload[bit >> 3] |= (uint8_t)(u & 0xFFu);
+                if (u >> 8) payload[(bit >> 3) + 1] |= (uint8_t)(u >> 8);
             }
             for (int64_t h = 0; h < k; ++h)
                 hp[t * k + h] = y[t * stride + hp_idx[h]];
@@ -306,8 +339,16 @@ void tpqo_dequant_reduce(const uint8_t *const *payloads, int64_t N, int64_t T,
                          int64_t E, const int32_t *hp_idx, int64_t k,
                          const float *s, double *ref64, float *chain32)
 {
+    tpqo_dequant_reduce_b(payloads, N, T, E, hp_idx, k, s, 4, ref64, chain32);
+}
+
+void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T,
+                           int64_t E, const int32_t *hp_idx, int64_t k,
+                           const float *s, int bits, double *ref64, float *chain32)
+{
     int64_t L = E - k;
-    int64_t lp_bytes = tpqo_lp_bytes(T, E, k);
+    int64_t lp_bytes = tpqo_lp_bytes_b(T, E, k, bits);
+    const unsigned cmask = (1u << bits) - 1u, sign = 1u << (bits - 1);
     int32_t *pos = (int32_t *)malloc(sizeof(int32_t) * (size_t)E); /* >=0: code slot c; <0: -(h+1) */
     {
         int32_t *slot_feature = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L > 0 ? L : 1));
@@ -324,9 +365,11 @@ void tpqo_dequant_reduce(const uint8_t *const *payloads, int64_t N, int64_t T,
             for (int64_t i = 0; i < N; ++i) {
                 const uint8_t *pl = payloads[i];
                 if (pos[j] >= 0) {
-                    int64_t p = t * L + pos[j];
-                    int nib = (p & 1) ? (pl[p >> 1] >> 4) : (pl[p >> 1] & 0xF);
-                    int q = (nib >= 8) ? nib - 16 : nib;
+                    int64_t bit = (t * L + pos[j]) * bits;
+                    unsigned w = pl[bit >> 3];
+                    if ((bit & 7) + bits > 8) w |= (unsigned)pl[(bit >> 3) + 1] << 8;
+                    unsigned u = (w >> (bit & 7)) & cmask;
+                    int q = (u & sign) ? (int)u - (int)(cmask + 1u) : (int)u;   /* two's complement, b bits */
                     float si = s[i * E + j];
                     acc64 += (double)q * (double)si;
                     acc32 = fmaf((float)q, si, acc32);
