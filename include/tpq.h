@@ -67,16 +67,20 @@ typedef struct tpq_comm_report {
     int64_t quantized_allgather_send;  /* (N-1) * P, unicast all-gather of payloads (the method)        */
     int64_t bf16_allgather_send;       /* (N-1) * 2*T*E, all-gather of the raw BF16 partial sums         */
     int64_t bf16_ring_allreduce_send;  /* 2*(N-1)/N * 2*T*E, bandwidth-optimal BF16 all-reduce           */
-    double bits_per_value;             /* 8*P / (T*E); equals 4 + 12k/E up to the 16-byte pad (Sec. 4)   */
-    double bits_per_value_formula;     /* 4 + 12k/E                                                      */
+    double bits_per_value;             /* 8*P / (T*E); equals b + (16-b)k/E up to the 16-byte pad (Sec. 4) */
+    double bits_per_value_formula;     /* b + (16-b)k/E for b-bit codes: 4 + 12k/E for the paper's Int4   */
 } tpq_comm_report;
 
 /* ---------------------------------------------------------------- context */
 
 /* Create a context for n_shards (N >= 1) devices and n_features (E >= 1)
- * features on the current CUDA device.  bits must be 4 (the paper's Int4,
- * Section 3); gamma is the moving-average constant of Eq. (1)-(2) (the paper
- * uses 0.01), 0 <= gamma <= 1.  Errors: INVALID_ARG, NOMEM, CUDA. */
+ * features on the current CUDA device.  bits is the code width: 4 is the
+ * paper's Int4 (Section 3) and the width the tiled kernels serve; 2..8 are
+ * accepted (the method "at lower and higher precision", Section 4 / Figure 3:
+ * step R/(2^bits - 1), codes -2^(bits-1) .. 2^(bits-1)-1, one little-endian
+ * stream of bits-wide codes) and run on the shape-generic kernels.  gamma is
+ * the moving-average constant of Eq. (1)-(2) (the paper uses 0.01),
+ * 0 <= gamma <= 1.  Errors: INVALID_ARG, NOMEM, CUDA. */
 tpq_status tpq_create(tpq_ctx **ctx, int n_shards, int n_features, int bits, float gamma);
 tpq_status tpq_destroy(tpq_ctx *ctx); /* NULL is accepted */
 tpq_status tpq_set_option(tpq_ctx *ctx, tpq_option opt, int value);
@@ -162,8 +166,10 @@ tpq_status tpq_get_features(tpq_ctx *ctx, int32_t *hp_idx_out_host);
  * ascending.  No header; the static steps are never transmitted.
  * Returns 0 before a feature set exists or for T <= 0. */
 size_t tpq_payload_bytes(const tpq_ctx *ctx, int64_t T);
-/* The same closed form without a context. */
+/* The same closed form without a context (Int4), and for a code width of
+ * 2..8 bits: roundup16(ceil(T*(E-k)*bits / 8)) + 2*T*k. */
 size_t tpq_payload_bytes_for(int64_t T, int64_t E, int64_t k);
+size_t tpq_payload_bytes_for_bits(int64_t T, int64_t E, int64_t k, int bits);
 
 /* Section 5 / Section 4: bytes per synchronisation and bits per value. */
 tpq_status tpq_comm_bytes(const tpq_ctx *ctx, int64_t T, tpq_comm_report *out);

@@ -45,6 +45,7 @@ SIGNATURES = {
     "tpq_get_features": (c_int, [c_void_p, POINTER(c_int32)]),
     "tpq_payload_bytes": (c_size_t, [c_void_p, c_int64]),
     "tpq_payload_bytes_for": (c_size_t, [c_int64, c_int64, c_int64]),
+    "tpq_payload_bytes_for_bits": (c_size_t, [c_int64, c_int64, c_int64, c_int]),
     "tpq_comm_bytes": (c_int, [c_void_p, c_int64, POINTER(CommReport)]),
     "tpq_quantize_pack": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, c_void_p, c_size_t, c_void_p]),
     "tpq_quantize_pack_batch": (c_int, [c_void_p, c_int, c_int, POINTER(c_void_p), c_int64, c_int64, POINTER(c_void_p),
@@ -97,7 +98,7 @@ class Tpq:
         if st != TPQ_OK:
             self._h = c_void_p()
             raise TpqError(st, "tpq_create failed")
-        self.N, self.E = n_shards, n_features
+        self.N, self.E, self.bits = n_shards, n_features, bits
 
     def close(self):
         if getattr(self, "_h", None) and self._h.value:
@@ -222,5 +223,7 @@ class Tpq:
         return int(lib().tpq_launch_count(self._h))
 
 
-def payload_bytes_for(T: int, E: int, k: int) -> int:
-    return int(lib().tpq_payload_bytes_for(T, E, k))
+def payload_bytes_for(T: int, E: int, k: int, bits: int = 4) -> int:
+    if bits == 4:
+        return int(lib().tpq_payload_bytes_for(T, E, k))
+    return int(lib().tpq_payload_bytes_for_bits(T, E, k, bits))

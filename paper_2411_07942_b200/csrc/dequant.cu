@@ -15,7 +15,7 @@ namespace {
 
 struct DQParams {
     const uint8_t *pl[TPQ_MAX_SHARDS];  // payloads, device order
-    int N, E, k;
+    int N, E, k, bits;
     int64_t T;
     int64_t lp_bytes;      // code section size (HP block starts here)
     const float *s_k;      // [N][E], 0 at selected features
@@ -26,7 +26,7 @@ struct DQParams {
 };
 
 // ----------------------------------------------------------------------------------------------
-// Shape-generic kernel: one thread per output element.
+// Shape-generic kernel: one thread per output element; any code width of 2..8 bits.
 // ----------------------------------------------------------------------------------------------
 template <bool FP32OUT>
 __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
@@ -39,11 +39,15 @@ __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
         const int ps = p.pos[j];
         float acc = 0.0f;
         if (ps >= 0) {
-            const int64_t q = t * L + ps;
+            const int64_t bit = (t * L + ps) * p.bits;  // first bit of the code in the little-endian stream
+            const int sh = (int)(bit & 7);
+            const bool two = sh + p.bits > 8;
+            const uint32_t cmask = (1u << p.bits) - 1u, sign = 1u << (p.bits - 1);
             for (int i = 0; i < p.N; ++i) {
-                const uint32_t b = p.pl[i][q >> 1];
-                const int nib = (q & 1) ? (b >> 4) : (b & 0xF);
-                const int code = (nib ^ 8) - 8;
+                uint32_t b = p.pl[i][bit >> 3];
+                if (two) b |= (uint32_t)p.pl[i][(bit >> 3) + 1] << 8;
+                const uint32_t u = (b >> sh) & cmask;
+                const int code = (int)(u ^ sign) - (int)sign;  // two's complement, `bits` wide
                 acc = __fmaf_rn((float)code, p.s_k[(size_t)i * p.E + j], acc);
             }
         } else {
@@ -1010,8 +1014,8 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
 void fill_params(DQParams &p, const tpq_ctx *c, const void *const *payloads, int64_t T, void *out, int64_t out_stride)
 {
     for (int i = 0; i < c->N; ++i) p.pl[i] = static_cast<const uint8_t *>(payloads[i]);
-    p.N = c->N; p.E = c->E; p.k = c->k; p.T = T;
-    p.lp_bytes = tpq_lp_bytes_i(T, c->E, c->k);
+    p.N = c->N; p.E = c->E; p.k = c->k; p.bits = c->bits; p.T = T;
+    p.lp_bytes = tpq_lp_bytes_i(T, c->E, c->k, c->bits);
     p.s_k = c->t.s_k; p.pos = c->t.pos; p.grp = c->t.grp;
     p.out = out; p.out_stride = out_stride;
 }
@@ -1021,6 +1025,7 @@ void fill_params(DQParams &p, const tpq_ctx *c, const void *const *payloads, int
 bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int fp32_out)
 {
     (void)fp32_out;
+    if (c->bits != 4) return false;  // the tiled kernels are Int4 kernels
     if (c->E % 8 || c->k % 8 || out_stride % 8 || T <= 0) return false;
     if (c->E - c->k < 8) return false;
     return true;

@@ -8,38 +8,43 @@
 namespace {
 
 // ----------------------------------------------------------------------------------------------
-// Shape-generic kernel: one thread per 32-bit word of the code stream (8 codes), any E, k, stride.
+// Shape-generic kernel: one thread per 32-bit word of the code stream, any E, k, stride and any code
+// width of 2..8 bits (a code that straddles two words is quantised by both words' threads).
 // ----------------------------------------------------------------------------------------------
-__device__ __forceinline__ int quant_one(uint16_t x, float inv_s)
+__device__ __forceinline__ int quant_one(uint16_t x, float inv_s, float lo, float hi)
 {
     float u = __fmul_rn(__uint_as_float((uint32_t)x << 16), inv_s);
-    u = fminf(fmaxf(u, -8.0f), 7.0f);
+    u = fminf(fmaxf(u, lo), hi);
     return __float2int_rn(u);
 }
 
 __global__ void __launch_bounds__(256) quantize_generic(const uint16_t *__restrict__ y, int64_t T, int64_t stride, int E,
-                                                        int k, const float *__restrict__ inv_s,
+                                                        int k, int bits, const float *__restrict__ inv_s,
                                                         const int32_t *__restrict__ lp_idx,
                                                         const int32_t *__restrict__ hp_idx,
                                                         uint32_t *__restrict__ lp_out, int64_t lp_words,
                                                         uint16_t *__restrict__ hp_out)
 {
     const int64_t L = E - k;
-    const int64_t n_nib = T * L;
+    const int64_t n_codes = T * L;
     const int64_t hp_elems = T * k;
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t gsz = (int64_t)gridDim.x * blockDim.x;
+    const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+    const uint32_t cmask = (1u << bits) - 1u;
     for (int64_t w = gid; w < lp_words; w += gsz) {
         uint32_t word = 0;
-        int64_t p = 8 * w;
-        if (p < n_nib) {
+        const int64_t bit0 = 32 * w;           // the word holds bits [bit0, bit0 + 32) of the stream
+        int64_t p = bit0 / bits;               // first code with a bit in the word
+        if (p < n_codes) {
             int64_t t = p / L;
             int64_t c = p - t * L;
 #pragma unroll 1
-            for (int n = 0; n < 8 && p < n_nib; ++n, ++p) {
+            for (; p < n_codes && p * bits < bit0 + 32; ++p) {
                 const int j = lp_idx[c];
-                const int q = quant_one(y[t * stride + j], inv_s[j]);
-                word |= (uint32_t)(q & 0xF) << (4 * n);
+                const uint32_t u = (uint32_t)quant_one(y[t * stride + j], inv_s[j], lo, hi) & cmask;
+                const int o = (int)(p * bits - bit0);   // may be negative: the code starts in the previous word
+                word |= (o >= 0) ? (u << o) : (u >> -o);
                 if (++c == L) {
                     c = 0;
                     ++t;
@@ -431,6 +436,7 @@ size_t qp_smem_bytes(int E, int G, int nstage) { return qp_layout(E, G, nstage).
 
 bool tpq_quantize_tiled_ok(const tpq_ctx *c, int64_t T, int64_t stride)
 {
+    if (c->bits != 4) return false;  // the tiled kernels are Int4 kernels
     const int E = c->E, k = c->k;
     if (E % 8 || k % 8 || stride % 8 || T <= 0) return false;
     if (E - k < 8) return false;
@@ -443,13 +449,13 @@ cudaError_t tpq_launch_quantize_generic(const tpq_ctx *c, int shard, const uint1
                                         uint8_t *payload, cudaStream_t st, int64_t *launches)
 {
     const int E = c->E, k = c->k;
-    const int64_t lpb = tpq_lp_bytes_i(T, E, k);
+    const int64_t lpb = tpq_lp_bytes_i(T, E, k, c->bits);
     const int64_t lp_words = lpb / 4;
     int64_t work = lp_words > T * k ? lp_words : T * (int64_t)k;
     int64_t blocks = (work + 255) / 256;
     if (blocks > 148LL * 32) blocks = 148LL * 32;
     if (blocks < 1) blocks = 1;
-    quantize_generic<<<(unsigned)blocks, 256, 0, st>>>(y, T, stride, E, k, c->t.inv_s + (size_t)shard * E, c->t.lp_idx,
+    quantize_generic<<<(unsigned)blocks, 256, 0, st>>>(y, T, stride, E, k, c->bits, c->t.inv_s + (size_t)shard * E, c->t.lp_idx,
                                                        c->t.hp_idx, reinterpret_cast<uint32_t *>(payload), lp_words,
                                                        reinterpret_cast<uint16_t *>(payload + lpb));
     ++*launches;

@@ -5,10 +5,11 @@
 namespace {
 
 // R^(i)_j = 2 max(-m, M); Rbar_j = sum_i R^(i)_j (binary32, devices ascending);
-// step s = R/15 floored at 2^-23 and its reciprocal (IEEE division, no fast-math).
+// step s = R/(2^bits - 1) (R/15 for Int4) floored at 2^-23 and its reciprocal (IEEE division, no fast-math).
 __global__ void __launch_bounds__(256) ranges_kernel(const float *__restrict__ m, const float *__restrict__ M, int N,
-                                                     int E, float *__restrict__ R, float *__restrict__ Rbar,
-                                                     float *__restrict__ s, float *__restrict__ inv_s)
+                                                     int E, float levels, float *__restrict__ R,
+                                                     float *__restrict__ Rbar, float *__restrict__ s,
+                                                     float *__restrict__ inv_s)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= E) return;
@@ -20,7 +21,7 @@ __global__ void __launch_bounds__(256) ranges_kernel(const float *__restrict__ m
         const float r = __fmul_rn(2.0f, A);
         R[o] = r;
         acc = (i == 0) ? r : __fadd_rn(acc, r);
-        float sv = __fdiv_rn(r, 15.0f);
+        float sv = __fdiv_rn(r, levels);
         if (!(sv >= 1.1920928955078125e-07f)) sv = 1.1920928955078125e-07f;
         s[o] = sv;
         inv_s[o] = __fdiv_rn(1.0f, sv);
@@ -122,9 +123,9 @@ __global__ void __launch_bounds__(1024) tables_kernel(tpq_tables t, int N, int E
 
 }  // namespace
 
-cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches)
+cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, int bits, cudaStream_t st, int64_t *launches)
 {
-    ranges_kernel<<<(E + 255) / 256, 256, 0, st>>>(t.m, t.M, N, E, t.R, t.Rbar, t.s, t.inv_s);
+    ranges_kernel<<<(E + 255) / 256, 256, 0, st>>>(t.m, t.M, N, E, (float)((1 << bits) - 1), t.R, t.Rbar, t.s, t.inv_s);
     ++*launches;
     return cudaGetLastError();
 }

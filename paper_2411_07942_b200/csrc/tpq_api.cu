@@ -60,7 +60,7 @@ bool all_calibrated(const tpq_ctx *c)
 // ranges -> (flags already on the device) -> tables; synchronises
 tpq_status build_tables(tpq_ctx *c, int k, bool topk)
 {
-    cudaError_t e = tpq_launch_ranges(c->t, c->N, c->E, 0, &c->launches);
+    cudaError_t e = tpq_launch_ranges(c->t, c->N, c->E, c->bits, 0, &c->launches);
     if (e != cudaSuccess) return cuda_fail(c, e, "ranges kernel");
     if (topk) {
         e = tpq_launch_topk_flags(c->t, c->E, k, 0, &c->launches);
@@ -111,7 +111,7 @@ tpq_status tpq_create(tpq_ctx **out, int n_shards, int n_features, int bits, flo
     if (!out) return TPQ_ERR_INVALID_ARG;
     *out = nullptr;
     if (n_shards < 1 || n_shards > TPQ_MAX_SHARDS || n_features < 1 || n_features > (1 << 22)) return TPQ_ERR_INVALID_ARG;
-    if (bits != 4) return TPQ_ERR_INVALID_ARG;
+    if (bits < 2 || bits > 8) return TPQ_ERR_INVALID_ARG;
     if (!(gamma >= 0.0f && gamma <= 1.0f)) return TPQ_ERR_INVALID_ARG;
     tpq_ctx *c = new (std::nothrow) tpq_ctx();
     if (!c) return TPQ_ERR_NOMEM;
@@ -326,10 +326,16 @@ size_t tpq_payload_bytes_for(int64_t T, int64_t E, int64_t k)
     return (size_t)(tpq_lp_bytes_i(T, E, k) + 2 * T * k);
 }
 
+size_t tpq_payload_bytes_for_bits(int64_t T, int64_t E, int64_t k, int bits)
+{
+    if (T <= 0 || E <= 0 || k < 0 || k > E || bits < 2 || bits > 8) return 0;
+    return (size_t)(tpq_lp_bytes_i(T, E, k, bits) + 2 * T * k);
+}
+
 size_t tpq_payload_bytes(const tpq_ctx *c, int64_t T)
 {
     if (!c || c->k < 0) return 0;
-    return tpq_payload_bytes_for(T, c->E, c->k);
+    return tpq_payload_bytes_for_bits(T, c->E, c->k, c->bits);
 }
 
 tpq_status tpq_comm_bytes(const tpq_ctx *c, int64_t T, tpq_comm_report *out)
@@ -343,7 +349,7 @@ tpq_status tpq_comm_bytes(const tpq_ctx *c, int64_t T, tpq_comm_report *out)
     out->bf16_allgather_send = (c->N - 1) * raw;
     out->bf16_ring_allreduce_send = 2 * (int64_t)(c->N - 1) * raw / c->N;
     out->bits_per_value = 8.0 * (double)P / ((double)T * c->E);
-    out->bits_per_value_formula = 4.0 + 12.0 * c->k / c->E;
+    out->bits_per_value_formula = c->bits + (16.0 - c->bits) * c->k / c->E;
     return TPQ_OK;
 }
 

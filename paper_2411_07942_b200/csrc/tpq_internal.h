@@ -51,10 +51,10 @@ struct tpq_ctx {
 // adjacent features is one aligned 32-bit word of the code stream.
 //
 // Payload geometry (Section 4 bit count; layout documented in tpq.h).
-static inline int64_t tpq_lp_bytes_i(int64_t T, int64_t E, int64_t k)
+static inline int64_t tpq_lp_bytes_i(int64_t T, int64_t E, int64_t k, int bits = 4)
 {
-    int64_t nib = T * (E - k);
-    int64_t b = (nib + 1) / 2;
+    int64_t nbits = T * (E - k) * bits;  // one flat little-endian bit stream of `bits`-bit codes
+    int64_t b = (nbits + 7) / 8;
     return (b + 15) / 16 * 16;
 }
 
@@ -72,7 +72,7 @@ cudaError_t tpq_static_scratch_address(int device, void **ptr_out);
 int tpq_static_scratch_splits(int64_t n_seq, int64_t S, int E, int sm_count);
 
 // Section 3: ranges, aggregate, steps; top-k flags (or flags given); index tables.
-cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_ranges(const tpq_tables &t, int N, int E, int bits, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_topk_flags(const tpq_tables &t, int E, int k, cudaStream_t st, int64_t *launches);
 cudaError_t tpq_launch_tables(const tpq_tables &t, int N, int E, int k, cudaStream_t st, int64_t *launches);
 

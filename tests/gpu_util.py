@@ -61,13 +61,13 @@ def bits_equal(a: np.ndarray, b: np.ndarray) -> bool:
     return a.shape == b.shape and bool(np.array_equal(a, b))
 
 
-def term_abs_sum(payloads, T, E, hp, s):
+def term_abs_sum(payloads, T, E, hp, s, bits=4):
     """sum_i |term_i| per output element (for the cancellation clause of the tolerance)."""
     k = len(hp)
     lp = oracle_np.lp_index(E, hp)
     out = np.zeros((T, E))
     for i, p in enumerate(payloads):
-        codes, hpv = oracle_np.unpack(np.asarray(p), T, E, k)
+        codes, hpv = oracle_np.unpack(np.asarray(p), T, E, k, bits)
         out[:, lp] += np.abs(codes.astype(np.float64)) * s[i, lp].astype(np.float64)[None, :]
         if k:
             out[:, np.asarray(hp, dtype=np.int64)] += np.abs(oracle_np.widen(hpv).astype(np.float64))
@@ -101,7 +101,7 @@ def run_sync(t: binding.Tpq, ys, k_expect=None, path=binding.PATH_AUTO, stride_p
     """Quantise every shard, dequantise+reduce to both output types, compare with the oracle.
     The context must already hold a feature set.  Returns the payloads (host)."""
     orc = oracle.c()
-    N, E = t.N, t.E
+    N, E, bits = t.N, t.E, t.bits
     T = ys[0].shape[0]
     hp = t.get_features()
     k = len(hp)
@@ -110,7 +110,7 @@ def run_sync(t: binding.Tpq, ys, k_expect=None, path=binding.PATH_AUTO, stride_p
     s, inv = t.get_scales()
     t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
     P = t.payload_bytes(T)
-    assert P == orc.payload_bytes(T, E, k)
+    assert P == orc.payload_bytes(T, E, k, bits)
     payload_bufs, payload_host = [], []
     for i in range(N):
         if stride_pad:
@@ -128,15 +128,15 @@ def run_sync(t: binding.Tpq, ys, k_expect=None, path=binding.PATH_AUTO, stride_p
         assert t.device_status() == 0
         assert guards_intact(whole, P), "quantize_pack wrote outside the payload"
         got = view.cpu().numpy()
-        want = orc.quantize_pack(ys[i], hp, inv[i])
+        want = orc.quantize_pack(ys[i], hp, inv[i], bits)
         if not np.array_equal(got, want):
             bad = np.nonzero(got != want)[0]
             raise AssertionError(f"payload of shard {i} differs at {bad.size} bytes, first {bad[:8]} "
-                                 f"(lp bytes {orc.lp_bytes(T, E, k)}, total {P})")
+                                 f"(lp bytes {orc.lp_bytes(T, E, k, bits)}, total {P})")
         payload_bufs.append((whole, view))
         payload_host.append(want)
-    ref, chain = orc.dequant_reduce(payload_host, T, E, hp, s)
-    abs_sum = term_abs_sum(payload_host, T, E, hp, s)
+    ref, chain = orc.dequant_reduce(payload_host, T, E, hp, s, bits=bits)
+    abs_sum = term_abs_sum(payload_host, T, E, hp, s, bits)
     ptrs = [v.data_ptr() for _, v in payload_bufs]
     # FP32 output
     whole, view = guarded(T * E * 4)

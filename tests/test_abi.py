@@ -66,7 +66,7 @@ def test_create_validates_before_touching_cuda(lib):
     import ctypes
 
     h = ctypes.c_void_p()
-    for args in [(0, 8, 4, 0.01), (2, 0, 4, 0.01), (2, 8, 8, 0.01), (2, 8, 4, -0.5), (2, 8, 4, 1.5), (65, 8, 4, 0.01)]:
+    for args in [(0, 8, 4, 0.01), (2, 0, 4, 0.01), (2, 8, 9, 0.01), (2, 8, 1, 0.01), (2, 8, 4, -0.5), (2, 8, 4, 1.5), (65, 8, 4, 0.01)]:
         assert lib.tpq_create(ctypes.byref(h), *args) == 1
         assert not h.value
     assert lib.tpq_create(None, 2, 8, 4, 0.01) == 1

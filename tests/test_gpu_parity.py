@@ -23,9 +23,9 @@ def _workload(N, T, E, seed, n_out=3, calib=(3, 8)):
     return synth.Workload("t", N, T, E, 0.6, n_out, 20.0, 200.0, calib[0], calib[1], seed)
 
 
-def _full_pipeline(w, k, path, stride_pad=0, chunks=None):
+def _full_pipeline(w, k, path, stride_pad=0, chunks=None, bits=4):
     orc = oracle.c()
-    t = binding.Tpq(w.n_shards, w.features)
+    t = binding.Tpq(w.n_shards, w.features, bits=bits)
     scale = synth.column_scales(w)
     cal = [synth.calibration_np(w, i, scale=scale) for i in range(w.n_shards)]
     m, M = gu.calibrate_both(t, cal, chunks=chunks)
@@ -37,7 +37,7 @@ def _full_pipeline(w, k, path, stride_pad=0, chunks=None):
     assert hp.tolist() == orc.select(Rbar, kk).tolist()
     _, _, gR, gRbar = t.get_ranges()
     assert gu.bits_equal(gR, R) and gu.bits_equal(gRbar, Rbar)
-    s, inv = orc.params(R)
+    s, inv = orc.params(R, bits)
     gs, ginv = t.get_scales()
     assert gu.bits_equal(gs, s) and gu.bits_equal(ginv, inv)
     ys = [synth.activations_np(w, i, w.tokens, scale=scale) for i in range(w.n_shards)]
@@ -56,6 +56,19 @@ def test_tiny_config_end_to_end():
                                      (4, 9, 24, 0), (2, 1, 8, 3), (5, 33, 100, -1)])
 def test_generic_path_odd_shapes(N, T, E, k):
     _full_pipeline(_workload(N, T, E, 100 + E + T), k, binding.PATH_AUTO)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 5, 6, 7, 8])
+@pytest.mark.parametrize("N,T,E,k", [(2, 16, 256, 4), (3, 17, 130, 2), (2, 5, 253, 9), (4, 67, 512, 8), (2, 3, 64, 0),
+                                     (8, 33, 1024, 16)])
+def test_other_code_widths(bits, N, T, E, k):
+    """The method at lower and higher precision (Section 4 / Figure 3): b-bit codes, step R/(2^b - 1),
+    payloads bit-exact against the oracle (codes straddle bytes and words for b = 3, 5, 6, 7), sums in
+    tolerance, bits per value b + (16-b)k/E up to the pad."""
+    _full_pipeline(_workload(N, T, E, 19 * E + T + bits), k, binding.PATH_AUTO, bits=bits)
+    t = binding.Tpq(N, E, bits=bits)
+    assert binding.payload_bytes_for(T, E, k, bits) == oracle.c().payload_bytes(T, E, k, bits)
+    t.close()
 
 
 @pytest.mark.parametrize("N,T,E,k,pad", [(2, 67, 512, 8, 0), (4, 301, 1024, 16, 0), (4, 37, 5120, 80, 64),

@@ -13,7 +13,7 @@ from util import bf16_bits as f32_to_bf16_bits, bf16_value
 def bf16_bits_to_f32(bits):
     return bf16_value(bits).astype(np.float32)
 
-WIDTHS = [2, 3, 5, 6, 8]
+WIDTHS = [2, 3, 5, 6, 7, 8]
 
 
 @pytest.mark.parametrize("bits", WIDTHS + [4])
