@@ -60,14 +60,14 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def payload_bytes(T, E, k):
-    nib = T * (E - k)
-    return ((nib + 1) // 2 + 15) // 16 * 16 + 2 * T * k
+def payload_bytes(T, E, k, bits=4):
+    nbits = T * (E - k) * bits
+    return ((nbits + 7) // 8 + 15) // 16 * 16 + 2 * T * k
 
 
-def algorithmic_bytes(N, T, E, k):
+def algorithmic_bytes(N, T, E, k, bits=4):
     """Bytes the method itself must move per launch (tables are O(N*E) and cache resident)."""
-    P = payload_bytes(T, E, k)
+    P = payload_bytes(T, E, k, bits)
     return {"quantize_pack": 2 * T * E + P, "dequant_reduce": N * P + 2 * T * E}
 
 
@@ -194,6 +194,8 @@ def main():
                     help="synthetic workload (default: the configuration the metric is quoted on; the others are "
                          "for profiling captures, e.g. `--workload large --tokens 1024 --sets 2`)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count")
+    ap.add_argument("--bits", type=int, default=4, help="code width (4 = the paper's Int4 and the bench's metric; "
+                                                        "2..8 run on the shape-generic kernels)")
     args = ap.parse_args()
     rank, local_rank, world = dist_env()
     if args.warmup < 3:
@@ -242,7 +244,7 @@ def main():
     sh = stream.cuda_stream
 
     # ---- static parameters: calibration (timed separately) + selection
-    t = binding.Tpq(N, E)
+    t = binding.Tpq(N, E, bits=args.bits)
     cal_seqs, cal_S = 8, w.calib_tokens
     cal_bufs = [synth.activations_torch(w, i, cal_seqs * cal_S, dev, stream=1, scale=scale) for i in range(N)]
     for i in range(N):
@@ -271,7 +273,7 @@ def main():
     del cal_bufs
     P = t.payload_bytes(T)
     comm = t.comm_bytes(T)
-    alg = algorithmic_bytes(N, T, E, k)
+    alg = algorithmic_bytes(N, T, E, k, args.bits)
 
     # ---- rotating buffer sets (inputs resident in HBM; working set > L2)
     sets = []
@@ -423,7 +425,10 @@ def main():
     else:
         dom, dom_ms, dom_bytes = "dequant_reduce", d_ms, alg["dequant_reduce"]
         traffic = NCU_TRAFFIC_BYTES["dequant_rows"]
-    if args.workload != WORKLOAD or args.tokens:
+    if args.bits != 4:
+        config["workload"] += f", {args.bits}-bit codes"
+        config["bits"] = args.bits
+    if args.workload != WORKLOAD or args.tokens or args.bits != 4:
         traffic = None  # the captured DRAM traffic is for the default workload's launches
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
