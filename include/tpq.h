@@ -55,9 +55,16 @@ typedef enum { TPQ_OUT_BF16 = 0, TPQ_OUT_FP32 = 1 } tpq_out_dtype;
 
 /* Options for tpq_set_option. */
 typedef enum {
-    TPQ_OPT_KERNEL_PATH = 0 /* 0 = automatic (default); 1 = always the shape-generic kernels;
-                               2 = the tiled kernels, TPQ_ERR_INVALID_ARG from the call if the
-                               shape does not admit them (E, k and strides multiples of 8) */
+    /* 0 = automatic (default); 1 = always the shape-generic kernels; 2 = the tiled kernels,
+     * TPQ_ERR_INVALID_ARG from the call if the shape does not admit them (E, k and strides
+     * multiples of 8, 4-bit codes). */
+    TPQ_OPT_KERNEL_PATH = 0,
+    /* Which tiled kernel tpq_dequant_reduce uses when the tiled path is taken: 0 = chosen from the
+     * shape (default); 1 = row kernel (needs N <= 4 and (E-k)/8 <= 768); 2 = tensor-map panel kernel
+     * (needs N <= 16 and E-k a multiple of 32); 3 = copy-ring panel kernel.  A kernel that the shape
+     * does not admit makes the call return TPQ_ERR_INVALID_ARG.  For tests and measurements: all
+     * kernels give identical results. */
+    TPQ_OPT_DEQUANT_KERNEL = 1
 } tpq_option;
 
 /* Bytes a real exchange would move per synchronisation and per device

@@ -18,6 +18,8 @@ TPQ_ERR_INVALID_ARG, TPQ_ERR_BAD_STATE, TPQ_ERR_SIZE, TPQ_ERR_ALIGN = 1, 2, 3, 4
 TPQ_ERR_CUDA, TPQ_ERR_NOMEM, TPQ_ERR_TIMEOUT = 5, 6, 7
 TPQ_OUT_BF16, TPQ_OUT_FP32 = 0, 1
 TPQ_OPT_KERNEL_PATH = 0
+TPQ_OPT_DEQUANT_KERNEL = 1
+DQ_AUTO, DQ_ROWS, DQ_TENSOR_PANELS, DQ_COPY_PANELS = 0, 1, 2, 3
 PATH_AUTO, PATH_GENERIC, PATH_TILED = 0, 1, 2
 
 _LIB_PATH = Path(__file__).resolve().parent / "libtpq.so"

@@ -1065,11 +1065,12 @@ cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads,
 // Row kernel geometry; returns false if the shape does not admit it.
 bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *ngroups_out, int *grid_out)
 {
+    const bool forced = c->dq_kernel == 1;
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
     // measured against the panel kernels: the row kernel wins only with few devices and at least about ten
     // rows per SM (the panel kernels start faster and scale better with N)
-    if (N > 4 || T < 10LL * c->sm_count) return false;
+    if (N > 4 || (!forced && T < 10LL * c->sm_count)) return false;
     if (L8 > 768) return false;  // consumer threads (register budget per thread)
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
@@ -1210,7 +1211,7 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     pp.CG = CG;
     pp.panels = (L8 + CG - 1) / CG;
     pp.n_chunks = (T + RC - 1) / RC;
-    if (pp.n_chunks * pp.panels < c->sm_count) return false;  // short inputs: the copy kernel starts faster
+    if (c->dq_kernel != 2 && pp.n_chunks * pp.panels < c->sm_count) return false;  // short inputs: the copy kernel starts faster
     pp.gy = 0;  // (unused: the blocks take equal runs of (panel, chunk) pairs)
     int nstage = 6;
     while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
@@ -1227,7 +1228,9 @@ cudaError_t launch_tpanels_cg(const tpq_ctx *c, const DTParams &tp, const DTMaps
     const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage);
     cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3((unsigned)c->sm_count), dim3(DT_THREADS), smem, st, tp, maps);
+    const int64_t total = (int64_t)tp.d.panels * tp.d.n_chunks;
+    const unsigned grid = (unsigned)(total < c->sm_count ? total : c->sm_count);
+    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3(grid), dim3(DT_THREADS), smem, st, tp, maps);
 }
 
 template <bool FP32OUT>
@@ -1249,7 +1252,8 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
     fill_params(p, c, payloads, T, out, out_stride);
     DXParams x;
     x.hp_idx = c->t.hp_idx; x.hole = c->t.hole; x.filler = c->t.filler; x.n_holes = c->n_holes; x.status = c->t.status;
-    {
+    const int want = c->dq_kernel;  // 0 automatic; 1 row, 2 tensor-map panel, 3 copy-ring panel kernel
+    if (want == 0 || want == 1) {
         DRParams pp;
         int grid = 0;
         if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.ngroups, &grid)) {
@@ -1270,8 +1274,9 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             ++*launches;
             return cudaGetLastError();
         }
+        if (want == 1) return cudaErrorInvalidValue;
     }
-    {
+    if (want == 0 || want == 2) {
         DTParams tp;
         DTMaps maps;
         if (tpanels_plan(const_cast<tpq_ctx *>(c), payloads, T, tp, maps)) {
@@ -1282,9 +1287,13 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             if (e == cudaSuccess) ++*launches;
             return e;
         }
+        if (want == 2) return cudaErrorInvalidValue;
     }
     DPParams dp;
-    if (!panels_plan(c, T, dp)) return tpq_launch_dequant_generic(c, payloads, T, out, fp32_out, out_stride, st, launches);
+    if (!panels_plan(c, T, dp)) {
+        if (want == 3) return cudaErrorInvalidValue;
+        return tpq_launch_dequant_generic(c, payloads, T, out, fp32_out, out_stride, st, launches);
+    }
     dp.q = p;
     dp.s_slot = c->t.s_slot; dp.lp_idx = c->t.lp_idx; dp.hp_idx = c->t.hp_idx;
     dp.filler = c->t.filler; dp.n_holes = c->n_holes;

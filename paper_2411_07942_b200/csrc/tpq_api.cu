@@ -171,6 +171,10 @@ tpq_status tpq_set_option(tpq_ctx *c, tpq_option opt, int value)
         c->kernel_path = value;
         return TPQ_OK;
     }
+    if (opt == TPQ_OPT_DEQUANT_KERNEL && value >= 0 && value <= 3) {
+        c->dq_kernel = value;
+        return TPQ_OK;
+    }
     return fail(c, TPQ_ERR_INVALID_ARG, "unknown option %d or value %d", (int)opt, value);
 }
 
@@ -443,6 +447,8 @@ tpq_status tpq_dequant_reduce(tpq_ctx *c, const void *const *payloads, int n_pay
     else
         e = tpq_launch_dequant_generic(c, payloads, T, out, fp32, out_stride, static_cast<cudaStream_t>(stream),
                                        &c->launches);
+    if (e == cudaErrorInvalidValue && c->dq_kernel != 0)
+        return fail(c, TPQ_ERR_INVALID_ARG, "shape does not admit dequant kernel %d", c->dq_kernel);
     if (e != cudaSuccess) return cuda_fail(c, e, "dequant_reduce kernel");
     return TPQ_OK;
 }

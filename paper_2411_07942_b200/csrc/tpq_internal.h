@@ -36,6 +36,7 @@ struct tpq_ctx {
     int sm_count;
     int smem_optin;     // max dynamic shared memory per block
     int kernel_path;    // TPQ_OPT_KERNEL_PATH
+    int dq_kernel;      // TPQ_OPT_DEQUANT_KERNEL
     int64_t counts[TPQ_MAX_SHARDS];
     tpq_tables t;
     void *scratch;      // calibration partial extremes

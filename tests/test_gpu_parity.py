@@ -159,6 +159,51 @@ def test_row_kernel_equals_generic_on_clustered_feature_sets():
         t.close()
 
 
+@pytest.mark.parametrize("N,T,E,k", [(4, 37, 512, 32), (2, 301, 1024, 32), (3, 16, 4096, 64), (4, 2, 256, 0), (1, 65, 6144, 96)])
+def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
+    """The row, tensor-map panel and copy-ring panel kernels forced in turn on shapes that admit all three
+    (short inputs included, where the automatic choice would not pick them): FP32 and BF16 outputs are
+    bit-identical to the shape-generic kernel's."""
+    w = _workload(N, T, E, 23 * E + T, calib=(2, 8))
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E)
+    gu.calibrate_both(t, [synth.calibration_np(w, i, scale=scale) for i in range(N)])
+    t.select_features(k)
+    P = t.payload_bytes(T)
+    pls = []
+    for i in range(N):
+        y = gu.dev_bf16(synth.activations_np(w, i, T, scale=scale))
+        buf = torch.empty(P, dtype=torch.uint8, device="cuda")
+        t.quantize_pack(i, y.data_ptr(), T, buf.data_ptr(), P)
+        pls.append(buf)
+    ptrs = [b.data_ptr() for b in pls]
+    outs = {}
+    for name, path, kern in [("generic", binding.PATH_GENERIC, binding.DQ_AUTO), ("rows", binding.PATH_TILED, binding.DQ_ROWS),
+                             ("tensor", binding.PATH_TILED, binding.DQ_TENSOR_PANELS),
+                             ("copy", binding.PATH_TILED, binding.DQ_COPY_PANELS)]:
+        t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+        t.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, kern)
+        o32 = torch.full((T, E), float("nan"), dtype=torch.float32, device="cuda")
+        o16 = torch.full((T, E), float("nan"), dtype=torch.bfloat16, device="cuda")
+        t.dequant_reduce(ptrs, T, o32.data_ptr(), binding.TPQ_OUT_FP32)
+        t.dequant_reduce(ptrs, T, o16.data_ptr(), binding.TPQ_OUT_BF16)
+        torch.cuda.synchronize()
+        assert t.device_status() == 0
+        outs[name] = (o32.view(torch.int32).cpu().numpy(), o16.view(torch.int16).cpu().numpy())
+    for name in ("rows", "tensor", "copy"):
+        assert np.array_equal(outs[name][0], outs["generic"][0]), name
+        assert np.array_equal(outs[name][1], outs["generic"][1]), name
+    # a kernel the shape does not admit is refused, not silently replaced
+    t2 = binding.Tpq(5, 512)
+    gu.calibrate_both(t2, [synth.calibration_np(_workload(5, 4, 512, 3, calib=(2, 8)), i) for i in range(5)])
+    t2.select_features(8)
+    t2.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, binding.DQ_ROWS)
+    with pytest.raises(binding.TpqError):
+        t2.dequant_reduce([pls[0].data_ptr()] * 5, 1, torch.empty((1, 512), dtype=torch.bfloat16, device="cuda").data_ptr())
+    t.close()
+    t2.close()
+
+
 def test_tiled_equals_generic_on_clustered_feature_sets():
     """Arbitrary feature sets (the paper's random-selection baseline and worse):
     runs of adjacent selected features, whole groups of 8, first and last feature."""
