@@ -371,10 +371,14 @@ tpq_status tpq_quantize_pack(tpq_ctx *c, int shard, const void *y, int64_t T, in
     if (!aligned16(y) || !aligned16(payload)) return fail(c, TPQ_ERR_ALIGN, "y and payload must be 16-byte aligned");
     if (cap < tpq_payload_bytes(c, T))
         return fail(c, TPQ_ERR_SIZE, "payload capacity %zu < %zu", cap, tpq_payload_bytes(c, T));
-    const bool tiled_ok = tpq_quantize_tiled_ok(c, T, stride);
+    const bool groups_ok = tpq_groups_ok(c, T, stride);
+    const bool tiled_ok = groups_ok || tpq_quantize_tiled_ok(c, T, stride);
     if (c->kernel_path == 2 && !tiled_ok) return fail(c, TPQ_ERR_INVALID_ARG, "shape does not admit the tiled kernel");
     cudaError_t e;
-    if (tiled_ok && c->kernel_path != 1)
+    if (groups_ok && c->kernel_path != 1)
+        e = tpq_launch_quantize_groups(c, shard, 1, &y, T, stride, &payload, static_cast<cudaStream_t>(stream),
+                                       &c->launches);
+    else if (tiled_ok && c->kernel_path != 1)
         e = tpq_launch_quantize_tiled(c, shard, static_cast<const uint16_t *>(y), T, stride,
                                       static_cast<uint8_t *>(payload), static_cast<cudaStream_t>(stream), &c->launches);
     else
@@ -404,10 +408,14 @@ tpq_status tpq_quantize_pack_batch(tpq_ctx *c, int first_shard, int n, const voi
         if (!aligned16(ys[b]) || !aligned16(payloads[b]))
             return fail(c, TPQ_ERR_ALIGN, "y and payload of shard %d must be 16-byte aligned", first_shard + b);
     }
-    const bool tiled_ok = tpq_quantize_tiled_ok(c, T, stride);
+    const bool groups_ok = tpq_groups_ok(c, T, stride);
+    const bool tiled_ok = groups_ok || tpq_quantize_tiled_ok(c, T, stride);
     if (c->kernel_path == 2 && !tiled_ok) return fail(c, TPQ_ERR_INVALID_ARG, "shape does not admit the tiled kernel");
     cudaError_t e = cudaSuccess;
-    if (tiled_ok && c->kernel_path != 1) {
+    if (groups_ok && c->kernel_path != 1) {
+        e = tpq_launch_quantize_groups(c, first_shard, n, ys, T, stride, payloads, static_cast<cudaStream_t>(stream),
+                                       &c->launches);
+    } else if (tiled_ok && c->kernel_path != 1) {
         e = tpq_launch_quantize_tiled_batch(c, first_shard, n, ys, T, stride, payloads, static_cast<cudaStream_t>(stream),
                                             &c->launches);
     } else {
@@ -438,10 +446,14 @@ tpq_status tpq_dequant_reduce(tpq_ctx *c, const void *const *payloads, int n_pay
     }
     if (!aligned16(out)) return fail(c, TPQ_ERR_ALIGN, "out must be 16-byte aligned");
     const int fp32 = dt == TPQ_OUT_FP32;
-    const bool tiled_ok = tpq_dequant_tiled_ok(c, T, out_stride, fp32);
+    const bool groups_ok = tpq_groups_ok(c, T, out_stride);
+    const bool tiled_ok = groups_ok || tpq_dequant_tiled_ok(c, T, out_stride, fp32);
     if (c->kernel_path == 2 && !tiled_ok) return fail(c, TPQ_ERR_INVALID_ARG, "shape does not admit the tiled kernel");
     cudaError_t e;
-    if (tiled_ok && c->kernel_path != 1)
+    if (groups_ok && c->kernel_path != 1)
+        e = tpq_launch_dequant_groups(c, payloads, T, out, fp32, out_stride, static_cast<cudaStream_t>(stream),
+                                      &c->launches);
+    else if (tiled_ok && c->kernel_path != 1)
         e = tpq_launch_dequant_tiled(c, payloads, T, out, fp32, out_stride, static_cast<cudaStream_t>(stream),
                                      &c->launches);
     else

@@ -87,6 +87,13 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
 cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
                                             int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches);
 
+// Code widths other than 4 bits on shapes that are multiples of 8 (groups.cu).
+bool tpq_groups_ok(const tpq_ctx *c, int64_t T, int64_t stride);
+cudaError_t tpq_launch_quantize_groups(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
+                                       int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_dequant_groups(const tpq_ctx *c, const void *const *payloads, int64_t T, void *out, int fp32_out,
+                                      int64_t out_stride, cudaStream_t st, int64_t *launches);
+
 // sum_i D^(i): dequantise + reduce.
 bool tpq_dequant_tiled_ok(const tpq_ctx *c, int64_t T, int64_t out_stride, int fp32_out);
 void tpq_dequant_release(tpq_ctx *c);  // frees dq_cache

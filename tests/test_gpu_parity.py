@@ -60,7 +60,7 @@ def test_generic_path_odd_shapes(N, T, E, k):
 
 @pytest.mark.parametrize("bits", [2, 3, 5, 6, 7, 8])
 @pytest.mark.parametrize("N,T,E,k", [(2, 16, 256, 4), (3, 17, 130, 2), (2, 5, 253, 9), (4, 67, 512, 8), (2, 3, 64, 0),
-                                     (8, 33, 1024, 16)])
+                                     (8, 33, 1024, 16), (2, 129, 5120, 80), (3, 50, 520, 16)])
 def test_other_code_widths(bits, N, T, E, k):
     """The method at lower and higher precision (Section 4 / Figure 3): b-bit codes, step R/(2^b - 1),
     payloads bit-exact against the oracle (codes straddle bytes and words for b = 3, 5, 6, 7), sums in
@@ -69,6 +69,30 @@ def test_other_code_widths(bits, N, T, E, k):
     t = binding.Tpq(N, E, bits=bits)
     assert binding.payload_bytes_for(T, E, k, bits) == oracle.c().payload_bytes(T, E, k, bits)
     t.close()
+
+
+@pytest.mark.parametrize("bits", [2, 3, 5, 6, 7, 8])
+def test_other_code_widths_group_kernels_equal_generic(bits):
+    """The group kernels (shapes that are multiples of 8) against the oracle and, bit for bit, against the
+    shape-generic kernels: strided input, clustered feature sets (several holes in a group, whole groups,
+    selected features at the end)."""
+    N, T, E = 3, 37, 512
+    w = _workload(N, T, E, 90 + bits, calib=(2, 8))
+    scale = synth.column_scales(w)
+    cal = [synth.calibration_np(w, i, scale=scale) for i in range(N)]
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+    rng = np.random.default_rng(bits)
+    sets = [list(range(0, 8)), list(range(0, 15)) + [511], list(range(3, 3 + 24)),
+            sorted(rng.permutation(E)[:64].tolist()), list(range(E - 8, E)), list(range(8, E)), []]
+    for hp in sets:
+        t = binding.Tpq(N, E, bits=bits)
+        gu.calibrate_both(t, cal)
+        t.set_features(hp)
+        a = gu.run_sync(t, ys, path=binding.PATH_GENERIC)
+        b = gu.run_sync(t, ys, path=binding.PATH_TILED, stride_pad=16)
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+        t.close()
 
 
 @pytest.mark.parametrize("N,T,E,k,pad", [(2, 67, 512, 8, 0), (4, 301, 1024, 16, 0), (4, 37, 5120, 80, 64),
