@@ -441,13 +441,14 @@ def test_llama_prefill_full_size():
     _full_pipeline(wc, -1, binding.PATH_AUTO)
 
 
-def test_large_config_sampled_rows():
-    """BASELINE config 5 shape (E = 8192, k = 128) at N = 16 and T = 2048 (the full 8192 rows need
-    2 GB per shard set; rows are independent, so fewer rows exercise the same launch shape).
-    Payload rows and output rows are compared with the oracle on sampled rows."""
+@pytest.mark.parametrize("T,batched", [(2048, False), (8192, True)])
+def test_large_config_sampled_rows(T, batched):
+    """BASELINE config 5 (N = 16, E = 8192, k = 128) at 2048 tokens with one quantize_pack call per shard and
+    at the full 8192 tokens in the launch configuration bench.py times (all shards in one batched launch).
+    Payload rows and output rows are compared with the oracle on sampled rows (rows are independent)."""
     orc = oracle.c()
     w = synth.WORKLOADS["large"]
-    N, E, T = w.n_shards, w.features, 2048
+    N, E = w.n_shards, w.features
     scale = synth.column_scales(w)
     t = binding.Tpq(N, E)
     cal = [synth.calibration_np(w, i, n_seq=2, tokens=64, scale=scale) for i in range(N)]
@@ -460,11 +461,12 @@ def test_large_config_sampled_rows():
     L = E - k
     lpb = orc.lp_bytes(T, E, k)
     ys = [synth.activations_torch(w, i, T, "cuda", scale=scale) for i in range(N)]
-    bufs = []
-    for i in range(N):
-        whole, view = gu.guarded(P)
-        t.quantize_pack(i, ys[i].data_ptr(), T, view.data_ptr(), P)
-        bufs.append((whole, view))
+    bufs = [gu.guarded(P) for _ in range(N)]
+    if batched:
+        t.quantize_pack_batch(0, [y.data_ptr() for y in ys], T, [v.data_ptr() for _, v in bufs], P)
+    else:
+        for i in range(N):
+            t.quantize_pack(i, ys[i].data_ptr(), T, bufs[i][1].data_ptr(), P)
     out = torch.empty((T, E), dtype=torch.float32, device="cuda")
     t.dequant_reduce([v.data_ptr() for _, v in bufs], T, out.data_ptr(), binding.TPQ_OUT_FP32)
     outb = torch.empty((T, E), dtype=torch.bfloat16, device="cuda")
