@@ -501,7 +501,7 @@ def test_large_config_sampled_rows(T, batched):
 
 @pytest.mark.parametrize("N,T,E,k,path", [(4, 301, 1024, 16, binding.PATH_TILED), (8, 64, 4608, 72, binding.PATH_TILED),
                                           (3, 17, 130, 2, binding.PATH_AUTO), (16, 40, 512, 8, binding.PATH_TILED),
-                                          (20, 9, 256, 8, binding.PATH_TILED)])
+                                          (20, 9, 256, 8, binding.PATH_TILED), (4, 2048, 5120, 80, binding.PATH_AUTO)])
 def test_batched_quantize_equals_per_shard_calls(N, T, E, k, path):
     """tpq_quantize_pack_batch writes, for every shard, exactly the payload of tpq_quantize_pack (and of the oracle)."""
     orc = oracle.c()
