@@ -187,19 +187,30 @@ __global__ void __launch_bounds__(GK_THREADS) dequant_groups(const DGParams p)
             for (int r = 0; r < R; ++r)
 #pragma unroll
                 for (int n = 0; n < 8; ++n) acc[r][n] = 0.0f;
-            for (int i = 0; i < p.N; ++i) {
-                const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.s_slot + (size_t)i * E + 8 * g));
-                const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.s_slot + (size_t)i * E + 8 * g + 4));
-                const float s[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+            constexpr int NI = 4;  // devices whose loads are in flight together
+            for (int i0 = 0; i0 < p.N; i0 += NI) {
+                uint64_t bits[NI][R];
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    if (r >= rows) break;
-                    const uint64_t bits = load_code_bytes<B>(p.pl[i] + ((t0 + r) * L8 + g) * B);
+                for (int ii = 0; ii < NI; ++ii)
 #pragma unroll
-                    for (int n = 0; n < 8; ++n) {
-                        // two's complement, B bits: shift the code to the top of a 64-bit integer and back
-                        const int code = (int)((int64_t)(bits << (64 - (n + 1) * B)) >> (64 - B));
-                        acc[r][n] = __fmaf_rn((float)code, s[n], acc[r][n]);
+                    for (int r = 0; r < R; ++r)
+                        if (i0 + ii < p.N && r < rows) bits[ii][r] = load_code_bytes<B>(p.pl[i0 + ii] + ((t0 + r) * L8 + g) * B);
+#pragma unroll
+                for (int ii = 0; ii < NI; ++ii) {
+                    const int i = i0 + ii;
+                    if (i >= p.N) break;
+                    const float4 s0 = __ldg(reinterpret_cast<const float4 *>(p.s_slot + (size_t)i * E + 8 * g));
+                    const float4 s1 = __ldg(reinterpret_cast<const float4 *>(p.s_slot + (size_t)i * E + 8 * g + 4));
+                    const float s[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        if (r >= rows) break;
+#pragma unroll
+                        for (int n = 0; n < 8; ++n) {
+                            // two's complement, B bits: shift the code to the top of a 64-bit integer and back
+                            const int code = (int)((int64_t)(bits[ii][r] << (64 - (n + 1) * B)) >> (64 - B));
+                            acc[r][n] = __fmaf_rn((float)code, s[n], acc[r][n]);
+                        }
                     }
                 }
             }
