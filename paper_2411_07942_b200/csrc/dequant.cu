@@ -909,11 +909,33 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
 
     if (!is_main) {
         // ---------------- fix-up warps
+        // A thread's items of a stage are the same (row of the stage, rank) pairs in every stage, so their
+        // columns, slots and steps are loaded once; sums are formed as soon as the stage has landed (they
+        // read shared memory only) and stored once the main warps' row stores are done.
         const int ft = tid - NT;
+        constexpr int FX_PRE = 2;  // items per thread kept in registers (more: the plain loop below)
+        int f_r[FX_PRE], f_h[FX_PRE], f_hpcol[FX_PRE], f_col[FX_PRE], f_word[FX_PRE], f_sh[FX_PRE];
+        float f_s[FX_PRE][NMAX];
+#pragma unroll
+        for (int j = 0; j < FX_PRE; ++j) {
+            const int item = ft + j * DR_FIXUP_THREADS;
+            const bool on = item < G * k;
+            f_r[j] = on ? item / k : -1;
+            f_h[j] = on ? item - f_r[j] * k : 0;
+            f_hpcol[j] = on ? __ldg(x.hp_idx + f_h[j]) : 0;
+            const bool hole = on && f_h[j] < x.n_holes;
+            f_col[j] = hole ? __ldg(x.filler + f_h[j]) : -1;
+            const int slot = hole ? __ldg(x.hole + f_h[j]) : 0;
+            f_word[j] = f_r[j] * L8 + (slot >> 3);
+            f_sh[j] = (slot & 7) * 4;
+#pragma unroll
+            for (int i = 0; i < NMAX; ++i) f_s[j][i] = (hole && i < N) ? __ldg(p.s_k + (size_t)i * E + f_col[j]) : 0.0f;
+        }
+        const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
         for (int it = 0;; ++it) {
             const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
             if (gi >= pp.ngroups) break;
-            if (!mbar_wait(smem_u32(&full[st]), parity) || !mbar_wait(smem_u32(&main_done[st]), parity)) {
+            if (!mbar_wait(smem_u32(&full[st]), parity)) {
                 atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
                 break;
             }
@@ -921,25 +943,56 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
             const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
             const uint8_t *stage = smem + (size_t)st * lay.stage;
             const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
-            const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
-            for (int item = ft; item < rows * k; item += DR_FIXUP_THREADS) {
+            float hv[FX_PRE], fv[FX_PRE];
+#pragma unroll
+            for (int j = 0; j < FX_PRE; ++j) {
+                hv[j] = 0.0f;
+                fv[j] = 0.0f;
+                if (f_r[j] >= 0 && f_r[j] < rows) {
+#pragma unroll
+                    for (int i = 0; i < NMAX; ++i)
+                        if (i < N) hv[j] = __fadd_rn(hv[j], __uint_as_float((uint32_t)hp[i * hp_dev + f_r[j] * k + f_h[j]] << 16));
+                    if (f_col[j] >= 0) {  // the hole's slot holds the codes of filler feature f_h
+#pragma unroll
+                        for (int i = 0; i < NMAX; ++i)
+                            if (i < N) {
+                                const uint32_t w = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[f_word[j]];
+                                const float code =
+                                    __fsub_rn(__uint_as_float((((w >> f_sh[j]) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
+                                fv[j] = __fmaf_rn(code, f_s[j][i], fv[j]);
+                            }
+                    }
+                }
+            }
+            if (!mbar_wait(smem_u32(&main_done[st]), parity)) {
+                atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
+                break;
+            }
+#pragma unroll
+            for (int j = 0; j < FX_PRE; ++j)
+                if (f_r[j] >= 0 && f_r[j] < rows) {
+                    const int64_t orow = (t0 + f_r[j]) * p.out_stride;
+                    store_one<FP32OUT>(p.out, orow + f_hpcol[j], hv[j]);
+                    if (f_col[j] >= 0) store_one<FP32OUT>(p.out, orow + f_col[j], fv[j]);
+                }
+            for (int item = ft + FX_PRE * DR_FIXUP_THREADS; item < rows * k; item += DR_FIXUP_THREADS) {
                 const int r = item / k, h = item - r * k;  // row of the stage, rank of the selected feature
                 const int64_t orow = (t0 + r) * p.out_stride;
-                float hv = 0.0f;
+                float v = 0.0f;
                 for (int i = 0; i < N; ++i)
-                    hv = __fadd_rn(hv, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
-                store_one<FP32OUT>(p.out, orow + __ldg(x.hp_idx + h), hv);
-                if (h < x.n_holes) {  // the hole's slot holds the codes of filler feature h
+                    v = __fadd_rn(v, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
+                store_one<FP32OUT>(p.out, orow + __ldg(x.hp_idx + h), v);
+                if (h < x.n_holes) {
                     const int slot = __ldg(x.hole + h), col = __ldg(x.filler + h);
-                    float fv = 0.0f;
+                    float u = 0.0f;
                     for (int i = 0; i < N; ++i) {
                         const uint32_t w =
                             reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + (slot >> 3)];
                         const float code = __fsub_rn(
                             __uint_as_float((((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
-                        fv = __fmaf_rn(code, __ldg(p.s_k + (size_t)i * E + col), fv);
+                        u = __fmaf_rn(code, __ldg(p.s_k + (size_t)i * E + col), u);
                     }
-                    store_one<FP32OUT>(p.out, orow + col, fv);
+                    store_one<FP32OUT>(p.out, orow + col, u);
                 }
             }
             __syncwarp();
