@@ -762,7 +762,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 }
 
 // ----------------------------------------------------------------------------------------------
-// Row kernel for N <= 4 devices, (E-k)/8 <= MAXT main threads and long inputs.
+// Row kernel for N <= 4 devices and (E-k)/8 <= MAXT main threads.
 //
 // One persistent block per SM with three kinds of warps:
 //   producer (1 warp)  streams groups of G rows of all N payloads (a code-row block and a BF16 block per
@@ -1118,12 +1118,12 @@ cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads,
 // Row kernel geometry; returns false if the shape does not admit it.
 bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *ngroups_out, int *grid_out)
 {
-    const bool forced = c->dq_kernel == 1;
+
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
-    // measured against the panel kernels: the row kernel wins only with few devices and at least about ten
-    // rows per SM (the panel kernels start faster and scale better with N)
-    if (N > 4 || (!forced && T < 10LL * c->sm_count)) return false;
+    // measured against the panel kernels: the row kernel wins with up to 4 devices at every input length
+    // (the panel kernels scale better with N)
+    if (N > 4) return false;
     if (L8 > 768) return false;  // consumer threads (register budget per thread)
     int g0 = 4;
     if (L8 % 4 == 0) g0 = 1;
