@@ -47,7 +47,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"quantize_tiled_batch": 88030464, "dequant_rows": 22074880}
+NCU_TRAFFIC_BYTES = {"quantize_tiled_batch": 88030464, "dequant_rows": 22081792}
 
 
 # ------------------------------------------------------------------ helpers
