@@ -228,6 +228,52 @@ def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
     t2.close()
 
 
+@pytest.mark.parametrize("N,T,E,k", [(4, 301, 1024, 16), (16, 1203, 2048, 32), (9, 100, 1040, 8)])
+def test_back_to_back_launches_and_graph_replay_give_the_eager_result(N, T, E, k):
+    """Calls enqueued back to back on one stream (the kernels start before the one ahead has drained and wait
+    for it before touching its data) and the same calls replayed from a CUDA graph give the bits of calls
+    separated by synchronisation; a step may overwrite the buffers of the step before."""
+    w = _workload(N, T, E, 29 * E + T, calib=(2, 8))
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E)
+    gu.calibrate_both(t, [synth.calibration_np(w, i, scale=scale) for i in range(N)])
+    t.select_features(k)
+    P = t.payload_bytes(T)
+    ys = [[gu.dev_bf16(synth.activations_np(w, i, T, scale=scale) ^ np.uint16(0x8000 * v)) for i in range(N)]
+          for v in range(2)]                     # two input sets (the second with every sign flipped)
+    pls = [torch.empty(P, dtype=torch.uint8, device="cuda") for _ in range(N)]
+    out = torch.empty((T, E), dtype=torch.bfloat16, device="cuda")
+    ptrs = [p_.data_ptr() for p_ in pls]
+
+    def step(v, stream):
+        t.quantize_pack_batch(0, [y.data_ptr() for y in ys[v]], T, ptrs, P, stream=stream)
+        t.dequant_reduce(ptrs, T, out.data_ptr(), stream=stream)
+
+    want = []
+    for v in range(2):                           # eager, synchronised
+        step(v, 0)
+        torch.cuda.synchronize()
+        want.append(out.view(torch.int16).cpu().numpy().copy())
+    assert not np.array_equal(want[0], want[1])
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                # back to back: payloads and output reused by consecutive steps
+        for rep in range(6):
+            step(rep & 1, side.cuda_stream)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.view(torch.int16).cpu().numpy(), want[1])
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step(1, side.cuda_stream)
+        step(0, side.cuda_stream)
+    out.zero_()
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert t.device_status() == 0
+    assert np.array_equal(out.view(torch.int16).cpu().numpy(), want[0])
+    t.close()
+
+
 def test_tiled_equals_generic_on_clustered_feature_sets():
     """Arbitrary feature sets (the paper's random-selection baseline and worse):
     runs of adjacent selected features, whole groups of 8, first and last feature."""
