@@ -75,6 +75,8 @@ class COracle:
         L.tpqo_quantize_pack_b.argtypes = [u16p, i64, i64, i64, i32p, i64, f32p, ci, u8p]
         L.tpqo_dequant_reduce_b.argtypes = [ctypes.POINTER(u8p), i64, i64, i64, i32p, i64, f32p, ci,
                                             ctypes.POINTER(ctypes.c_double), f32p]
+        L.tpqo_dequant_reduce_bias_b.argtypes = [ctypes.POINTER(u8p), i64, i64, i64, i32p, i64, f32p, ci, f32p,
+                                                 ctypes.POINTER(ctypes.c_double), f32p]
 
     def num_threads(self) -> int:
         return int(self.lib.tpqo_num_threads())
@@ -173,7 +175,7 @@ class COracle:
         return out
 
     def dequant_reduce(self, payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray,
-                       want_chain32: bool = True, bits: int = 4):
+                       want_chain32: bool = True, bits: int = 4, bias=None):
         N = len(payloads)
         hp = np.ascontiguousarray(hp_idx, dtype=np.int32)
         k = hp.shape[0]
@@ -187,7 +189,13 @@ class COracle:
         ref = np.empty((T, E), np.float64)
         chain = np.empty((T, E), np.float32) if want_chain32 else None
         hp_arg = hp if k else np.zeros(1, np.int32)
-        if bits == 4:
+        if bias is not None:
+            b = np.ascontiguousarray(bias, dtype=np.float32)
+            assert b.shape == (E,)
+            self.lib.tpqo_dequant_reduce_bias_b(arr, N, T, E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(s, ctypes.c_float),
+                                                bits, _ptr(b, ctypes.c_float), _ptr(ref, ctypes.c_double),
+                                                _ptr(chain, ctypes.c_float) if want_chain32 else None)
+        elif bits == 4:
             self.lib.tpqo_dequant_reduce(arr, N, T, E, _ptr(hp_arg, ctypes.c_int32), k, _ptr(s, ctypes.c_float),
                                          _ptr(ref, ctypes.c_double),
                                          _ptr(chain, ctypes.c_float) if want_chain32 else None)

@@ -180,7 +180,7 @@ def unpack(payload: np.ndarray, T: int, E: int, k: int, bits: int = 4):
 
 
 # ------------------------------------------------------------------ decompression + sum
-def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray, bits: int = 4):
+def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray, bits: int = 4, bias=None):
     """Sum over devices of the dequantised payloads, in float64, original feature order."""
     k = len(hp_idx)
     lp = lp_index(E, hp_idx)
@@ -190,4 +190,6 @@ def dequant_reduce(payloads, T: int, E: int, hp_idx: np.ndarray, s: np.ndarray, 
         out[:, lp] += codes.astype(np.float64) * s[i, lp].astype(np.float64)[None, :]
         if k:
             out[:, np.asarray(hp_idx, dtype=np.int64)] += widen(hp).astype(np.float64)
+    if bias is not None:    # f(x) = sum_i f_i(x_i) + b
+        out += np.asarray(bias, dtype=F32).astype(np.float64)[None, :]
     return out

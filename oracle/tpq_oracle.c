@@ -46,6 +46,8 @@ void tpqo_quantize_pack_b(const uint16_t *y, int64_t T, int64_t E, int64_t strid
                           const float *inv_s, int bits, uint8_t *payload);
 void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T, int64_t E, const int32_t *hp_idx,
                            int64_t k, const float *s, int bits, double *ref64, float *chain32);
+void tpqo_dequant_reduce_bias_b(const uint8_t *const *payloads, int64_t N, int64_t T, int64_t E, const int32_t *hp_idx,
+                                int64_t k, const float *s, int bits, const float *bias, double *ref64, float *chain32);
 
 #ifdef _OPENMP
 #include <omp.h>
@@ -346,6 +348,16 @@ void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T,
                            int64_t E, const int32_t *hp_idx, int64_t k,
                            const float *s, int bits, double *ref64, float *chain32)
 {
+    tpqo_dequant_reduce_bias_b(payloads, N, T, E, hp_idx, k, s, bits, NULL, ref64, chain32);
+}
+
+/* Section 2: the synchronised layer output is f(x) = sum_i f^(i)(x^(i)) + b.  With a bias b[E] (binary32)
+ * the reference adds it in binary64 and the chain adds it last, chain32 = fl(acc32 + b_j); bias == NULL
+ * leaves the sum as it is. */
+void tpqo_dequant_reduce_bias_b(const uint8_t *const *payloads, int64_t N, int64_t T,
+                                int64_t E, const int32_t *hp_idx, int64_t k,
+                                const float *s, int bits, const float *bias, double *ref64, float *chain32)
+{
     int64_t L = E - k;
     int64_t lp_bytes = tpqo_lp_bytes_b(T, E, k, bits);
     const unsigned cmask = (1u << bits) - 1u, sign = 1u << (bits - 1);
@@ -381,6 +393,11 @@ void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T,
                     volatile float tmp = acc32 + v;
                     acc32 = tmp;
                 }
+            }
+            if (bias) {
+                acc64 += (double)bias[j];
+                volatile float tmp = acc32 + bias[j];
+                acc32 = tmp;
             }
             if (ref64) ref64[t * E + j] = acc64;
             if (chain32) chain32[t * E + j] = acc32;

@@ -120,3 +120,30 @@ def test_aggregated_error_is_irwin_hall(corc, norc, N):
     emp = (np.arange(xs.size) + 0.5) / xs.size
     ks = np.abs(emp - _irwin_hall_cdf(xs, N)).max()
     assert ks < 0.01, ks
+
+
+def test_bias_is_added_after_the_sum(corc, norc):
+    """Section 2: f(x) = sum_i f_i(x_i) + b.  The reference with a bias is the reference without it plus b,
+    exactly (binary64); the chain adds b last; a zero bias changes no value; with every feature selected
+    and one device the output is y + b computed by the library."""
+    rng = np.random.default_rng(12)
+    N, T, E = 3, 7, 48
+    hp = np.array([1, 5, 20, 47], np.int32)
+    y = [bf16_bits((rng.normal(0, 2, (T, E))).astype(np.float32)) for _ in range(N)]
+    R = np.stack([2 * np.abs(bf16_value(v)).max(axis=0) for v in y]).astype(np.float32)
+    s, inv = corc.params(R)
+    pls = [corc.quantize_pack(y[i], hp, inv[i]) for i in range(N)]
+    bias = rng.normal(0, 3, E).astype(np.float32)
+    ref0, chain0 = corc.dequant_reduce(pls, T, E, hp, s)
+    ref1, chain1 = corc.dequant_reduce(pls, T, E, hp, s, bias=bias)
+    assert np.array_equal(ref1, ref0 + bias.astype(np.float64)[None, :])
+    assert np.array_equal(chain1, (chain0 + bias[None, :]).astype(np.float32))
+    assert np.array_equal(norc.dequant_reduce(pls, T, E, hp, s, 4, bias), ref1)
+    refz, chainz = corc.dequant_reduce(pls, T, E, hp, s, bias=np.zeros(E, np.float32))
+    assert np.array_equal(refz, ref0) and np.array_equal(chainz + 0.0, chain0 + 0.0)
+    # every feature selected, one device: the payload is y itself
+    allhp = np.arange(E, dtype=np.int32)
+    p1 = corc.quantize_pack(y[0], allhp, inv[0])
+    ref, chain = corc.dequant_reduce([p1], T, E, allhp, s[:1], bias=bias)
+    assert np.array_equal(ref, bf16_value(y[0]) + bias.astype(np.float64)[None, :])
+    assert np.array_equal(chain, (bf16_value(y[0]).astype(np.float32) + bias[None, :]).astype(np.float32))
