@@ -353,6 +353,13 @@ def main():
     q_ms = time_loop(q_only, reps) / N          # per single-shard launch
     qb_ms = time_loop(qb_only, reps)            # per batched launch (N shards)
     d_ms = time_loop(d_only, reps)
+    bias_dev = torch.zeros(E, dtype=torch.float32, device=dev).normal_(generator=torch.Generator(device=dev).manual_seed(7))
+
+    def db_only(b):         # the same with the layer's bias added in the kernel's store (Section 2)
+        _, _, out, _, parr = sets[b % args.sets]
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh, bias_ptr=bias_dev.data_ptr())
+
+    db_ms = time_loop(db_only, reps)
     # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
     # what the launch path costs, relevant for the decode-sized workloads
     graph_ms = None
@@ -455,6 +462,7 @@ def main():
     extra = {
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
         "step_cuda_graph_replay_ms": graph_ms,
+        "dequant_reduce_bias_ms_per_launch": db_ms,
         "payload_bytes_per_shard": int(comm.payload_bytes),
         "comm_bytes_per_rank": {"quantized_allgather": int(comm.quantized_allgather_send),
                                 "bf16_allgather": int(comm.bf16_allgather_send),

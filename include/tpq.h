@@ -219,6 +219,15 @@ tpq_status tpq_quantize_pack_batch(tpq_ctx *ctx, int first_shard, int n, const v
 tpq_status tpq_dequant_reduce(tpq_ctx *ctx, const void *const *payloads_dev_host, int n_payloads, int64_t T,
                               void *out_dev, tpq_out_dtype dt, int64_t out_row_stride_elems, void *cuda_stream);
 
+/* The same with the layer's bias added after the sum (Section 2: f(x) = sum_i f^(i)(x^(i)) + b):
+ * out[t][j] = round(fl32(acc[t][j] + bias[j])), acc the binary32 sum of tpq_dequant_reduce before its
+ * final rounding.  bias_dev: DEVICE pointer to E binary32 values, 16-byte aligned, read during the
+ * call's kernels (the caller keeps it alive and unchanged until they have run).  Errors as
+ * tpq_dequant_reduce, plus INVALID_ARG for a NULL bias and ALIGN for a misaligned one. */
+tpq_status tpq_dequant_reduce_bias(tpq_ctx *ctx, const void *const *payloads_dev_host, int n_payloads, int64_t T,
+                                   void *out_dev, tpq_out_dtype out_dtype, int64_t out_row_stride,
+                                   const float *bias_dev, void *stream);
+
 /* ------------------------------------------------- checkpoint and status */
 
 /* Serialise / restore the whole static state (N, E, bits, gamma, counts, m, M,

@@ -53,6 +53,8 @@ SIGNATURES = {
     "tpq_quantize_pack_batch": (c_int, [c_void_p, c_int, c_int, POINTER(c_void_p), c_int64, c_int64, POINTER(c_void_p),
                                         c_size_t, c_void_p]),
     "tpq_dequant_reduce": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p]),
+    "tpq_dequant_reduce_bias": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p,
+                                        c_void_p]),
     "tpq_get_state": (c_int, [c_void_p, c_void_p, POINTER(c_size_t)]),
     "tpq_set_state": (c_int, [c_void_p, c_void_p, c_size_t]),
     "tpq_device_status": (c_int, [c_void_p]),
@@ -203,10 +205,14 @@ class Tpq:
                                                   payload_capacity, stream))
 
     def dequant_reduce(self, payload_ptrs, T: int, out_ptr: int, out_dtype: int = TPQ_OUT_BF16,
-                       out_row_stride: int | None = None, stream: int = 0):
+                       out_row_stride: int | None = None, stream: int = 0, bias_ptr: int | None = None):
         arr = payload_ptrs if isinstance(payload_ptrs, ctypes.Array) else (c_void_p * len(payload_ptrs))(*payload_ptrs)
-        self._check(lib().tpq_dequant_reduce(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype,
-                                             self.E if out_row_stride is None else out_row_stride, stream))
+        stride = self.E if out_row_stride is None else out_row_stride
+        if bias_ptr is None:
+            self._check(lib().tpq_dequant_reduce(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride, stream))
+        else:
+            self._check(lib().tpq_dequant_reduce_bias(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride,
+                                                      bias_ptr, stream))
 
     def get_state(self) -> bytes:
         n = c_size_t(0)

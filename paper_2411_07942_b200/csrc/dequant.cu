@@ -23,6 +23,7 @@ struct DQParams {
     const uint32_t *grp;   // [E/8]
     void *out;
     int64_t out_stride;
+    const float *bias;     // [E] added after the sum (Section 2: f(x) = sum_i f_i(x_i) + b), or NULL
 };
 
 // ----------------------------------------------------------------------------------------------
@@ -57,6 +58,7 @@ __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
                 acc = __fadd_rn(acc, __uint_as_float((uint32_t)v << 16));
             }
         }
+        if (p.bias) acc = __fadd_rn(acc, p.bias[j]);
         if (FP32OUT)
             static_cast<float *>(p.out)[t * p.out_stride + j] = acc;
         else
@@ -275,8 +277,30 @@ __device__ __forceinline__ void cp_async_wait()
 // lp_idx[8g+n] and goes to that feature's column
 template <bool FP32OUT>
 __device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *lp_idx, int64_t t0, int g, uint32_t mask,
-                                              const float2 (&acc)[DP_R][4])
+                                              const float2 (&acc_in)[DP_R][4])
 {
+    float2 acc[DP_R][4];
+#pragma unroll
+    for (int r = 0; r < DP_R; ++r)
+#pragma unroll
+        for (int h = 0; h < 4; ++h) acc[r][h] = acc_in[r][h];
+    if (p.bias) {
+        // lane n belongs to feature 8g+n, or, at a hole, to the filler feature whose codes sit in the slot
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g));
+        const float4 b1 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g + 4));
+        float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        const uint32_t holes = __ldg(p.grp + g) & 0xFFu;
+        if (holes) {
+#pragma unroll
+            for (int n = 0; n < 8; ++n)
+                if (holes & (1u << n)) b[n] = __ldg(p.bias + __ldg(lp_idx + 8 * g + n));
+        }
+#pragma unroll
+        for (int r = 0; r < DP_R; ++r)
+#pragma unroll
+            for (int h = 0; h < 4; ++h)
+                acc[r][h] = __fadd2_rn(acc[r][h], make_float2(b[2 * h], b[2 * h + 1]));
+    }
     if (mask == 0) {
 #pragma unroll
         for (int r = 0; r < DP_R; ++r)
@@ -416,7 +440,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                 static_cast<uint16_t *>(p.out)[orow + filler_col] =
                     __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
         }
-        store_one<FP32OUT>(p.out, orow + sel_col, v);
+        store_one<FP32OUT>(p.out, orow + sel_col, p.bias ? __fadd_rn(v, __ldg(p.bias + sel_col)) : v);
     };
     // the items of the chunk whose first row is tcp: this thread's pipelined one (sum v) and, in panels with
     // more items than threads, the rest
@@ -434,7 +458,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                 else
                     static_cast<uint16_t *>(p.out)[fl_row + my_fcol] = (uint16_t)__float_as_uint(fl_f);
             }
-            store_one<FP32OUT>(p.out, fl_row + my_col, fl_v);
+            store_one<FP32OUT>(p.out, fl_row + my_col, p.bias ? __fadd_rn(fl_v, __ldg(p.bias + my_col)) : fl_v);
             fl_on = false;
         }
     };
@@ -702,7 +726,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                     static_cast<uint16_t *>(p.out)[orow + filler_col] =
                         __ldcg(static_cast<const uint16_t *>(p.out) + orow + sel_col);
             }
-            store_one<FP32OUT>(p.out, orow + sel_col, v);
+            store_one<FP32OUT>(p.out, orow + sel_col, p.bias ? __fadd_rn(v, __ldg(p.bias + sel_col)) : v);
         };
 
         for (int64_t ch = chb; ch < che; ++ch) {
@@ -849,7 +873,7 @@ __device__ __forceinline__ long long tpq_dnow()
 #define TPQ_DMARK(slot) do { } while (0)
 #endif
 
-template <int NMAX, int MAXT, bool FP32OUT>
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
 __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -1003,6 +1027,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
             for (int j = 0; j < FX_PRE; ++j)
                 if (f_r[j] >= 0 && f_r[j] < rows) {
                     const int64_t orow = (t0 + f_r[j]) * p.out_stride;
+                    if (HAS_BIAS) {
+                        hv[j] = __fadd_rn(hv[j], __ldg(p.bias + f_hpcol[j]));
+                        if (f_col[j] >= 0) fv[j] = __fadd_rn(fv[j], __ldg(p.bias + f_col[j]));
+                    }
                     store_one<FP32OUT>(p.out, orow + f_hpcol[j], hv[j]);
                     if (f_col[j] >= 0) store_one<FP32OUT>(p.out, orow + f_col[j], fv[j]);
                 }
@@ -1012,7 +1040,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
                 float v = 0.0f;
                 for (int i = 0; i < N; ++i)
                     v = __fadd_rn(v, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
-                store_one<FP32OUT>(p.out, orow + __ldg(x.hp_idx + h), v);
+                {
+                    const int hc = __ldg(x.hp_idx + h);
+                    store_one<FP32OUT>(p.out, orow + hc, HAS_BIAS ? __fadd_rn(v, __ldg(p.bias + hc)) : v);
+                }
                 if (h < x.n_holes) {
                     const int slot = __ldg(x.hole + h), col = __ldg(x.filler + h);
                     float u = 0.0f;
@@ -1023,7 +1054,7 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
                             __uint_as_float((((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
                         u = __fmaf_rn(code, __ldg(p.s_k + (size_t)i * E + col), u);
                     }
-                    store_one<FP32OUT>(p.out, orow + col, u);
+                    store_one<FP32OUT>(p.out, orow + col, HAS_BIAS ? __fadd_rn(u, __ldg(p.bias + col)) : u);
                 }
             }
             __syncwarp();
@@ -1077,6 +1108,16 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
                 }
             }
             if (live) {
+                if (HAS_BIAS) {  // (a hole's lane gets its own column's bias here and is overwritten by the fix-up)
+                    const float4 b0 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld));
+                    const float4 b1 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld + 4));
+                    const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y),
+                                         make_float2(b1.z, b1.w)};
+#pragma unroll
+                    for (int r = 0; r < 2; ++r)
+#pragma unroll
+                        for (int h = 0; h < 4; ++h) acc[r][h] = __fadd2_rn(acc[r][h], b[h]);
+                }
                 store_group<FP32OUT>(orow, 0, acc[0], 0u);
                 if (two) store_group<FP32OUT>(orow + out_row_bytes, 0, acc[1], 0u);
             }
@@ -1102,6 +1143,7 @@ void fill_params(DQParams &p, const tpq_ctx *c, const void *const *payloads, int
     p.lp_bytes = tpq_lp_bytes_i(T, c->E, c->k, c->bits);
     p.s_k = c->t.s_k; p.pos = c->t.pos; p.grp = c->t.grp;
     p.out = out; p.out_stride = out_stride;
+    p.bias = c->call_bias;
 }
 
 }  // namespace
@@ -1132,18 +1174,25 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
 
 namespace {
 
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
+cudaError_t launch_rows_v(const DRParams &pp, int grid, int threads, size_t smem, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS>, dim3(grid), dim3(threads), smem, st, pp);
+    return e;
+}
+
 template <int NMAX, int MAXT>
 cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads, size_t smem, cudaStream_t st)
 {
-    cudaError_t e;
-    if (fp32_out) {
-        e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, true>, dim3(grid), dim3(threads), smem, st, pp);
-    } else {
-        e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e == cudaSuccess) e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, false>, dim3(grid), dim3(threads), smem, st, pp);
-    }
-    return e;
+    const bool bias = pp.q.bias != nullptr;
+    if (fp32_out)
+        return bias ? launch_rows_v<NMAX, MAXT, true, true>(pp, grid, threads, smem, st)
+                    : launch_rows_v<NMAX, MAXT, true, false>(pp, grid, threads, smem, st);
+    return bias ? launch_rows_v<NMAX, MAXT, false, true>(pp, grid, threads, smem, st)
+                : launch_rows_v<NMAX, MAXT, false, false>(pp, grid, threads, smem, st);
 }
 
 // Row kernel geometry; returns false if the shape does not admit it.

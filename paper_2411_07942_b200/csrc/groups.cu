@@ -158,6 +158,7 @@ struct DGParams {
     const uint32_t *grp;
     const int32_t *lp_idx, *hp_idx;
     void *out;
+    const float *bias;  // [E] added after the sum, or NULL
 };
 
 template <bool FP32OUT>
@@ -215,6 +216,15 @@ __global__ void __launch_bounds__(GK_THREADS) dequant_groups(const DGParams p)
                 }
             }
             const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
+            if (p.bias) {
+#pragma unroll
+                for (int n = 0; n < 8; ++n) {
+                    const int col = (mask & (1u << n)) ? __ldg(p.lp_idx + 8 * g + n) : 8 * g + n;
+                    const float b = __ldg(p.bias + col);
+#pragma unroll
+                    for (int r = 0; r < R; ++r) acc[r][n] = __fadd_rn(acc[r][n], b);
+                }
+            }
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 if (r >= rows) break;
@@ -270,7 +280,9 @@ __global__ void __launch_bounds__(GK_THREADS) dequant_groups(const DGParams p)
             for (int r = 0; r < R; ++r) {
                 if (r >= rows) break;
 #pragma unroll
-                for (int n = 0; n < 8; ++n) gk_store<FP32OUT>(p.out, (t0 + r) * p.out_stride + col[n], acc[r][n]);
+                for (int n = 0; n < 8; ++n)
+                    gk_store<FP32OUT>(p.out, (t0 + r) * p.out_stride + col[n],
+                                      p.bias ? __fadd_rn(acc[r][n], __ldg(p.bias + col[n])) : acc[r][n]);
             }
         }
     }
@@ -349,6 +361,7 @@ cudaError_t tpq_launch_dequant_groups(const tpq_ctx *c, const void *const *paylo
     p.out_stride = out_stride;
     p.s_slot = c->t.s_slot; p.grp = c->t.grp; p.lp_idx = c->t.lp_idx; p.hp_idx = c->t.hp_idx;
     p.out = out;
+    p.bias = c->call_bias;
     const int64_t units = ((T + 1) / 2) * (int64_t)((E - k) / 8 + k / 8);
     const unsigned grid = gk_grid(units, c->sm_count);
     switch (c->bits) {

@@ -428,10 +428,33 @@ tpq_status tpq_quantize_pack_batch(tpq_ctx *c, int first_shard, int n, const voi
     return TPQ_OK;
 }
 
+static tpq_status dequant_reduce_impl(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
+                                      tpq_out_dtype dt, int64_t out_stride, void *stream);
+
 tpq_status tpq_dequant_reduce(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
                               tpq_out_dtype dt, int64_t out_stride, void *stream)
 {
     if (!c) return TPQ_ERR_INVALID_ARG;
+    c->call_bias = nullptr;
+    return dequant_reduce_impl(c, payloads, n_payloads, T, out, dt, out_stride, stream);
+}
+
+tpq_status tpq_dequant_reduce_bias(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
+                                   tpq_out_dtype dt, int64_t out_stride, const float *bias, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (!bias) return fail(c, TPQ_ERR_INVALID_ARG, "bias is NULL (use tpq_dequant_reduce)");
+    if (!aligned16(bias)) return fail(c, TPQ_ERR_ALIGN, "bias must be 16-byte aligned");
+    c->call_bias = bias;
+    const tpq_status st = dequant_reduce_impl(c, payloads, n_payloads, T, out, dt, out_stride, stream);
+    c->call_bias = nullptr;
+    return st;
+}
+
+static tpq_status dequant_reduce_impl(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
+                                      tpq_out_dtype dt, int64_t out_stride, void *stream)
+{
     c->err[0] = 0;
     if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set: call tpq_select_features or tpq_set_features");
     if (n_payloads != c->N) return fail(c, TPQ_ERR_INVALID_ARG, "n_payloads = %d, expected N = %d", n_payloads, c->N);

@@ -43,6 +43,7 @@ struct tpq_ctx {
     size_t scratch_bytes;
     int64_t launches;
     void *dq_cache;     // tensor maps of recently used payloads (dequant.cu)
+    const float *call_bias;  // bias of the tpq_dequant_reduce_bias call in progress (NULL otherwise)
     char err[512];
 };
 

@@ -274,6 +274,54 @@ def test_back_to_back_launches_and_graph_replay_give_the_eager_result(N, T, E, k
     t.close()
 
 
+@pytest.mark.parametrize("N,T,E,k,bits", [(4, 37, 512, 32, 4), (2, 301, 1024, 32, 4), (3, 150, 4096, 64, 4), (2, 5, 253, 9, 4),
+                                          (3, 33, 512, 8, 8), (2, 19, 130, 2, 3), (4, 64, 512, 0, 4)])
+def test_bias_is_added_after_the_sum(N, T, E, k, bits):
+    """tpq_dequant_reduce_bias (Section 2: f(x) = sum_i f_i(x_i) + b) on every kernel the shape admits:
+    FP32 output bit-identical to the oracle's chain fl(acc + b), BF16 output to its rounding; hole, filler and
+    selected columns get their own bias."""
+    orc = oracle.c()
+    w = _workload(N, T, E, 37 * E + T, calib=(2, 8))
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E, bits=bits)
+    gu.calibrate_both(t, [synth.calibration_np(w, i, scale=scale) for i in range(N)])
+    hp = t.select_features(k)
+    s_, inv = t.get_scales()
+    P = t.payload_bytes(T)
+    ys = [synth.activations_np(w, i, T, scale=scale) for i in range(N)]
+    host = [orc.quantize_pack(ys[i], hp, inv[i], bits) for i in range(N)]
+    pls = [torch.from_numpy(h).cuda() for h in host]
+    ptrs = [b.data_ptr() for b in pls]
+    bias = (np.random.default_rng(E + T).normal(0, 1, E) * np.abs(s_).mean(axis=0) * 5).astype(np.float32)
+    bias_d = torch.from_numpy(bias).cuda()
+    ref, chain = orc.dequant_reduce(host, T, E, hp, s_, bits=bits, bias=bias)
+    want16 = orc.round_bf16(chain)
+    tiled = E % 8 == 0 and k % 8 == 0
+    kernels = [(binding.PATH_GENERIC, binding.DQ_AUTO)]
+    if tiled:
+        kernels.append((binding.PATH_TILED, binding.DQ_AUTO))
+    if tiled and bits == 4:
+        kernels += [(binding.PATH_TILED, binding.DQ_COPY_PANELS)]
+        if N <= 4:
+            kernels.append((binding.PATH_TILED, binding.DQ_ROWS))
+        if (E - k) % 32 == 0:
+            kernels.append((binding.PATH_TILED, binding.DQ_TENSOR_PANELS))
+    for path, kern in kernels:
+        t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+        t.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, kern)
+        o32 = torch.full((T, E), float("nan"), dtype=torch.float32, device="cuda")
+        o16 = torch.full((T, E), float("nan"), dtype=torch.bfloat16, device="cuda")
+        t.dequant_reduce(ptrs, T, o32.data_ptr(), binding.TPQ_OUT_FP32, bias_ptr=bias_d.data_ptr())
+        t.dequant_reduce(ptrs, T, o16.data_ptr(), binding.TPQ_OUT_BF16, bias_ptr=bias_d.data_ptr())
+        torch.cuda.synchronize()
+        assert t.device_status() == 0
+        assert gu.bits_equal(o32.cpu().numpy(), chain), (path, kern)
+        assert np.array_equal(o16.view(torch.int16).cpu().numpy().view(np.uint16), want16), (path, kern)
+    with pytest.raises(binding.TpqError):
+        t.dequant_reduce(ptrs, T, o32.data_ptr(), binding.TPQ_OUT_FP32, bias_ptr=bias_d.data_ptr() + 4)
+    t.close()
+
+
 def test_tiled_equals_generic_on_clustered_feature_sets():
     """Arbitrary feature sets (the paper's random-selection baseline and worse):
     runs of adjacent selected features, whole groups of 8, first and last feature."""
