@@ -129,33 +129,63 @@ __global__ void __launch_bounds__(256) colminmax_generic(const uint16_t *__restr
 
 // Eq. (1)-(2): combine the row splits of every sequence, then fold the sequences in order.
 // m <- fl( fl((1-gamma) m) + fl(gamma min) ); the first sequence a device sees initialises.
-__global__ void __launch_bounds__(256) ema_fold(const int16_t *__restrict__ part_lo,
-                                                const int16_t *__restrict__ part_hi, int64_t n_seq, int n_split, int E,
-                                                float *__restrict__ m, float *__restrict__ M, int64_t count0,
-                                                float gamma)
+//
+// A block owns EF_X features.  Its EF_Y thread rows first reduce the splits of EF_Q sequences side by side
+// (extremes are order-free, and these loads are the latency of the kernel: one thread walking every partial
+// of a feature pays one L2 round trip per sequence and split), park the per-sequence extremes in shared
+// memory, and the first thread row then runs the moving average over them in sequence order.
+constexpr int EF_X = 32, EF_Y = 8, EF_Q = 64;
+
+__global__ void __launch_bounds__(EF_X *EF_Y) ema_fold(const int16_t *__restrict__ part_lo,
+                                                       const int16_t *__restrict__ part_hi, int64_t n_seq, int n_split,
+                                                       int E, float *__restrict__ m, float *__restrict__ M,
+                                                       int64_t count0, float gamma)
 {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= E) return;
+    __shared__ int16_t s_lo[EF_Q][EF_X], s_hi[EF_Q][EF_X];
+    const int x = threadIdx.x & (EF_X - 1), yl = threadIdx.x / EF_X;
+    const int j = blockIdx.x * EF_X + x;
+    const bool live = j < E;
     const float c = __fsub_rn(1.0f, gamma);
-    float mj = m[j], Mj = M[j];
-    for (int64_t q = 0; q < n_seq; ++q) {
-        int lo = 0x7FFF, hi = -0x8000;
-        for (int sp = 0; sp < n_split; ++sp) {
-            const int64_t o = (q * n_split + sp) * (int64_t)E + j;
-            lo = min(lo, (int)part_lo[o]);
-            hi = max(hi, (int)part_hi[o]);
-        }
-        const float mn = key_to_float((int16_t)lo), mx = key_to_float((int16_t)hi);
-        if (count0 + q == 0) {
-            mj = mn;
-            Mj = mx;
-        } else {
-            mj = __fadd_rn(__fmul_rn(c, mj), __fmul_rn(gamma, mn));
-            Mj = __fadd_rn(__fmul_rn(c, Mj), __fmul_rn(gamma, mx));
-        }
+    float mj = 0.f, Mj = 0.f;
+    if (live && yl == 0) {
+        mj = m[j];
+        Mj = M[j];
     }
-    m[j] = mj;
-    M[j] = Mj;
+    for (int64_t q0 = 0; q0 < n_seq; q0 += EF_Q) {
+        const int nq = (int)((n_seq - q0 < EF_Q) ? n_seq - q0 : EF_Q);
+        for (int u = yl; u < nq; u += EF_Y) {
+            int lo = 0x7FFF, hi = -0x8000;
+            if (live) {
+                const int16_t *pl = part_lo + (q0 + u) * n_split * (int64_t)E + j;
+                const int16_t *ph = part_hi + (q0 + u) * n_split * (int64_t)E + j;
+#pragma unroll 4
+                for (int sp = 0; sp < n_split; ++sp) {
+                    lo = min(lo, (int)pl[(int64_t)sp * E]);
+                    hi = max(hi, (int)ph[(int64_t)sp * E]);
+                }
+            }
+            s_lo[u][x] = (int16_t)lo;
+            s_hi[u][x] = (int16_t)hi;
+        }
+        __syncthreads();
+        if (live && yl == 0) {
+            for (int u = 0; u < nq; ++u) {
+                const float mn = key_to_float(s_lo[u][x]), mx = key_to_float(s_hi[u][x]);
+                if (count0 + q0 + u == 0) {
+                    mj = mn;
+                    Mj = mx;
+                } else {
+                    mj = __fadd_rn(__fmul_rn(c, mj), __fmul_rn(gamma, mn));
+                    Mj = __fadd_rn(__fmul_rn(c, Mj), __fmul_rn(gamma, mx));
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (live && yl == 0) {
+        m[j] = mj;
+        M[j] = Mj;
+    }
 }
 
 int pick_splits(int64_t n_seq, int64_t S, int E, int sm_count)
@@ -202,7 +232,7 @@ cudaError_t tpq_launch_calibrate(const uint16_t *y, int64_t n_seq, int64_t S, in
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    ema_fold<<<(E + 255) / 256, 256, 0, st>>>(part_lo, part_hi, n_seq, n_split, E, m, M, count0, gamma);
+    ema_fold<<<(E + EF_X - 1) / EF_X, EF_X * EF_Y, 0, st>>>(part_lo, part_hi, n_seq, n_split, E, m, M, count0, gamma);
     ++*launches;
     return cudaGetLastError();
 }

@@ -514,6 +514,24 @@ def test_calibration_prefill_sized_sequences():
         t.close()
 
 
+def test_calibration_many_sequences_per_call():
+    """More sequences in one call than the fold kernel holds side by side (several passes, a ragged last one),
+    with E not a multiple of its feature tile, in one call and split over calls with a non-zero count."""
+    for (n_seq, S, E) in [(150, 9, 200), (65, 130, 264), (64, 3, 40)]:
+        w = synth.Workload("c", 1, 1, E, 0.7, 3, 20.0, 200.0, n_seq, S, 4100 + E)
+        cal = synth.calibration_np(w, 0)
+        a = binding.Tpq(1, E)
+        m, M = gu.calibrate_both(a, [cal])
+        gm, gM = a.get_ranges(with_R=False)
+        assert gu.bits_equal(gm, m) and gu.bits_equal(gM, M)
+        b = binding.Tpq(1, E)
+        gu.calibrate_both(b, [cal], chunks=[1, n_seq - 2, 1])
+        hm, hM = b.get_ranges(with_R=False)
+        assert gu.bits_equal(hm, m) and gu.bits_equal(hM, M)
+        a.close()
+        b.close()
+
+
 def test_signed_zero_and_infinity_extremes():
     t = binding.Tpq(1, 8)
     y = np.zeros((1, 4, 8), np.uint16)
