@@ -360,6 +360,39 @@ def main():
         t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh, bias_ptr=bias_dev.data_ptr())
 
     db_ms = time_loop(db_only, reps)
+
+    # the fused exchange (Section 5) on one GPU: one shard's payload stored into 1 and into N local receive slots
+    # and its arrival words published; then the bounded wait ahead of the reduction (words already set)
+    words = torch.zeros(2 * N, dtype=torch.int32, device=dev)
+    push_epoch = [0]
+
+    def push_fn(n_dst):
+        arrs = []
+        for b in range(args.sets):
+            ys, pls, _, _, _ = sets[b]
+            arrs.append(((ctypes.c_void_p * n_dst)(*[pls[d].data_ptr() for d in range(n_dst)]),
+                         (ctypes.c_void_p * n_dst)(*[words.data_ptr() + 4 * d for d in range(n_dst)])))
+
+        def fn(b):
+            ys, _, _, _, _ = sets[b % args.sets]
+            da, aa = arrs[b % args.sets]
+            for i in range(N):      # N launches per pass, like the single-shard loop above
+                push_epoch[0] += 1
+                t.quantize_pack_push(i, ys[i].data_ptr(), T, da, aa, P, push_epoch[0], stream=sh)
+        return fn
+
+    push_max = min(N, 16)
+    p1_ms = time_loop(push_fn(1), reps) / N
+    pn_ms = time_loop(push_fn(push_max), reps) / N
+    words.fill_(1)
+    torch.cuda.synchronize()
+
+    def wd_only(b):
+        _, _, out, _, parr = sets[b % args.sets]
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh, arrived_ptr=words.data_ptr(), epoch=1,
+                         timeout_ns=50_000_000)
+
+    wd_ms = time_loop(wd_only, reps)
     # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
     # what the launch path costs, relevant for the decode-sized workloads
     graph_ms = None
@@ -463,6 +496,9 @@ def main():
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
         "step_cuda_graph_replay_ms": graph_ms,
         "dequant_reduce_bias_ms_per_launch": db_ms,
+        "exchange_one_gpu": {"quantize_pack_push_1_dst_ms": p1_ms, f"quantize_pack_push_{push_max}_dst_ms": pn_ms,
+                             "dequant_reduce_arrivals_ms": wd_ms,
+                             "note": "destinations are local buffers; across GPUs the stores cross NVLink"},
         "payload_bytes_per_shard": int(comm.payload_bytes),
         "comm_bytes_per_rank": {"quantized_allgather": int(comm.quantized_allgather_send),
                                 "bf16_allgather": int(comm.bf16_allgather_send),

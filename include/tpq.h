@@ -228,6 +228,49 @@ tpq_status tpq_dequant_reduce_bias(tpq_ctx *ctx, const void *const *payloads_dev
                                    void *out_dev, tpq_out_dtype out_dtype, int64_t out_row_stride,
                                    const float *bias_dev, void *stream);
 
+/* ------------------------------------------------- exchange (Section 5) */
+
+/* Section 5 describes the system-level form of the method: the payloads are all-gathered and every
+ * device then reduces locally.  These two calls are that exchange without a collective library: the
+ * quantiser stores its payload straight into every destination (its own receive slot and, through
+ * peer-mapped pointers over NVLink, the slot it owns in each peer's receive buffer), and the reducing
+ * side waits, with a limit, for the N arrival words in its own memory.
+ *
+ * tpq_quantize_pack_push: C^(i) of tpq_quantize_pack for one shard, the payload written to n_dst
+ * destinations (byte-identical in each), then `epoch` written to the n_dst arrival words with release
+ * semantics at system scope once every byte of every destination has been stored.
+ *   dst_dev_host     : HOST array of n_dst DEVICE pointers (local or peer-mapped), each of dst_capacity
+ *                      >= tpq_payload_bytes(ctx, T) bytes, 16-byte aligned
+ *   arrived_dev_host : HOST array of n_dst DEVICE pointers to 32-bit words, 4-byte aligned, one per
+ *                      destination, in the same memory as the destination
+ *   n_dst            : 1 .. 16
+ *   epoch            : the step's tag; a receiver waits for exactly this value, so consecutive steps
+ *                      on the same slot use different tags
+ * T must be >= 1.  Enqueues on cuda_stream.  The caller owns the slot discipline (a slot is not
+ * pushed again before its reader has finished: two alternating slot sets suffice when every step
+ * waits for all N arrivals).  Errors: BAD_STATE, INVALID_ARG, ALIGN, SIZE, CUDA. */
+tpq_status tpq_quantize_pack_push(tpq_ctx *ctx, int shard, const void *y_bf16_dev, int64_t T, int64_t row_stride_elems,
+                                  void *const *dst_dev_host, uint32_t *const *arrived_dev_host, int n_dst,
+                                  size_t dst_capacity, uint32_t epoch, void *cuda_stream);
+
+/* Enqueue a wait, on cuda_stream, until the n arrival words at arrived_dev (DEVICE pointer, this GPU's
+ * memory, 4-byte aligned) all equal `epoch`; work enqueued behind it on the stream (tpq_dequant_reduce)
+ * then reads complete payloads.  The wait gives up after timeout_ns (0: one second; at most 5 s): the
+ * context's device status becomes TPQ_ERR_TIMEOUT (tpq_device_status), the kernel returns, the stream
+ * continues and whatever is reduced afterwards is unspecified.  n: 1 .. 1024.
+ * Errors: INVALID_ARG, ALIGN, CUDA. */
+tpq_status tpq_wait_arrivals(tpq_ctx *ctx, const uint32_t *arrived_dev, int n, uint32_t epoch, uint64_t timeout_ns,
+                             void *cuda_stream);
+
+/* tpq_dequant_reduce (with the bias of tpq_dequant_reduce_bias when bias_dev is not NULL) whose kernels wait
+ * themselves, in their prologue and with the limit of tpq_wait_arrivals, for the N arrival words at
+ * arrived_dev (word i beside payload i) before they read any payload: the wait costs no launch of its own.
+ * Errors as tpq_dequant_reduce and tpq_wait_arrivals; expiry is reported through tpq_device_status. */
+tpq_status tpq_dequant_reduce_arrivals(tpq_ctx *ctx, const void *const *payloads_dev_host, int n_payloads, int64_t T,
+                                       void *out_dev, tpq_out_dtype out_dtype, int64_t out_row_stride,
+                                       const float *bias_dev, const uint32_t *arrived_dev, uint32_t epoch,
+                                       uint64_t timeout_ns, void *cuda_stream);
+
 /* ------------------------------------------------- checkpoint and status */
 
 /* Serialise / restore the whole static state (N, E, bits, gamma, counts, m, M,

@@ -55,6 +55,11 @@ SIGNATURES = {
     "tpq_dequant_reduce": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p]),
     "tpq_dequant_reduce_bias": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p,
                                         c_void_p]),
+    "tpq_quantize_pack_push": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, POINTER(c_void_p), POINTER(c_void_p),
+                                       c_int, c_size_t, ctypes.c_uint32, c_void_p]),
+    "tpq_dequant_reduce_arrivals": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p,
+                                            c_void_p, ctypes.c_uint32, ctypes.c_uint64, c_void_p]),
+    "tpq_wait_arrivals": (c_int, [c_void_p, c_void_p, c_int, ctypes.c_uint32, ctypes.c_uint64, c_void_p]),
     "tpq_get_state": (c_int, [c_void_p, c_void_p, POINTER(c_size_t)]),
     "tpq_set_state": (c_int, [c_void_p, c_void_p, c_size_t]),
     "tpq_device_status": (c_int, [c_void_p]),
@@ -205,14 +210,30 @@ class Tpq:
                                                   payload_capacity, stream))
 
     def dequant_reduce(self, payload_ptrs, T: int, out_ptr: int, out_dtype: int = TPQ_OUT_BF16,
-                       out_row_stride: int | None = None, stream: int = 0, bias_ptr: int | None = None):
+                       out_row_stride: int | None = None, stream: int = 0, bias_ptr: int | None = None,
+                       arrived_ptr: int | None = None, epoch: int = 0, timeout_ns: int = 0):
         arr = payload_ptrs if isinstance(payload_ptrs, ctypes.Array) else (c_void_p * len(payload_ptrs))(*payload_ptrs)
         stride = self.E if out_row_stride is None else out_row_stride
-        if bias_ptr is None:
+        if arrived_ptr is not None:
+            self._check(lib().tpq_dequant_reduce_arrivals(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride,
+                                                          bias_ptr, arrived_ptr, epoch & 0xFFFFFFFF, timeout_ns, stream))
+        elif bias_ptr is None:
             self._check(lib().tpq_dequant_reduce(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride, stream))
         else:
             self._check(lib().tpq_dequant_reduce_bias(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride,
                                                       bias_ptr, stream))
+
+    def quantize_pack_push(self, shard: int, y_ptr: int, T: int, dst_ptrs, arrived_ptrs, dst_capacity: int, epoch: int,
+                           row_stride: int | None = None, stream: int = 0):
+        n = len(dst_ptrs)
+        assert len(arrived_ptrs) == n
+        da = dst_ptrs if isinstance(dst_ptrs, ctypes.Array) else (c_void_p * n)(*dst_ptrs)
+        aa = arrived_ptrs if isinstance(arrived_ptrs, ctypes.Array) else (c_void_p * n)(*arrived_ptrs)
+        self._check(lib().tpq_quantize_pack_push(self._h, shard, y_ptr, T, self.E if row_stride is None else row_stride,
+                                                 da, aa, n, dst_capacity, epoch & 0xFFFFFFFF, stream))
+
+    def wait_arrivals(self, arrived_ptr: int, n: int, epoch: int, timeout_ns: int = 0, stream: int = 0):
+        self._check(lib().tpq_wait_arrivals(self._h, arrived_ptr, n, epoch & 0xFFFFFFFF, timeout_ns, stream))
 
     def get_state(self) -> bytes:
         n = c_size_t(0)

@@ -24,6 +24,7 @@ struct DQParams {
     void *out;
     int64_t out_stride;
     const float *bias;     // [E] added after the sum (Section 2: f(x) = sum_i f_i(x_i) + b), or NULL
+    tpq_arrivals arr;      // arrival words to wait for before the first payload read (words == NULL: none)
 };
 
 // ----------------------------------------------------------------------------------------------
@@ -32,6 +33,10 @@ struct DQParams {
 template <bool FP32OUT>
 __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
 {
+    if (p.arr.words) {
+        tpq_block_wait_arrivals(p.arr);
+        __syncthreads();
+    }
     const int64_t total = p.T * (int64_t)p.E;
     const int64_t L = p.E - p.k;
     for (int64_t a = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; a < total; a += (int64_t)gridDim.x * blockDim.x) {
@@ -385,6 +390,10 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
     };
     tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
+    if (pp.q.arr.words) {
+        tpq_block_wait_arrivals(pp.q.arr);
+        __syncthreads();
+    }
 #pragma unroll
     for (int s = 0; s < DP_STAGES - 1; ++s) issue();
 
@@ -670,7 +679,10 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
         }
         const int g = panel * CG + cg;
         const bool live = tid < DT_MAIN && g < L8;
-        if (f == f0) tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
+        if (f == f0) {
+            tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
+            tpq_block_wait_arrivals(tp.d.q.arr);
+        }
         __syncthreads();
         if (f == f0) tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
@@ -913,6 +925,7 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
     }
     tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
+    tpq_block_wait_arrivals(p.arr);
     __syncthreads();
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
@@ -1144,6 +1157,7 @@ void fill_params(DQParams &p, const tpq_ctx *c, const void *const *payloads, int
     p.s_k = c->t.s_k; p.pos = c->t.pos; p.grp = c->t.grp;
     p.out = out; p.out_stride = out_stride;
     p.bias = c->call_bias;
+    p.arr = c->call_arr;
 }
 
 }  // namespace

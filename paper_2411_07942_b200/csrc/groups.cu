@@ -159,6 +159,7 @@ struct DGParams {
     const int32_t *lp_idx, *hp_idx;
     void *out;
     const float *bias;  // [E] added after the sum, or NULL
+    tpq_arrivals arr;   // arrival words to wait for before the first payload read (words == NULL: none)
 };
 
 template <bool FP32OUT>
@@ -173,6 +174,10 @@ __device__ __forceinline__ void gk_store(void *out, int64_t off, float v)
 template <int B, bool FP32OUT>
 __global__ void __launch_bounds__(GK_THREADS) dequant_groups(const DGParams p)
 {
+    if (p.arr.words) {
+        tpq_block_wait_arrivals(p.arr);
+        __syncthreads();
+    }
     constexpr int R = 2;
     const int E = p.E, k = p.k, L8 = (E - k) >> 3, k8 = k >> 3, GW = L8 + k8;
     const int64_t n_rb = (p.T + R - 1) / R;
@@ -362,6 +367,7 @@ cudaError_t tpq_launch_dequant_groups(const tpq_ctx *c, const void *const *paylo
     p.s_slot = c->t.s_slot; p.grp = c->t.grp; p.lp_idx = c->t.lp_idx; p.hp_idx = c->t.hp_idx;
     p.out = out;
     p.bias = c->call_bias;
+    p.arr = c->call_arr;
     const int64_t units = ((T + 1) / 2) * (int64_t)((E - k) / 8 + k / 8);
     const unsigned grid = gk_grid(units, c->sm_count);
     switch (c->bits) {

@@ -98,6 +98,11 @@ struct QPParams {
     const int32_t *hp_idx;  // [k]
     int64_t lp_words;       // words of the code section, padding included
     int *status;
+    // push mode (one shard, n_dst copies of its payload: payload[0 .. n_dst), possibly in peers' memory)
+    int n_dst;
+    uint32_t epoch;                     // value written to every arrival word once the payload is complete
+    uint32_t *arrived[QP_MAX_BATCH];    // arrival word beside destination d (same memory as payload[d])
+    unsigned int *done;                 // blocks that have finished their stores (returns to 0)
 #ifdef TPQ_TRACE
     long long *trace;
 #endif
@@ -199,7 +204,9 @@ __device__ __forceinline__ long long tpq_now()
 #define TPQ_MARK(slot) do { } while (0)
 #endif
 
-template <int GPT, int G, int TB>  // TB: upper bound of the block size (register budget)
+// PUSH: every payload store goes to n_dst destinations (plain stores; a destination may be a peer's
+// memory), and the block that finishes last publishes the arrival words.
+template <int GPT, int G, int TB, bool PUSH>  // TB: upper bound of the block size (register budget)
 __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -390,8 +397,16 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                     }
                 }
                 if (live) {
+                    if constexpr (PUSH) {
+                        for (int d = 0; d < p.n_dst; ++d) {
+                            uint32_t *const o = reinterpret_cast<uint32_t *>(p.payload[d]) + t0 * L8 + g;
 #pragma unroll
-                    for (int r = 0; r < G; ++r) lp_out[(t0 + r) * L8 + g] = word[r];
+                            for (int r = 0; r < G; ++r) o[r * L8] = word[r];
+                        }
+                    } else {
+#pragma unroll
+                        for (int r = 0; r < G; ++r) lp_out[(t0 + r) * L8 + g] = word[r];
+                    }
                 }
             } else if (live) {
                 // ragged last stage, or a warp on the serial path: every hole patched by its owner
@@ -406,14 +421,26 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                         const uint32_t q = quant_bits(x, __ldg(inv_s + f)) & 0xFu;
                         word = (word & ~(0xFu << (4 * n))) | (q << (4 * n));
                     }
-                    lp_out[(t0 + r) * L8 + g] = word;
+                    if constexpr (PUSH) {
+                        for (int d = 0; d < p.n_dst; ++d)
+                            reinterpret_cast<uint32_t *>(p.payload[d])[(t0 + r) * L8 + g] = word;
+                    } else {
+                        lp_out[(t0 + r) * L8 + g] = word;
+                    }
                 }
             }
             (void)nh;
         }
         for (int h = tid; h < k; h += NT) {
             const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
-            for (int r = 0; r < rows; ++r) hp_out[(t0 + r) * k + h] = stage16[r * E + j];
+            if constexpr (PUSH) {
+                for (int d = 0; d < p.n_dst; ++d) {
+                    uint16_t *const o = reinterpret_cast<uint16_t *>(p.payload[d] + p.lp_bytes) + t0 * k + h;
+                    for (int r = 0; r < rows; ++r) o[r * k] = stage16[r * E + j];
+                }
+            } else {
+                for (int r = 0; r < rows; ++r) hp_out[(t0 + r) * k + h] = stage16[r * E + j];
+            }
         }
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
@@ -426,7 +453,61 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     // zero padding of the code section (at most 3 words), by the block that owned the last rows
     if ((p.ngroups - 1) % p.cps == bx) {
         const int64_t valid = p.T * L8;
-        for (int64_t w = valid + tid; w < p.lp_words; w += NT) lp_out[w] = 0u;
+        for (int64_t w = valid + tid; w < p.lp_words; w += NT) {
+            if constexpr (PUSH) {
+                for (int d = 0; d < p.n_dst; ++d) reinterpret_cast<uint32_t *>(p.payload[d])[w] = 0u;
+            } else {
+                lp_out[w] = 0u;
+            }
+        }
+    }
+    if constexpr (PUSH) {
+        // Publication.  The block's consumer threads meet (their stores happen-before the fence below), one
+        // thread orders them before its count at system scope; the block that counts last has thereby
+        // observed every other block's stores and releases the arrival words to the destinations' owners.
+        asm volatile("bar.sync 2, %0;" ::"r"(NT) : "memory");
+        if (tid == 0) {
+            __threadfence_system();
+            const unsigned int prev = atomicAdd(p.done, 1u);
+            if (prev == gridDim.x - 1) {
+                *p.done = 0u;  // the next launch in the stream starts from zero
+                // one fence (acquire side of the counts above, release side of the words below), then the
+                // words as relaxed system-scope stores: together a release of everything observed so far
+                __threadfence_system();
+                for (int d = 0; d < p.n_dst; ++d)
+                    asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p.arrived[d]), "r"(p.epoch) : "memory");
+            }
+        }
+    }
+}
+
+// Arrival words published on their own (after payload copies made by the copy engine in stream order).
+__global__ void publish_arrivals(QPParams p)
+{
+    const int d = threadIdx.x;
+    if (d < p.n_dst) {
+        __threadfence_system();
+        asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p.arrived[d]), "r"(p.epoch) : "memory");
+    }
+}
+
+// Bounded wait for n arrival words (this GPU's own memory, written by the pushing devices) to reach `epoch`.
+__global__ void wait_arrivals(const uint32_t *arrived, int n, uint32_t epoch, unsigned long long timeout_ns, int *status)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (;;) {
+        uint32_t v;
+        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(arrived + i) : "memory");
+        if (v == epoch) return;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+        if (t1 - t0 > timeout_ns) {
+            atomicExch(status, (int)TPQ_ERR_TIMEOUT);
+            return;
+        }
+        __nanosleep(200);
     }
 }
 
@@ -470,13 +551,22 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
     return tpq_launch_quantize_tiled_batch(c, shard, 1, ys, T, stride, pls, st, launches);
 }
 
-cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
-                                            int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches)
+namespace {
+
+struct PushArgs {
+    int n_dst;
+    void *const *dst;
+    uint32_t *const *arrived;
+    uint32_t epoch;
+};
+
+cudaError_t launch_tiled(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T, int64_t stride,
+                         void *const *payloads, const PushArgs *push, cudaStream_t st, int64_t *launches)
 {
     if (n > QP_MAX_BATCH) {  // more shards than one launch carries: several launches
         for (int b = 0; b < n; b += QP_MAX_BATCH) {
             const int nb = n - b < QP_MAX_BATCH ? n - b : QP_MAX_BATCH;
-            cudaError_t e = tpq_launch_quantize_tiled_batch(c, shard0 + b, nb, ys + b, T, stride, payloads + b, st, launches);
+            cudaError_t e = launch_tiled(c, shard0 + b, nb, ys + b, T, stride, payloads + b, nullptr, st, launches);
             if (e != cudaSuccess) return e;
         }
         return cudaSuccess;
@@ -505,6 +595,15 @@ cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n,
         p.y[b] = static_cast<const uint16_t *>(ys[b]);
         p.payload[b] = static_cast<uint8_t *>(payloads[b]);
     }
+    p.n_dst = 0; p.epoch = 0; p.done = c->t.push_done;
+    if (push) {  // one shard, n_dst destinations
+        p.n_dst = push->n_dst;
+        p.epoch = push->epoch;
+        for (int d = 0; d < push->n_dst; ++d) {
+            p.payload[d] = static_cast<uint8_t *>(push->dst[d]);
+            p.arrived[d] = push->arrived[d];
+        }
+    }
     p.cps = cps; p.lp_bytes = lpb;
     p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
     p.inv_s = c->t.inv_s + (size_t)shard0 * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
@@ -517,9 +616,9 @@ cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n,
     cudaError_t e = cudaSuccess;
 #define TPQ_QP_LAUNCH(GPT, GG, TB)                                                                                   \
     do {                                                                                                             \
-        e = cudaFuncSetAttribute(quantize_tiled<GPT, GG, TB>, cudaFuncAttributeMaxDynamicSharedMemorySize,           \
-                                 (int)smem);                                                                         \
-        if (e == cudaSuccess) e = tpq_launch_pdl(quantize_tiled<GPT, GG, TB>, dim3((unsigned)grid), dim3(nt + 32), smem, st, p); \
+        auto kern = push ? quantize_tiled<GPT, GG, TB, true> : quantize_tiled<GPT, GG, TB, false>;                   \
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);                      \
+        if (e == cudaSuccess) e = tpq_launch_pdl(kern, dim3((unsigned)grid), dim3(nt + 32), smem, st, p);            \
     } while (0)
 #define TPQ_QP_LAUNCH_G(GPT, TB)                          \
     do {                                                  \
@@ -545,6 +644,46 @@ cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n,
 #undef TPQ_QP_LAUNCH_G
 #undef TPQ_QP_LAUNCH
     if (e != cudaSuccess) return e;
+    ++*launches;
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
+                                            int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches)
+{
+    return launch_tiled(c, shard0, n, ys, T, stride, payloads, nullptr, st, launches);
+}
+
+int tpq_push_max_dst() { return QP_MAX_BATCH; }
+
+cudaError_t tpq_launch_quantize_tiled_push(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
+                                           void *const *dst, uint32_t *const *arrived, int n_dst, uint32_t epoch,
+                                           cudaStream_t st, int64_t *launches)
+{
+    const void *ys[1] = {y};
+    void *pls[1] = {dst[0]};
+    const PushArgs push = {n_dst, dst, arrived, epoch};
+    return launch_tiled(c, shard, 1, ys, T, stride, pls, &push, st, launches);
+}
+
+cudaError_t tpq_launch_publish_arrivals(uint32_t *const *arrived, int n_dst, uint32_t epoch, cudaStream_t st,
+                                        int64_t *launches)
+{
+    QPParams p = {};
+    p.n_dst = n_dst;
+    p.epoch = epoch;
+    for (int d = 0; d < n_dst; ++d) p.arrived[d] = arrived[d];
+    publish_arrivals<<<1, 32, 0, st>>>(p);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t tpq_launch_wait_arrivals(const tpq_ctx *c, const uint32_t *arrived, int n, uint32_t epoch,
+                                     unsigned long long timeout_ns, cudaStream_t st, int64_t *launches)
+{
+    wait_arrivals<<<(n + 63) / 64, 64, 0, st>>>(arrived, n, epoch, timeout_ns, c->t.status);
     ++*launches;
     return cudaGetLastError();
 }

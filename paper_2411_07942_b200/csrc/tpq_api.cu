@@ -46,7 +46,7 @@ void free_tables(tpq_tables &t)
 {
     cudaFree(t.m); cudaFree(t.M); cudaFree(t.R); cudaFree(t.Rbar); cudaFree(t.s); cudaFree(t.inv_s);
     cudaFree(t.s_k); cudaFree(t.s_slot); cudaFree(t.flag); cudaFree(t.hpre); cudaFree(t.pos); cudaFree(t.hp_idx);
-    cudaFree(t.lp_idx); cudaFree(t.hole); cudaFree(t.filler); cudaFree(t.grp); cudaFree(t.status);
+    cudaFree(t.lp_idx); cudaFree(t.hole); cudaFree(t.filler); cudaFree(t.grp); cudaFree(t.status); cudaFree(t.push_done);
     memset(&t, 0, sizeof t);
 }
 
@@ -139,9 +139,11 @@ tpq_status tpq_create(tpq_ctx **out, int n_shards, int n_features, int bits, flo
     if (e == cudaSuccess) e = dalloc(&t.filler, E);
     if (e == cudaSuccess) e = dalloc(&t.grp, (E + 7) / 8);
     if (e == cudaSuccess) e = dalloc(&t.status, 1);
+    if (e == cudaSuccess) e = dalloc(&t.push_done, 1);
     if (e == cudaSuccess) e = cudaMemset(t.m, 0, NE * sizeof(float));
     if (e == cudaSuccess) e = cudaMemset(t.M, 0, NE * sizeof(float));
     if (e == cudaSuccess) e = cudaMemset(t.status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(t.push_done, 0, sizeof(unsigned int));
     if (e != cudaSuccess) {
         tpq_status st = (e == cudaErrorMemoryAllocation) ? TPQ_ERR_NOMEM : TPQ_ERR_CUDA;
         free_tables(t);
@@ -428,6 +430,65 @@ tpq_status tpq_quantize_pack_batch(tpq_ctx *c, int first_shard, int n, const voi
     return TPQ_OK;
 }
 
+// Section 5 (system level: all-gather, then a local reduction): the exchange fused into the quantiser.
+tpq_status tpq_quantize_pack_push(tpq_ctx *c, int shard, const void *y, int64_t T, int64_t stride, void *const *dst,
+                                  uint32_t *const *arrived, int n_dst, size_t cap, uint32_t epoch, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set: call tpq_select_features or tpq_set_features");
+    if (shard < 0 || shard >= c->N) return fail(c, TPQ_ERR_INVALID_ARG, "shard %d out of range [0, %d)", shard, c->N);
+    if (n_dst < 1 || n_dst > tpq_push_max_dst())
+        return fail(c, TPQ_ERR_INVALID_ARG, "n_dst %d out of range [1, %d]", n_dst, tpq_push_max_dst());
+    if (T < 1) return fail(c, TPQ_ERR_INVALID_ARG, "T < 1 (an empty step has nothing to publish)");
+    if (!y || !dst || !arrived) return fail(c, TPQ_ERR_INVALID_ARG, "NULL pointer");
+    if (stride < c->E) return fail(c, TPQ_ERR_INVALID_ARG, "row stride %lld < E", (long long)stride);
+    if (!aligned16(y)) return fail(c, TPQ_ERR_ALIGN, "y must be 16-byte aligned");
+    if (cap < tpq_payload_bytes(c, T))
+        return fail(c, TPQ_ERR_SIZE, "destination capacity %zu < %zu", cap, tpq_payload_bytes(c, T));
+    for (int d = 0; d < n_dst; ++d) {
+        if (!dst[d] || !arrived[d]) return fail(c, TPQ_ERR_INVALID_ARG, "NULL destination %d", d);
+        if (!aligned16(dst[d])) return fail(c, TPQ_ERR_ALIGN, "destination %d must be 16-byte aligned", d);
+        if (reinterpret_cast<uintptr_t>(arrived[d]) & 3u)
+            return fail(c, TPQ_ERR_ALIGN, "arrival word %d must be 4-byte aligned", d);
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (c->kernel_path != 1 && tpq_quantize_tiled_ok(c, T, stride)) {
+        e = tpq_launch_quantize_tiled_push(c, shard, static_cast<const uint16_t *>(y), T, stride, dst, arrived, n_dst, epoch,
+                                           st, &c->launches);
+        if (e != cudaSuccess) return cuda_fail(c, e, "quantize_pack_push kernel");
+        return TPQ_OK;
+    }
+    // other shapes and code widths: quantise into the first destination, copy it to the others in stream
+    // order, then publish the arrival words
+    void *first = dst[0];
+    if (tpq_groups_ok(c, T, stride) && c->kernel_path != 1)
+        e = tpq_launch_quantize_groups(c, shard, 1, &y, T, stride, &first, st, &c->launches);
+    else
+        e = tpq_launch_quantize_generic(c, shard, static_cast<const uint16_t *>(y), T, stride,
+                                        static_cast<uint8_t *>(first), st, &c->launches);
+    const size_t bytes = tpq_payload_bytes(c, T);
+    for (int d = 1; d < n_dst && e == cudaSuccess; ++d)
+        if (dst[d] != first) e = cudaMemcpyAsync(dst[d], first, bytes, cudaMemcpyDefault, st);
+    if (e == cudaSuccess) e = tpq_launch_publish_arrivals(arrived, n_dst, epoch, st, &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e, "quantize_pack_push (copy path)");
+    return TPQ_OK;
+}
+
+tpq_status tpq_wait_arrivals(tpq_ctx *c, const uint32_t *arrived, int n, uint32_t epoch, uint64_t timeout_ns, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (!arrived || n < 1 || n > 1024) return fail(c, TPQ_ERR_INVALID_ARG, "arrival words: NULL or n = %d outside [1, 1024]", n);
+    if (reinterpret_cast<uintptr_t>(arrived) & 3u) return fail(c, TPQ_ERR_ALIGN, "arrival words must be 4-byte aligned");
+    if (timeout_ns == 0) timeout_ns = 1000000000ull;  // one second
+    if (timeout_ns > 5000000000ull) return fail(c, TPQ_ERR_INVALID_ARG, "timeout above 5 s");
+    cudaError_t e = tpq_launch_wait_arrivals(c, arrived, n, epoch, timeout_ns, static_cast<cudaStream_t>(stream), &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e, "wait_arrivals kernel");
+    return TPQ_OK;
+}
+
 static tpq_status dequant_reduce_impl(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
                                       tpq_out_dtype dt, int64_t out_stride, void *stream);
 
@@ -436,6 +497,7 @@ tpq_status tpq_dequant_reduce(tpq_ctx *c, const void *const *payloads, int n_pay
 {
     if (!c) return TPQ_ERR_INVALID_ARG;
     c->call_bias = nullptr;
+    c->call_arr = tpq_arrivals{};
     return dequant_reduce_impl(c, payloads, n_payloads, T, out, dt, out_stride, stream);
 }
 
@@ -447,8 +509,28 @@ tpq_status tpq_dequant_reduce_bias(tpq_ctx *c, const void *const *payloads, int 
     if (!bias) return fail(c, TPQ_ERR_INVALID_ARG, "bias is NULL (use tpq_dequant_reduce)");
     if (!aligned16(bias)) return fail(c, TPQ_ERR_ALIGN, "bias must be 16-byte aligned");
     c->call_bias = bias;
+    c->call_arr = tpq_arrivals{};
     const tpq_status st = dequant_reduce_impl(c, payloads, n_payloads, T, out, dt, out_stride, stream);
     c->call_bias = nullptr;
+    return st;
+}
+
+tpq_status tpq_dequant_reduce_arrivals(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
+                                       tpq_out_dtype dt, int64_t out_stride, const float *bias, const uint32_t *arrived,
+                                       uint32_t epoch, uint64_t timeout_ns, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (bias && !aligned16(bias)) return fail(c, TPQ_ERR_ALIGN, "bias must be 16-byte aligned");
+    if (!arrived) return fail(c, TPQ_ERR_INVALID_ARG, "arrival words are NULL (use tpq_dequant_reduce)");
+    if (reinterpret_cast<uintptr_t>(arrived) & 3u) return fail(c, TPQ_ERR_ALIGN, "arrival words must be 4-byte aligned");
+    if (timeout_ns == 0) timeout_ns = 1000000000ull;  // one second
+    if (timeout_ns > 5000000000ull) return fail(c, TPQ_ERR_INVALID_ARG, "timeout above 5 s");
+    c->call_bias = bias;
+    c->call_arr = tpq_arrivals{arrived, epoch, c->N, timeout_ns, c->t.status};
+    const tpq_status st = dequant_reduce_impl(c, payloads, n_payloads, T, out, dt, out_stride, stream);
+    c->call_bias = nullptr;
+    c->call_arr = tpq_arrivals{};
     return st;
 }
 

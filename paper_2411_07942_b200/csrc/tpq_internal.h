@@ -25,6 +25,17 @@ struct tpq_tables {
     int32_t *filler;     // [E]    first n_holes entries: unselected features at or above L, ascending
     uint32_t *grp;       // [ceil(E/8)] per group of 8 features: (selected before the group << 8) | 8-bit mask
     int *status;         // device status word (0 = ok)
+    unsigned int *push_done;  // blocks of a pushing quantiser that have finished (0 between launches)
+};
+
+// Arrival words a reduction waits for before it reads the payloads (the fused exchange): n words in this
+// GPU's memory, each written with `epoch` by the device that pushed the matching payload.
+struct tpq_arrivals {
+    const uint32_t *words;
+    uint32_t epoch;
+    int n;
+    unsigned long long timeout_ns;
+    int *status;
 };
 
 struct tpq_ctx {
@@ -44,6 +55,7 @@ struct tpq_ctx {
     int64_t launches;
     void *dq_cache;     // tensor maps of recently used payloads (dequant.cu)
     const float *call_bias;  // bias of the tpq_dequant_reduce_bias call in progress (NULL otherwise)
+    tpq_arrivals call_arr;   // arrival words the reduction in progress waits for (words == NULL: none)
     char err[512];
 };
 
@@ -88,6 +100,18 @@ cudaError_t tpq_launch_quantize_tiled(const tpq_ctx *c, int shard, const uint16_
 cudaError_t tpq_launch_quantize_tiled_batch(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
                                             int64_t stride, void *const *payloads, cudaStream_t st, int64_t *launches);
 
+// Push mode of the tiled quantiser: every payload store goes to n_dst destinations and the last block to
+// finish writes `epoch` to the n_dst arrival words (release, system scope).  n_dst <= tpq_push_max_dst().
+int tpq_push_max_dst();
+cudaError_t tpq_launch_quantize_tiled_push(const tpq_ctx *c, int shard, const uint16_t *y, int64_t T, int64_t stride,
+                                           void *const *dst, uint32_t *const *arrived, int n_dst, uint32_t epoch,
+                                           cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_publish_arrivals(uint32_t *const *arrived, int n_dst, uint32_t epoch, cudaStream_t st,
+                                        int64_t *launches);
+// Bounded wait until n arrival words equal `epoch`; on expiry the context's device status becomes TPQ_ERR_TIMEOUT.
+cudaError_t tpq_launch_wait_arrivals(const tpq_ctx *c, const uint32_t *arrived, int n, uint32_t epoch,
+                                     unsigned long long timeout_ns, cudaStream_t st, int64_t *launches);
+
 // Code widths other than 4 bits on shapes that are multiples of 8 (groups.cu).
 bool tpq_groups_ok(const tpq_ctx *c, int64_t T, int64_t stride);
 cudaError_t tpq_launch_quantize_groups(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
@@ -110,6 +134,29 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
 #ifdef __CUDACC__
 __device__ __forceinline__ void tpq_grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void tpq_grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Bounded wait of a block for the arrival words (every block waits by itself; call it ahead of a
+// __syncthreads() that precedes the block's first payload read).  On expiry the status word becomes
+// TPQ_ERR_TIMEOUT and the block carries on: its output is then unspecified.
+__device__ __forceinline__ void tpq_block_wait_arrivals(const tpq_arrivals &a)
+{
+    if (a.words == nullptr) return;
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+        unsigned long long t0, t1;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+        for (;;) {
+            uint32_t v;
+            asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(a.words + i) : "memory");
+            if (v == a.epoch) break;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+            if (t1 - t0 > a.timeout_ns) {
+                atomicExch(a.status, (int)TPQ_ERR_TIMEOUT);
+                break;
+            }
+            __nanosleep(100);
+        }
+    }
+}
 
 template <typename... KArgs, typename... Args>
 cudaError_t tpq_launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
