@@ -15,6 +15,7 @@ NVCC_FLAGS = [
     "-std=c++17", "-O3", "-lineinfo",
     "-gencode", "arch=compute_100a,code=sm_100a",
     "-Xcompiler", "-fPIC", "-shared",
+    "--threads", "0",  # the translation units compile side by side
     # IEEE arithmetic everywhere: no fast-math; the kernels use explicit _rn intrinsics
     # wherever the rounding sequence is part of the result.
 ]

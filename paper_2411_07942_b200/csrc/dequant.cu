@@ -326,7 +326,7 @@ __device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *
     }
 }
 
-template <int CG, bool FP32OUT>
+template <int CG, bool FP32OUT, bool HAS_WAIT>
 __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams pp)
 {
     extern __shared__ __align__(128) uint8_t dp_smem[];
@@ -342,6 +342,10 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
     const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
     const int tid = threadIdx.x;
     float4 *const dp_steps = reinterpret_cast<float4 *>(dp_smem);  // [N][2][CG]
+    if constexpr (HAS_WAIT) {  // (first thing, with no load of its own in flight; an instantiation of its own)
+        tpq_block_wait_arrivals(p.arr);
+        __syncthreads();
+    }
     const int panel = blockIdx.x % pp.panels, by = blockIdx.x / pp.panels;
     const int cg = tid & (CG - 1), rs = tid / CG;
     const int g = panel * CG + cg;
@@ -390,10 +394,6 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
     };
     tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
-    if (pp.q.arr.words) {
-        tpq_block_wait_arrivals(pp.q.arr);
-        __syncthreads();
-    }
 #pragma unroll
     for (int s = 0; s < DP_STAGES - 1; ++s) issue();
 
@@ -640,6 +640,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     const int64_t total = (int64_t)pp.panels * pp.n_chunks;
     const int64_t f0 = total * blockIdx.x / gridDim.x, f1 = total * (blockIdx.x + 1) / gridDim.x;
 
+    tpq_block_wait_arrivals(p.arr);  // (first thing, with no load of its own in flight; a barrier follows)
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
@@ -679,10 +680,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
         }
         const int g = panel * CG + cg;
         const bool live = tid < DT_MAIN && g < L8;
-        if (f == f0) {
-            tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
-            tpq_block_wait_arrivals(tp.d.q.arr);
-        }
+        if (f == f0) tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
         __syncthreads();
         if (f == f0) tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
@@ -885,7 +883,7 @@ __device__ __forceinline__ long long tpq_dnow()
 #define TPQ_DMARK(slot) do { } while (0)
 #endif
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
 __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -901,6 +899,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
     uint64_t *empty = full + nstage;
     uint64_t *main_done = empty + nstage;
 
+    // (first thing, with no load of its own in flight: behind the table loads below it would make every
+    // thread wait for them ahead of the barrier that releases the producer; and an instantiation of its
+    // own: even a branch that is never taken costs this prologue a few hundred cycles)
+    if constexpr (HAS_WAIT) tpq_block_wait_arrivals(p.arr);
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
@@ -925,7 +927,6 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
     }
     tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
-    tpq_block_wait_arrivals(p.arr);
     __syncthreads();
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
@@ -1188,14 +1189,21 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
 
 namespace {
 
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+cudaError_t launch_rows_w(const DRParams &pp, int grid, int threads, size_t smem, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(threads), smem, st, pp);
+    return e;
+}
+
 template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
 cudaError_t launch_rows_v(const DRParams &pp, int grid, int threads, size_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS>, dim3(grid), dim3(threads), smem, st, pp);
-    return e;
+    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, true>(pp, grid, threads, smem, st)
+                          : launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, false>(pp, grid, threads, smem, st);
 }
 
 template <int NMAX, int MAXT>
@@ -1257,13 +1265,19 @@ bool panels_plan(const tpq_ctx *c, int64_t T, DPParams &pp)
     return true;
 }
 
+template <int CG, bool FP32OUT, bool HAS_WAIT>
+cudaError_t launch_panels_w(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
+{
+    const size_t smem = dp_smem_bytes(c->N, CG);
+    cudaError_t e = cudaFuncSetAttribute(dequant_panels<CG, FP32OUT, HAS_WAIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    return tpq_launch_pdl(dequant_panels<CG, FP32OUT, HAS_WAIT>, dim3((unsigned)(pp.panels * pp.gy)), dim3(DP_THREADS), smem, st, pp);
+}
+
 template <int CG, bool FP32OUT>
 cudaError_t launch_panels_cg(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
 {
-    const size_t smem = dp_smem_bytes(c->N, CG);
-    cudaError_t e = cudaFuncSetAttribute(dequant_panels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    return tpq_launch_pdl(dequant_panels<CG, FP32OUT>, dim3((unsigned)(pp.panels * pp.gy)), dim3(DP_THREADS), smem, st, pp);
+    return pp.q.arr.words ? launch_panels_w<CG, FP32OUT, true>(c, pp, st) : launch_panels_w<CG, FP32OUT, false>(c, pp, st);
 }
 
 template <bool FP32OUT>

@@ -138,24 +138,33 @@ __device__ __forceinline__ void tpq_grid_dep_launch() { asm volatile("griddepcon
 // Bounded wait of a block for the arrival words (every block waits by itself; call it ahead of a
 // __syncthreads() that precedes the block's first payload read).  On expiry the status word becomes
 // TPQ_ERR_TIMEOUT and the block carries on: its output is then unspecified.
-__device__ __forceinline__ void tpq_block_wait_arrivals(const tpq_arrivals &a)
+// (Out of line on purpose: inlined, the polling loop's atomics and acquire loads cost the kernels' prologues
+// a few hundred cycles even when there is nothing to wait for.)
+static __device__ __noinline__ void tpq_poll_arrivals(const uint32_t *words, uint32_t epoch, int n,
+                                                      unsigned long long timeout_ns, int *status)
 {
-    if (a.words == nullptr) return;
-    for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
         unsigned long long t0, t1;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
         for (;;) {
             uint32_t v;
-            asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(a.words + i) : "memory");
-            if (v == a.epoch) break;
+            asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(words + i) : "memory");
+            if (v == epoch) break;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
-            if (t1 - t0 > a.timeout_ns) {
-                atomicExch(a.status, (int)TPQ_ERR_TIMEOUT);
+            if (t1 - t0 > timeout_ns) {
+                atomicExch(status, (int)TPQ_ERR_TIMEOUT);
                 break;
             }
             __nanosleep(100);
         }
+        // the payloads are read next through bulk asynchronous copies as well as plain loads
+        asm volatile("fence.proxy.async;" ::: "memory");
     }
+}
+
+__device__ __forceinline__ void tpq_block_wait_arrivals(const tpq_arrivals &a)
+{
+    if (a.words != nullptr) tpq_poll_arrivals(a.words, a.epoch, a.n, a.timeout_ns, a.status);
 }
 
 template <typename... KArgs, typename... Args>
