@@ -205,6 +205,17 @@ class COracle:
                                            _ptr(chain, ctypes.c_float) if want_chain32 else None)
         return ref, chain
 
+    def linear_bf16(self, x_bits: np.ndarray, w_bits: np.ndarray) -> np.ndarray:
+        """Section 2: y = bf16(x W^T), x [T][K], w [E][K] BF16 patterns; exact sum, one rounding."""
+        x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+        w = np.ascontiguousarray(w_bits, dtype=np.uint16)
+        T, K = x.shape
+        E, K2 = w.shape
+        assert K == K2
+        y = np.empty((T, E), np.uint16)
+        self.lib.tpqo_linear_bf16(_ptr(x, ctypes.c_uint16), _ptr(w, ctypes.c_uint16), T, K, E, _ptr(y, ctypes.c_uint16))
+        return y
+
     def round_bf16(self, x: np.ndarray) -> np.ndarray:
         x = np.ascontiguousarray(x, dtype=np.float32)
         out = np.empty(x.shape, np.uint16)

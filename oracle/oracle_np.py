@@ -43,6 +43,26 @@ def round_bf16(x: np.ndarray) -> np.ndarray:
     return r.astype(np.uint16)
 
 
+def round_bf16_f64(v: np.ndarray) -> np.ndarray:
+    """float64 -> BF16 bit patterns with ONE rounding (nearest, ties to even); finite inputs within BF16's
+    normal range (the layer outputs this is used for)."""
+    v = np.asarray(v, dtype=np.float64)
+    a = np.abs(v)
+    _, e = np.frexp(a)                              # a = f 2^e, 0.5 <= f < 1
+    q = np.maximum(e - 8, -133)                     # weight of the last of 8 significant bits
+    r = np.rint(np.ldexp(a, -q))                    # exact scaling; rint rounds half to even
+    out = np.copysign(np.ldexp(r, q), v).astype(F32)  # representable: the conversion is exact
+    return (out.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
+
+
+def linear_bf16(x_bits: np.ndarray, w_bits: np.ndarray) -> np.ndarray:
+    """Section 2: y = bf16(x W^T) for x [T][K], w [E][K] given as BF16 patterns.  Products of BF16 values
+    are exact in float64; the library matmul sums them in float64; one rounding to BF16."""
+    x = widen(x_bits).astype(np.float64)
+    w = widen(w_bits).astype(np.float64)
+    return round_bf16_f64(x @ w.T)
+
+
 def _order_key(bits: np.ndarray) -> np.ndarray:
     """Monotone integer key of non-NaN BF16 patterns with -0 below +0."""
     b = np.asarray(bits, dtype=np.uint16).astype(np.int32)

@@ -46,6 +46,7 @@ void tpqo_quantize_pack_b(const uint16_t *y, int64_t T, int64_t E, int64_t strid
                           const float *inv_s, int bits, uint8_t *payload);
 void tpqo_dequant_reduce_b(const uint8_t *const *payloads, int64_t N, int64_t T, int64_t E, const int32_t *hp_idx,
                            int64_t k, const float *s, int bits, double *ref64, float *chain32);
+void tpqo_linear_bf16(const uint16_t *x, const uint16_t *w, int64_t T, int64_t K, int64_t E, uint16_t *y);
 void tpqo_dequant_reduce_bias_b(const uint8_t *const *payloads, int64_t N, int64_t T, int64_t E, const int32_t *hp_idx,
                                 int64_t k, const float *s, int bits, const float *bias, double *ref64, float *chain32);
 
@@ -410,4 +411,41 @@ void tpqo_dequant_reduce_bias_b(const uint8_t *const *payloads, int64_t N, int64
 void tpqo_round_bf16_f32(const float *x, int64_t n, uint16_t *out)
 {
     for (int64_t a = 0; a < n; ++a) out[a] = bf16_round(x[a]);
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * Section 2: the layer ahead of the synchronisation point on device i, f^(i)(x^(i)) = x^(i) W^(i),
+ * x: [T][K], W^T stored as w: [E][K] (one row per output feature), all BF16; the output is BF16 too
+ * (the models of Section 4 run in BF16).  Written as the definition: every product of two BF16 values is
+ * exact in binary64, the K products are summed in binary64 in index order, and the sum is rounded ONCE,
+ * from binary64, to the nearest BF16 (ties to even).  (Reading: the paper does not say how the layer
+ * accumulates; a BF16 layer is specified by its rounded exact result, and an implementation that
+ * accumulates in binary32 may differ from it by one BF16 unit in the last place.)
+ * ---------------------------------------------------------------------------------------------- */
+static uint16_t bf16_round_f64(double v)
+{
+    if (v != v) return 0x7FC0;
+    if (v == 0.0) return signbit(v) ? 0x8000 : 0x0000;
+    const double a = fabs(v);
+    if (a >= 3.3961775292304601e38) return signbit(v) ? 0xFF80 : 0x7F80; /* >= max BF16 + half a unit: infinity */
+    int e;
+    (void)frexp(a, &e);          /* a = f * 2^e, 0.5 <= f < 1: the leading bit has weight 2^(e-1) */
+    int q = e - 1 - 7;           /* weight of the last kept bit (8 significant bits) */
+    if (q < -133) q = -133;      /* subnormal BF16: fixed spacing 2^-133 */
+    const double r = nearbyint(ldexp(a, -q)); /* default rounding mode: nearest, ties to even; the scaling is exact */
+    const float f = (float)ldexp(signbit(v) ? -r : r, q); /* exactly representable in binary32 */
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return (uint16_t)(u >> 16);
+}
+
+void tpqo_linear_bf16(const uint16_t *x, const uint16_t *w, int64_t T, int64_t K, int64_t E, uint16_t *y)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t t = 0; t < T; ++t)
+        for (int64_t j = 0; j < E; ++j) {
+            double acc = 0.0;
+            for (int64_t c = 0; c < K; ++c) acc += (double)bf16_widen(x[t * K + c]) * (double)bf16_widen(w[j * K + c]);
+            y[t * E + j] = bf16_round_f64(acc);
+        }
 }
