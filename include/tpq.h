@@ -228,6 +228,32 @@ tpq_status tpq_dequant_reduce_bias(tpq_ctx *ctx, const void *const *payloads_dev
                                    void *out_dev, tpq_out_dtype out_dtype, int64_t out_row_stride,
                                    const float *bias_dev, void *stream);
 
+/* ------------------------------------------------- the layer ahead of the synchronisation point (Section 2) */
+
+/* Section 2 defines what is synchronised: the output of the last linear layer of an attention or
+ * feed-forward block, f^(i)(x^(i)) = x^(i) W^(i) on device i.  These two calls compute that product on the
+ * tensor cores and compress it in the same kernel, so the [T][E] partial sums are never written:
+ *   payload = C^(i)( bf16( x W^T ) ),  x: [T][K] BF16,  W: [E][K] BF16 (one row per output feature),
+ * FP32 accumulation, one rounding to BF16 (the layer's output type), then exactly tpq_quantize_pack.
+ *
+ * tpq_permute_weight: once per weight matrix and feature set, gather the rows of w_bf16_dev ([E][K],
+ * row-major, 16-byte aligned) into the payload's slot order: row c < E-k is the feature that code slot c
+ * carries, row E-k+h the h-th selected feature.  w_slots_dev: [E][K], 16-byte aligned, not aliasing w.
+ * Errors: BAD_STATE (no feature set), INVALID_ARG, ALIGN, CUDA. */
+tpq_status tpq_permute_weight(tpq_ctx *ctx, const void *w_bf16_dev, int64_t K, void *w_slots_dev, void *cuda_stream);
+
+/* tpq_linear_quantize_pack: the fused layer for one device.
+ *   x_bf16_dev  : [T][K] BF16, row-major, 16-byte aligned; K a multiple of 8
+ *   w_slots_dev : output of tpq_permute_weight for the current feature set
+ *   payload_dev : as tpq_quantize_pack; byte-identical to tpq_quantize_pack applied to bf16(x W^T)
+ *   y_slots_dev : NULL, or [T][E] BF16 (16-byte aligned) that receives the rounded partial sums in slot
+ *                 order (column c as the rows of w_slots_dev) -- for verification or a residual path
+ * Needs 4-bit codes and E, k multiples of 8 (INVALID_ARG otherwise).  Enqueues on cuda_stream; T == 0 is a
+ * no-op.  Errors: BAD_STATE, INVALID_ARG, ALIGN, SIZE, CUDA; TPQ_ERR_TIMEOUT through tpq_device_status. */
+tpq_status tpq_linear_quantize_pack(tpq_ctx *ctx, int shard, const void *x_bf16_dev, const void *w_slots_dev, int64_t T,
+                                    int64_t K, void *payload_dev, size_t payload_capacity, void *y_slots_dev,
+                                    void *cuda_stream);
+
 /* ------------------------------------------------- exchange (Section 5) */
 
 /* Section 5 describes the system-level form of the method: the payloads are all-gathered and every

@@ -55,6 +55,9 @@ SIGNATURES = {
     "tpq_dequant_reduce": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p]),
     "tpq_dequant_reduce_bias": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p,
                                         c_void_p]),
+    "tpq_permute_weight": (c_int, [c_void_p, c_void_p, c_int64, c_void_p, c_void_p]),
+    "tpq_linear_quantize_pack": (c_int, [c_void_p, c_int, c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_size_t, c_void_p,
+                                         c_void_p]),
     "tpq_quantize_pack_push": (c_int, [c_void_p, c_int, c_void_p, c_int64, c_int64, POINTER(c_void_p), POINTER(c_void_p),
                                        c_int, c_size_t, ctypes.c_uint32, c_void_p]),
     "tpq_dequant_reduce_arrivals": (c_int, [c_void_p, POINTER(c_void_p), c_int, c_int64, c_void_p, c_int, c_int64, c_void_p,
@@ -222,6 +225,14 @@ class Tpq:
         else:
             self._check(lib().tpq_dequant_reduce_bias(self._h, arr, len(payload_ptrs), T, out_ptr, out_dtype, stride,
                                                       bias_ptr, stream))
+
+    def permute_weight(self, w_ptr: int, K: int, w_slots_ptr: int, stream: int = 0):
+        self._check(lib().tpq_permute_weight(self._h, w_ptr, K, w_slots_ptr, stream))
+
+    def linear_quantize_pack(self, shard: int, x_ptr: int, w_slots_ptr: int, T: int, K: int, payload_ptr: int,
+                             payload_capacity: int, y_slots_ptr: int | None = None, stream: int = 0):
+        self._check(lib().tpq_linear_quantize_pack(self._h, shard, x_ptr, w_slots_ptr, T, K, payload_ptr, payload_capacity,
+                                                   y_slots_ptr, stream))
 
     def quantize_pack_push(self, shard: int, y_ptr: int, T: int, dst_ptrs, arrived_ptrs, dst_capacity: int, epoch: int,
                            row_stride: int | None = None, stream: int = 0):

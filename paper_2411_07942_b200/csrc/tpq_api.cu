@@ -489,6 +489,43 @@ tpq_status tpq_wait_arrivals(tpq_ctx *c, const uint32_t *arrived, int n, uint32_
     return TPQ_OK;
 }
 
+// Section 2: the layer ahead of the synchronisation point, f^(i)(x^(i)) = x^(i) W^(i), fused with C^(i).
+tpq_status tpq_permute_weight(tpq_ctx *c, const void *w, int64_t K, void *w_slots, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set: call tpq_select_features or tpq_set_features");
+    if (!w || !w_slots || w == w_slots) return fail(c, TPQ_ERR_INVALID_ARG, "NULL or aliased weight buffers");
+    if (K < 1) return fail(c, TPQ_ERR_INVALID_ARG, "K < 1");
+    if (!aligned16(w) || !aligned16(w_slots)) return fail(c, TPQ_ERR_ALIGN, "weight buffers must be 16-byte aligned");
+    cudaError_t e = tpq_launch_permute_weight(c, w, w_slots, K, static_cast<cudaStream_t>(stream), &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e, "permute_weight kernel");
+    return TPQ_OK;
+}
+
+tpq_status tpq_linear_quantize_pack(tpq_ctx *c, int shard, const void *x, const void *w_slots, int64_t T, int64_t K,
+                                    void *payload, size_t cap, void *y_slots, void *stream)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set: call tpq_select_features or tpq_set_features");
+    if (shard < 0 || shard >= c->N) return fail(c, TPQ_ERR_INVALID_ARG, "shard %d out of range [0, %d)", shard, c->N);
+    if (T < 0) return fail(c, TPQ_ERR_INVALID_ARG, "T < 0");
+    if (T == 0) return TPQ_OK;
+    if (!x || !w_slots || !payload) return fail(c, TPQ_ERR_INVALID_ARG, "NULL buffer");
+    if (!aligned16(x) || !aligned16(w_slots) || !aligned16(payload) || (y_slots && !aligned16(y_slots)))
+        return fail(c, TPQ_ERR_ALIGN, "x, w_slots, payload and y_slots must be 16-byte aligned");
+    if (!tpq_linear_ok(c, T, K))
+        return fail(c, TPQ_ERR_INVALID_ARG,
+                    "the fused layer needs 4-bit codes, E and k multiples of 8 and K a multiple of 8 (K = %lld)", (long long)K);
+    if (cap < tpq_payload_bytes(c, T))
+        return fail(c, TPQ_ERR_SIZE, "payload capacity %zu < %zu", cap, tpq_payload_bytes(c, T));
+    cudaError_t e = tpq_launch_linear_quantize(c, shard, x, w_slots, T, K, payload, y_slots, static_cast<cudaStream_t>(stream),
+                                               &c->launches);
+    if (e != cudaSuccess) return cuda_fail(c, e, "linear_quantize kernel");
+    return TPQ_OK;
+}
+
 static tpq_status dequant_reduce_impl(tpq_ctx *c, const void *const *payloads, int n_payloads, int64_t T, void *out,
                                       tpq_out_dtype dt, int64_t out_stride, void *stream);
 

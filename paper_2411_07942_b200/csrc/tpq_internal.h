@@ -112,6 +112,13 @@ cudaError_t tpq_launch_publish_arrivals(uint32_t *const *arrived, int n_dst, uin
 cudaError_t tpq_launch_wait_arrivals(const tpq_ctx *c, const uint32_t *arrived, int n, uint32_t epoch,
                                      unsigned long long timeout_ns, cudaStream_t st, int64_t *launches);
 
+// The pre-synchronisation linear layer fused with the compressor (linear.cu): tensor-core GEMM whose epilogue
+// quantises and packs.  w_slots is the [E][K] weight matrix with its rows in slot order (tpq_launch_permute_weight).
+bool tpq_linear_ok(const tpq_ctx *c, int64_t T, int64_t K);
+cudaError_t tpq_launch_permute_weight(const tpq_ctx *c, const void *w, void *out, int64_t K, cudaStream_t st, int64_t *launches);
+cudaError_t tpq_launch_linear_quantize(const tpq_ctx *c, int shard, const void *x, const void *w_slots, int64_t T, int64_t K,
+                                       void *payload, void *y_slots, cudaStream_t st, int64_t *launches);
+
 // Code widths other than 4 bits on shapes that are multiples of 8 (groups.cu).
 bool tpq_groups_ok(const tpq_ctx *c, int64_t T, int64_t stride);
 cudaError_t tpq_launch_quantize_groups(const tpq_ctx *c, int shard0, int n, const void *const *ys, int64_t T,
