@@ -7,10 +7,11 @@
 // fillers) and columns L .. E-1 are the selected features in rank order.  The epilogue therefore has no hole
 // logic: a group of 8 columns is either one 32-bit word of codes or 8 BF16 values of the BF16 block.
 //
-// Kernel: tcgen05 (5th-generation tensor cores).  A block owns a 128 x BN tile of the output; operands are
-// staged by TMA (128-byte swizzle) in a ring of shared-memory stages; one thread issues tcgen05.mma
-// (M = 128, N = BN, K = 16, BF16 x BF16 -> FP32) with the accumulator in tensor memory; four epilogue warps
-// read it back (tcgen05.ld), round to BF16 (the layer's output type), quantise and store.
+// Kernel: tcgen05 (5th-generation tensor cores), persistent: one block per SM walks 128 x BN tiles of the
+// output.  Operands are staged by TMA (128-byte swizzle) in a ring of shared-memory stages that runs on
+// across tiles; one thread issues tcgen05.mma (M = 128, N = BN, K = 16, BF16 x BF16 -> FP32) into one of TWO
+// accumulators in tensor memory; four epilogue warps read the other one back (tcgen05.ld), round to BF16
+// (the layer's output type), quantise and store, while the tensor cores work on the next tile.
 //   warp 0    TMA producer (one lane)
 //   warp 1    tensor-memory allocation (whole warp), MMA issue (one lane), de-allocation
 //   warps 2-5 epilogue; warp w reads the 32 accumulator rows of lane quadrant w % 4
@@ -34,12 +35,13 @@ __host__ __device__ constexpr int lq_stages(int BN)
     int n = (int)((200u * 1024u) / lq_stage_bytes(BN));
     return n > 8 ? 8 : n;
 }
-__host__ __device__ constexpr uint32_t lq_tmem_cols(int BN) { return BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256; }
+// two accumulators (the epilogue drains one while the tensor cores fill the other), a power of two of columns
+__host__ __device__ constexpr uint32_t lq_tmem_cols(int BN) { return 2 * BN <= 64 ? 64 : 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512; }
 __host__ __device__ constexpr size_t lq_smem_bytes(int BN)
 {
-    // 1024 B of slack for the manual alignment; stages; 160 B: barriers (full[8], empty[8], accumulator) and the
-    // tensor-memory address; the tile's reciprocal steps
-    return 1024 + (size_t)lq_stages(BN) * lq_stage_bytes(BN) + 160 + (size_t)BN * 4;
+    // 1024 B of slack for the manual alignment; stages; 176 B: barriers (full[8], empty[8], accumulators 2 x 2)
+    // and the tensor-memory address; the reciprocal steps of two tiles
+    return 1024 + (size_t)lq_stages(BN) * lq_stage_bytes(BN) + 176 + 2 * (size_t)BN * 4;
 }
 
 struct LQParams {
@@ -169,34 +171,36 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
     constexpr uint32_t TCOLS = lq_tmem_cols(BN);
     const uint32_t base = (lq_smem_u32(lq_raw) + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
     uint8_t *const gen = lq_raw + (base - lq_smem_u32(lq_raw));
-    const uint32_t bars = base + NS * STAGE;  // full[NS], empty[NS], accumulator
-    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(gen + NS * STAGE + 136);
-    float *const inv_tile = reinterpret_cast<float *>(gen + NS * STAGE + 160);
+    // after the stages: full[8], empty[8], acc_full[2], acc_empty[2] (8 bytes each), the tensor-memory address,
+    // then the reciprocal steps of two tiles
+    const uint32_t bars = base + NS * STAGE;
+    uint32_t *const tmem_slot = reinterpret_cast<uint32_t *>(gen + NS * STAGE + 160);
+    float *const inv_tiles = reinterpret_cast<float *>(gen + NS * STAGE + 176);
     auto full = [&](int s) { return bars + 8u * s; };
     auto empty = [&](int s) { return bars + 8u * (8 + s); };
-    const uint32_t accum = bars + 8u * 16;
+    auto acc_full = [&](int b) { return bars + 8u * (16 + b); };
+    auto acc_empty = [&](int b) { return bars + 8u * (18 + b); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.x * LQ_BM, n0 = blockIdx.y * BN;
     const int L = p.E - p.k, L8 = L >> 3;
     const int nkb = (p.K + LQ_BK - 1) / LQ_BK;
+    // tiles in row-major order of (column tile, row tile): neighbouring blocks share a weight tile
+    const int mt = (int)((p.T + LQ_BM - 1) / LQ_BM), nt = (p.E + BN - 1) / BN;
+    const int tiles = mt * nt;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
             lq_mbar_init(full(s), 1);
             lq_mbar_init(empty(s), 1);
         }
-        lq_mbar_init(accum, 1);
+        for (int b = 0; b < 2; ++b) {
+            lq_mbar_init(acc_full(b), 1);
+            lq_mbar_init(acc_empty(b), 4);  // one arrival per epilogue warp
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tc_alloc(lq_smem_u32(tmem_slot), TCOLS);
-    if (warp >= 2) {  // the tile's reciprocal steps in slot order (0 beyond the code slots)
-        for (int c = tid - 64; c < BN; c += LQ_THREADS - 64) {
-            const int col = n0 + c;
-            inv_tile[c] = (col < L) ? __ldg(p.inv_s + __ldg(p.lp_idx + col)) : 0.0f;
-        }
-    }
     tc_fence_before();
     tpq_grid_dep_wait();  // the operands and the payload buffer may still be in use by the kernel ahead
     __syncthreads();
@@ -207,56 +211,93 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
 
     if (warp == 0) {
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % NS;
-                if (kb >= NS && !lq_mbar_wait(empty(s), ((kb / NS) - 1) & 1)) {
-                    ok = false;
-                    break;
+            int it = 0;  // k-blocks issued so far, over all of this block's tiles
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile % mt) * LQ_BM, n0 = (tile / mt) * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % NS;
+                    if (it >= NS && !lq_mbar_wait(empty(s), ((it / NS) - 1) & 1)) {
+                        ok = false;
+                        break;
+                    }
+                    lq_mbar_expect_tx(full(s), STAGE);
+                    lq_tma_load_2d(base + s * STAGE, &map_x, kb * LQ_BK, m0, full(s));
+                    lq_tma_load_2d(base + s * STAGE + LQ_A_BYTES, &map_w, kb * LQ_BK, n0, full(s));
                 }
-                lq_mbar_expect_tx(full(s), STAGE);
-                lq_tma_load_2d(base + s * STAGE, &map_x, kb * LQ_BK, m0, full(s));
-                lq_tma_load_2d(base + s * STAGE + LQ_A_BYTES, &map_w, kb * LQ_BK, n0, full(s));
-                ++issued;
             }
             if (!ok)  // giving up: let the copies already issued land before the block's shared memory is released
-                for (int j = issued > NS ? issued - NS : 0; j < issued; ++j) (void)lq_mbar_wait(full(j % NS), (j / NS) & 1);
+                for (int j = it > NS ? it - NS : 0; j < it; ++j) (void)lq_mbar_wait(full(j % NS), (j / NS) & 1);
         }
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = lq_instr_desc(BN);
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % NS;
-                if (!lq_mbar_wait(full(s), (kb / NS) & 1)) {
+            int it = 0, n_tile = 0;
+            for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x, ++n_tile) {
+                const int b = n_tile & 1;
+                // the epilogue must have drained this accumulator (used two tiles ago)
+                if (n_tile >= 2 && !lq_mbar_wait(acc_empty(b), ((n_tile >> 1) - 1) & 1)) {
                     ok = false;
                     break;
                 }
                 tc_fence_after();
-                const uint32_t a = base + s * STAGE, b = a + LQ_A_BYTES;
+                const uint32_t d = tmem + (uint32_t)(b * BN);
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % NS;
+                    if (!lq_mbar_wait(full(s), (it / NS) & 1)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a = base + s * STAGE, bb = a + LQ_A_BYTES;
 #pragma unroll
-                for (int k4 = 0; k4 < LQ_BK / 16; ++k4)
-                    tc_mma_bf16(tmem, lq_smem_desc(a + k4 * 32), lq_smem_desc(b + k4 * 32), idesc, (kb | k4) != 0);
-                tc_commit(empty(s));  // arrives when the MMAs above have read the stage
+                    for (int k4 = 0; k4 < LQ_BK / 16; ++k4)
+                        tc_mma_bf16(d, lq_smem_desc(a + k4 * 32), lq_smem_desc(bb + k4 * 32), idesc, (kb | k4) != 0);
+                    tc_commit(empty(s));  // arrives when the MMAs above have read the stage
+                }
+                if (ok) tc_commit(acc_full(b));  // arrives when the tile's accumulator is complete
             }
-            if (ok) tc_commit(accum);  // arrives when the accumulator is complete
         }
         __syncwarp();
     } else {
-        // ---------------- epilogue
-        if (!lq_mbar_wait(accum, 0)) ok = false;
-        ok = __all_sync(0xffffffffu, ok);  // the tensor-memory loads below are warp-wide
-        tc_fence_after();
-        const int q = warp & 3;
-        const int64_t row = (int64_t)m0 + q * 32 + lane;
-        const bool row_on = ok && row < p.T;
+        // ---------------- epilogue: tile i is drained while the tensor cores work on tile i + 1
+        const int q = warp & 3, et = tid - 64;
         uint32_t *const lp_out = reinterpret_cast<uint32_t *>(p.payload);
         uint16_t *const hp_out = reinterpret_cast<uint16_t *>(p.payload + p.lp_bytes);
-        if (ok) {
+        int n_tile = 0;
+        for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n_tile) {
+            const int b = n_tile & 1;
+            const int m0 = (tile % mt) * LQ_BM, n0 = (tile / mt) * BN;
+            float *const inv_tile = inv_tiles + b * BN;
+            for (int c = et; c < BN; c += 128) {  // the tile's reciprocal steps in slot order
+                const int col = n0 + c;
+                inv_tile[c] = (col < L) ? __ldg(p.inv_s + __ldg(p.lp_idx + col)) : 0.0f;
+            }
+            // barrier of the four epilogue warps (the steps above are in place) that also tells every thread
+            // whether ANY of them has given up: they leave the loop together, none is left waiting here
+            uint32_t any_bad;
+            asm volatile(
+                "{\n\t.reg .pred p, q;\n\t"
+                "setp.ne.u32 q, %1, 0;\n\t"
+                "bar.red.or.pred p, 1, 128, q;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(any_bad)
+                : "r"((uint32_t)!ok)
+                : "memory");
+            if (any_bad) {
+                ok = false;
+                break;
+            }
+            if (!lq_mbar_wait(acc_full(b), (n_tile >> 1) & 1)) ok = false;
+            ok = __all_sync(0xffffffffu, ok);  // the tensor-memory loads below are warp-wide
+            if (!ok) continue;                 // (reported at the next barrier above; no tile follows a lost one)
+            tc_fence_after();
+            const int64_t row = (int64_t)m0 + q * 32 + lane;
+            const bool row_on = row < p.T;
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 if (n0 + c0 >= p.E) break;  // uniform
                 uint32_t r[32];
-                tc_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                tc_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * BN + c0), r);
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int col = n0 + c0 + 8 * g;
@@ -287,9 +328,13 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
                     }
                 }
             }
+            // this warp has read its quadrant of the accumulator: hand it back to the MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(acc_empty(b)) : "memory");
         }
         // zero padding of the code section (its size is rounded up to 16 bytes)
-        if (blockIdx.x == 0 && blockIdx.y == 0 && warp == 2) {
+        if (blockIdx.x == 0 && warp == 2) {
             const int64_t valid = p.T * L8, words = p.lp_bytes / 4;
             for (int64_t w = valid + lane; w < words; w += 32) lp_out[w] = 0u;
         }
@@ -357,14 +402,15 @@ bool lq_map(const void *ptr, int64_t rows, int64_t K, int box_rows, CUtensorMap 
 }
 
 template <int BN>
-cudaError_t lq_launch(const LQParams &p, const void *x, const void *w, cudaStream_t st)
+cudaError_t lq_launch(const LQParams &p, const void *x, const void *w, int sm_count, cudaStream_t st)
 {
     CUtensorMap mx, mw;
     if (!lq_map(x, p.T, p.K, LQ_BM, &mx) || !lq_map(w, p.E, p.K, BN, &mw)) return cudaErrorNotSupported;
     const size_t smem = lq_smem_bytes(BN);
     cudaError_t e = cudaFuncSetAttribute(linear_quantize<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const dim3 grid((unsigned)((p.T + LQ_BM - 1) / LQ_BM), (unsigned)((p.E + BN - 1) / BN));
+    const int64_t tiles = ((p.T + LQ_BM - 1) / LQ_BM) * ((p.E + BN - 1) / BN);
+    const dim3 grid((unsigned)(tiles < sm_count ? tiles : sm_count));  // persistent: a block walks tiles b, b + grid, ...
     return tpq_launch_pdl(linear_quantize<BN>, grid, dim3(LQ_THREADS), smem, st, p, mx, mw);
 }
 
@@ -411,9 +457,9 @@ cudaError_t tpq_launch_linear_quantize(const tpq_ctx *c, int shard, const void *
             best = bn;
         }
     }
-    cudaError_t e = best == 256 ? lq_launch<256>(p, x, w_slots, st)
-                  : best == 192 ? lq_launch<192>(p, x, w_slots, st)
-                                : lq_launch<128>(p, x, w_slots, st);
+    cudaError_t e = best == 256 ? lq_launch<256>(p, x, w_slots, c->sm_count, st)
+                  : best == 192 ? lq_launch<192>(p, x, w_slots, c->sm_count, st)
+                                : lq_launch<128>(p, x, w_slots, c->sm_count, st);
     if (e == cudaSuccess) ++*launches;
     return e;
 }
