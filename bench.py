@@ -60,6 +60,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense BF16 TFLOP/s of the library GEMM on this machine (burst figure: the fused layer is timed alone)."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
 def payload_bytes(T, E, k, bits=4):
     nbits = T * (E - k) * bits
     return ((nbits + 7) // 8 + 15) // 16 * 16 + 2 * T * k
@@ -393,6 +402,39 @@ def main():
                          timeout_ns=50_000_000)
 
     wd_ms = time_loop(wd_only, reps)
+
+    # ---- the layer ahead of the synchronisation point fused with the compressor (Section 2): x [T][K] times the
+    # device's slice of the down projection, K = 2.7 E / N rounded to 64 (Llama's 13824 / 4 at E = 5120), against
+    # the library GEMM followed by quantize_pack.  Tensor-bound; an extra, not the headline path.
+    fused = None
+    if args.bits == 4 and E % 8 == 0 and k % 8 == 0:
+        Kd = max(64, int(round(2.7 * E / N / 64)) * 64)
+        gen = torch.Generator(device=dev).manual_seed(11)
+        xk = torch.randn((T, Kd), device=dev, generator=gen).to(torch.bfloat16)
+        wk = (torch.randn((E, Kd), device=dev, generator=gen) / Kd ** 0.5).to(torch.bfloat16)
+        wslots = torch.empty_like(wk)
+        t.permute_weight(wk.data_ptr(), Kd, wslots.data_ptr(), stream=sh)
+        ytmp = torch.empty((T, E), dtype=torch.bfloat16, device=dev)
+        pl0 = sets[0][1][0]
+
+        def fused_fn(b):
+            t.linear_quantize_pack(0, xk.data_ptr(), wslots.data_ptr(), T, Kd, pl0.data_ptr(), P, stream=sh)
+
+        def unfused_fn(b):
+            with torch.cuda.stream(stream):
+                torch.matmul(xk, wk.t(), out=ytmp)
+            t.quantize_pack(0, ytmp.data_ptr(), T, pl0.data_ptr(), P, stream=sh)
+
+        def gemm_fn(b):
+            with torch.cuda.stream(stream):
+                torch.matmul(xk, wk.t(), out=ytmp)
+
+        f_ms, u_ms, g_ms = time_loop(fused_fn, reps), time_loop(unfused_fn, reps), time_loop(gemm_fn, reps)
+        tpeak, tkind = measured_tensor_peak()
+        flops = 2.0 * T * Kd * E
+        fused = {"shape": f"x [{T}][{Kd}] . w [{E}][{Kd}]^T", "fused_ms": f_ms, "fused_TFLOPs": flops / f_ms / 1e9,
+                 "frac_of_" + tkind + "_bf16_peak": flops / f_ms / 1e9 / tpeak, "peak_TFLOPs": tpeak,
+                 "library_gemm_then_quantize_pack_ms": u_ms, "library_gemm_alone_ms": g_ms}
     # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
     # what the launch path costs, relevant for the decode-sized workloads
     graph_ms = None
@@ -496,6 +538,7 @@ def main():
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
         "step_cuda_graph_replay_ms": graph_ms,
         "dequant_reduce_bias_ms_per_launch": db_ms,
+        "fused_layer": fused,
         "exchange_one_gpu": {"quantize_pack_push_1_dst_ms": p1_ms, f"quantize_pack_push_{push_max}_dst_ms": pn_ms,
                              "dequant_reduce_arrivals_ms": wd_ms,
                              "note": "destinations are local buffers; across GPUs the stores cross NVLink"},

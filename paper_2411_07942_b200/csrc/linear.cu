@@ -161,6 +161,20 @@ __device__ __forceinline__ uint32_t lq_code(float x, float inv)
     return __float_as_uint(__fadd_rn(u, 12582912.0f)) & 0xFu;
 }
 
+// Tile order: bands of LQ_GROUP_M row tiles; inside a band column tile by column tile, the band's row tiles
+// innermost.  Blocks that run together share a weight tile, and a band's rows of x (LQ_GROUP_M x 128 x K
+// values) stay in L2 while every column tile passes over them, whatever T is.
+constexpr int LQ_GROUP_M = 16;
+__device__ __forceinline__ void lq_tile_origin(int tile, int mt, int nt, int BN, int &m0, int &n0)
+{
+    const int per_band = LQ_GROUP_M * nt;
+    const int band = tile / per_band, in_band = tile - band * per_band;
+    const int rows = (mt - band * LQ_GROUP_M < LQ_GROUP_M) ? mt - band * LQ_GROUP_M : LQ_GROUP_M;  // the last band may be short
+    const int n = in_band / rows, m = band * LQ_GROUP_M + (in_band - n * rows);
+    m0 = m * LQ_BM;
+    n0 = n * BN;
+}
+
 template <int BN>
 __global__ void __launch_bounds__(LQ_THREADS, 1)
 linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w)
@@ -184,7 +198,6 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int L = p.E - p.k, L8 = L >> 3;
     const int nkb = (p.K + LQ_BK - 1) / LQ_BK;
-    // tiles in row-major order of (column tile, row tile): neighbouring blocks share a weight tile
     const int mt = (int)((p.T + LQ_BM - 1) / LQ_BM), nt = (p.E + BN - 1) / BN;
     const int tiles = mt * nt;
 
@@ -213,7 +226,8 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
         if (lane == 0) {
             int it = 0;  // k-blocks issued so far, over all of this block's tiles
             for (int tile = blockIdx.x; tile < tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % mt) * LQ_BM, n0 = (tile / mt) * BN;
+                int m0, n0;
+                lq_tile_origin(tile, mt, nt, BN, m0, n0);
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % NS;
                     if (it >= NS && !lq_mbar_wait(empty(s), ((it / NS) - 1) & 1)) {
@@ -267,7 +281,8 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
         int n_tile = 0;
         for (int tile = blockIdx.x; tile < tiles; tile += gridDim.x, ++n_tile) {
             const int b = n_tile & 1;
-            const int m0 = (tile % mt) * LQ_BM, n0 = (tile / mt) * BN;
+            int m0, n0;
+            lq_tile_origin(tile, mt, nt, BN, m0, n0);
             float *const inv_tile = inv_tiles + b * BN;
             for (int c = et; c < BN; c += 128) {  // the tile's reciprocal steps in slot order
                 const int col = n0 + c;
@@ -444,16 +459,19 @@ cudaError_t tpq_launch_linear_quantize(const tpq_ctx *c, int shard, const void *
     p.payload = static_cast<uint8_t *>(payload);
     p.y_slots = static_cast<uint16_t *>(y_slots);
     p.status = c->t.status;
-    // tile width: the one that wastes the fewest block slots over whole waves of the grid
+    // Tile width.  A block's time is (tiles it walks) x (k-blocks per tile) x (time per k-block), and the time
+    // per k-block barely depends on the width (the operand pipeline, not the tensor pipe, sets it: measured
+    // 385 / 376 / 344 ns for 256 / 192 / 128 columns), so the widest tile wins unless a narrower one saves a
+    // whole wave of the persistent grid.
     const int64_t mt = (T + LQ_BM - 1) / LQ_BM;
     int best = 256;
-    double best_eff = 0.0;
+    double best_cost = 0.0;
     for (int bn : {256, 192, 128}) {
         const int64_t tiles = mt * ((c->E + bn - 1) / bn);
         const int64_t waves = (tiles + c->sm_count - 1) / c->sm_count;
-        const double eff = (double)T * c->E / ((double)waves * c->sm_count * LQ_BM * bn);
-        if (eff > best_eff + 1e-9) {
-            best_eff = eff;
+        const double cost = (double)waves * (bn == 256 ? 385.0 : bn == 192 ? 376.0 : 344.0);
+        if (best_cost == 0.0 || cost < best_cost - 1e-9) {
+            best_cost = cost;
             best = bn;
         }
     }
