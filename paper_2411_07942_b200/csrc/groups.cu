@@ -74,11 +74,17 @@ struct QGParams {
     const int32_t *lp_idx, *hp_idx;
 };
 
+// Work layout of both kernels: the GW = (E-k)/8 + k/8 thread columns of a row (groups, then octets of
+// selected features) are cut into chunks of GK_THREADS; grid.x = chunks x row lanes.  A thread keeps its column
+// for its whole life (its tables are loaded once) and walks blocks of R rows with the stride of the row lanes.
 template <int B>
 __global__ void __launch_bounds__(GK_THREADS) quantize_groups(const QGParams p)
 {
     constexpr int R = 4;
     const int E = p.E, k = p.k, L8 = (E - k) >> 3, k8 = k >> 3, GW = L8 + k8;
+    const int chunks = (GW + GK_THREADS - 1) / GK_THREADS;
+    const int gi = (int)(blockIdx.x % chunks) * GK_THREADS + threadIdx.x;
+    const int lane0 = blockIdx.x / chunks, lanes = gridDim.x / chunks;
     const int sh = blockIdx.y;
     const uint16_t *const y = p.y[sh];
     uint8_t *const pl = p.payload[sh];
@@ -89,49 +95,71 @@ __global__ void __launch_bounds__(GK_THREADS) quantize_groups(const QGParams p)
         const int64_t code_bytes = p.T * L8 * B;
         if (blockIdx.x == 0 && code_bytes + threadIdx.x < p.lp_bytes) pl[code_bytes + threadIdx.x] = 0;
     }
-    for (int64_t u = (int64_t)blockIdx.x * GK_THREADS + threadIdx.x; u < n_rb * GW; u += (int64_t)gridDim.x * GK_THREADS) {
-        const int64_t rb = u / GW;
-        const int gi = (int)(u - rb * GW);
-        const int64_t t0 = rb * R;
-        if (gi < L8) {
-            const int g = gi;
-            const float4 i0 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g));
-            const float4 i1 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g + 4));
-            float inv[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
-            const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
-            int fidx[8];
+    if (gi >= GW) return;
+    if (gi < L8) {
+        const int g = gi;
+        const float4 i0 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g));
+        const float4 i1 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g + 4));
+        float inv[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
+        const uint32_t mask = __ldg(p.grp + g) & 0xFFu;
+        // holes: the slot carries the filler feature.  The first hole of the group is handled without a branch
+        // (its filler value is fetched with the row), further ones (rare) in a branch.
+        const int first = mask ? __ffs(mask) - 1 : 0;
+        const int f_first = mask ? __ldg(p.lp_idx + 8 * g + first) : 8 * g;
+        const uint32_t more = mask & (mask - 1);
+        if (mask) {
 #pragma unroll
-            for (int n = 0; n < 8; ++n) {
-                fidx[n] = 8 * g + n;
-                if (mask & (1u << n)) {  // a hole: the slot carries the filler feature
-                    fidx[n] = __ldg(p.lp_idx + 8 * g + n);
-                    inv[n] = __ldg(inv_s + fidx[n]);
-                }
+            for (int n = 0; n < 8; ++n)
+                if (mask & (1u << n)) inv[n] = __ldg(inv_s + __ldg(p.lp_idx + 8 * g + n));
+        }
+        for (int64_t rb = lane0; rb < n_rb; rb += lanes) {
+            const int64_t t0 = rb * R;
+            uint4 v[R];
+            uint32_t fv[R];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {  // all loads first; rows past the end re-read the last row
+                const int64_t t = (t0 + r < p.T) ? t0 + r : p.T - 1;
+                const uint16_t *const row = y + t * p.stride;
+                v[r] = __ldcs(reinterpret_cast<const uint4 *>(row + 8 * g));
+                fv[r] = (uint32_t)__ldg(row + f_first) << 16;
             }
+            uint8_t *dst = pl + (t0 * L8 + g) * B;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
-                const int64_t t = t0 + r;
-                if (t >= p.T) break;
-                const uint16_t *const row = y + t * p.stride;
-                const uint4 v = __ldcs(reinterpret_cast<const uint4 *>(row + 8 * g));
-                uint32_t xb[8] = {v.x << 16, v.x & 0xFFFF0000u, v.y << 16, v.y & 0xFFFF0000u,
-                                  v.z << 16, v.z & 0xFFFF0000u, v.w << 16, v.w & 0xFFFF0000u};
-                uint64_t bits = 0;
+                if (t0 + r >= p.T) break;
+                uint32_t xb[8] = {v[r].x << 16, v[r].x & 0xFFFF0000u, v[r].y << 16, v[r].y & 0xFFFF0000u,
+                                  v[r].z << 16, v[r].z & 0xFFFF0000u, v[r].w << 16, v[r].w & 0xFFFF0000u};
+                if (mask) {
+#pragma unroll
+                    for (int n = 0; n < 8; ++n) xb[n] = (n == first) ? fv[r] : xb[n];
+                    if (more) {
+                        const uint16_t *const row = y + (t0 + r) * p.stride;
+#pragma unroll
+                        for (int n = 0; n < 8; ++n)
+                            if (more & (1u << n)) xb[n] = (uint32_t)__ldg(row + __ldg(p.lp_idx + 8 * g + n)) << 16;
+                    }
+                }
+                // codes 0..3 and 4..7 are gathered in two 32-bit halves (4 B <= 32 bits each); the code is read
+                // from the low bits of fl(u + 1.5 * 2^23): nearest-even rounding without a conversion instruction
+                uint32_t half[2] = {0u, 0u};
 #pragma unroll
                 for (int n = 0; n < 8; ++n) {
-                    if (mask & (1u << n)) xb[n] = (uint32_t)__ldg(row + fidx[n]) << 16;
                     float uq = __fmul_rn(__uint_as_float(xb[n]), inv[n]);
                     uq = fminf(fmaxf(uq, lo), hi);
-                    const uint32_t q = (uint32_t)__float2int_rn(uq) & ((1u << B) - 1u);
-                    bits |= (uint64_t)q << (n * B);
+                    const uint32_t q = __float_as_uint(__fadd_rn(uq, 12582912.0f)) & ((1u << B) - 1u);
+                    half[n >> 2] |= q << ((n & 3) * B);
                 }
-                store_code_bytes<B>(pl + (t * L8 + g) * B, bits);
+                store_code_bytes<B>(dst, (uint64_t)half[0] | ((uint64_t)half[1] << (4 * B)));
+                dst += (size_t)L8 * B;
             }
-        } else {
-            const int h8 = gi - L8;
-            const int4 c0 = __ldg(reinterpret_cast<const int4 *>(p.hp_idx + 8 * h8));
-            const int4 c1 = __ldg(reinterpret_cast<const int4 *>(p.hp_idx + 8 * h8) + 1);
-            const int col[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        }
+    } else {
+        const int h8 = gi - L8;
+        const int4 c0 = __ldg(reinterpret_cast<const int4 *>(p.hp_idx + 8 * h8));
+        const int4 c1 = __ldg(reinterpret_cast<const int4 *>(p.hp_idx + 8 * h8) + 1);
+        const int col[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        for (int64_t rb = lane0; rb < n_rb; rb += lanes) {
+            const int64_t t0 = rb * R;
 #pragma unroll
             for (int r = 0; r < R; ++r) {
                 const int64_t t = t0 + r;
@@ -293,13 +321,27 @@ __global__ void __launch_bounds__(GK_THREADS) dequant_groups(const DGParams p)
     }
 }
 
-unsigned gk_grid(int64_t units, int sm_count)
+// flat grid of the dequantiser: one unit = (row block, thread column)
+unsigned gk_grid_units(int64_t units, int sm_count)
 {
     int64_t blocks = (units + GK_THREADS - 1) / GK_THREADS;
     const int64_t cap = (int64_t)sm_count * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     return (unsigned)blocks;
+}
+
+// grid.x = column chunks x row lanes; every row lane walks the same number of row blocks (no lane is left
+// with one block more than the others), up to about 32 blocks per SM
+unsigned gk_grid(int GW, int64_t row_blocks, int sm_count)
+{
+    const int64_t chunks = (GW + GK_THREADS - 1) / GK_THREADS;
+    int64_t lanes_max = ((int64_t)sm_count * 32 + chunks - 1) / chunks;
+    if (lanes_max < 1) lanes_max = 1;
+    const int64_t iters = (row_blocks + lanes_max - 1) / lanes_max;
+    int64_t lanes = (row_blocks + iters - 1) / (iters > 0 ? iters : 1);
+    if (lanes < 1) lanes = 1;
+    return (unsigned)(chunks * lanes);
 }
 
 }  // namespace
@@ -326,8 +368,7 @@ cudaError_t tpq_launch_quantize_groups(const tpq_ctx *c, int shard0, int n, cons
         p.E = E; p.k = k;
         p.inv_s = c->t.inv_s + (size_t)(shard0 + b0) * E;
         p.grp = c->t.grp; p.lp_idx = c->t.lp_idx; p.hp_idx = c->t.hp_idx;
-        const int64_t units = ((T + 3) / 4) * (int64_t)((E - k) / 8 + k / 8);
-        const dim3 grid(gk_grid(units, c->sm_count), (unsigned)nb);
+        const dim3 grid(gk_grid((E - k) / 8 + k / 8, (T + 3) / 4, c->sm_count), (unsigned)nb);
         switch (c->bits) {
         case 2: quantize_groups<2><<<grid, GK_THREADS, 0, st>>>(p); break;
         case 3: quantize_groups<3><<<grid, GK_THREADS, 0, st>>>(p); break;
@@ -369,7 +410,7 @@ cudaError_t tpq_launch_dequant_groups(const tpq_ctx *c, const void *const *paylo
     p.bias = c->call_bias;
     p.arr = c->call_arr;
     const int64_t units = ((T + 1) / 2) * (int64_t)((E - k) / 8 + k / 8);
-    const unsigned grid = gk_grid(units, c->sm_count);
+    const unsigned grid = gk_grid_units(units, c->sm_count);
     switch (c->bits) {
     case 2: launch_dequant_groups_b<2>(p, fp32_out, grid, st); break;
     case 3: launch_dequant_groups_b<3>(p, fp32_out, grid, st); break;
