@@ -33,7 +33,7 @@ def _setup(N, T, K, E, k, seed):
     return xs, ws
 
 
-@pytest.mark.parametrize("N,T,K,E,k", [(2, 100, 64, 256, 8), (2, 300, 200, 1032, 16), (1, 128, 128, 192, 0),
+@pytest.mark.parametrize("N,T,K,E,k", [(1, 1, 8, 16, 8), (1, 5, 16, 64, 0), (2, 130, 72, 264, 8), (2, 100, 64, 256, 8), (2, 300, 200, 1032, 16), (1, 128, 128, 192, 0),
                                        (2, 517, 1280, 2048, 32), (4, 2048, 3456, 5120, 80)])
 def test_fused_layer(N, T, K, E, k):
     orc = oracle.c()
