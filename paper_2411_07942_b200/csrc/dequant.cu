@@ -844,7 +844,9 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 // Main and fix-up warps release a stage through the "empty" mbarrier; no block-wide barrier in the loop.
 // G is a multiple of 4/gcd(4, L/8) so that every stage starts 16-byte aligned in the code stream.
 // ----------------------------------------------------------------------------------------------
-constexpr int DR_FIXUP_THREADS = 128;
+// fix-up threads: 128, or 96 where that takes the block from 25 warps (allocated as 28: 72 registers per
+// thread) to 24 (80 registers) and two rows per stage leave few items
+constexpr int DR_FIXUP_MAX = 128;
 
 struct DRLayout {
     size_t lp_stage, hp_stage, stage, bars, total;
@@ -883,15 +885,15 @@ __device__ __forceinline__ long long tpq_dnow()
 #define TPQ_DMARK(slot) do { } while (0)
 #endif
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
-__global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(const DRParams pp)
+template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+__global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     TPQ_DMARK(0);
     const DQParams &p = pp.q;
     const DXParams &x = pp.x;
     const int tid = threadIdx.x;
-    const int NT = blockDim.x - DR_FIXUP_THREADS - 32;  // main threads; then the fix-up warps; then the producer warp
+    const int NT = blockDim.x - FX - 32;  // main threads; then the fix-up warps; then the producer warp
     const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;  // G rows per stage, even
     const int L = E - k, L8 = L >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
@@ -906,7 +908,7 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
     if (tid == 0) {
         for (int s = 0; s < nstage; ++s) {
             mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), (NT + DR_FIXUP_THREADS) / 32);
+            mbar_init(smem_u32(&empty[s]), (NT + FX) / 32);
             mbar_init(smem_u32(&main_done[s]), NT / 32);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -930,10 +932,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
     __syncthreads();
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
 
-    if (tid >= NT + DR_FIXUP_THREADS) {
+    if (tid >= NT + FX) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
         // copies of the stage are issued by 2N lanes at once
-        const int pl = tid - NT - DR_FIXUP_THREADS;
+        const int pl = tid - NT - FX;
         int st = 0;
         uint32_t parity = 1;  // parity of the "empty" phase to wait for
         for (int it = 0;; ++it) {
@@ -984,10 +986,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
         const int ft = tid - NT;
         constexpr int FX_PRE = 2;  // items per thread kept in registers (more: the plain loop below)
         int f_r[FX_PRE], f_h[FX_PRE], f_hpcol[FX_PRE], f_col[FX_PRE], f_word[FX_PRE], f_sh[FX_PRE];
-        float f_s[FX_PRE][NMAX];
+        float f_s[FX_PRE][NMAX], f_bh[FX_PRE], f_bf[FX_PRE];
 #pragma unroll
         for (int j = 0; j < FX_PRE; ++j) {
-            const int item = ft + j * DR_FIXUP_THREADS;
+            const int item = ft + j * FX;
             const bool on = item < G * k;
             f_r[j] = on ? item / k : -1;
             f_h[j] = on ? item - f_r[j] * k : 0;
@@ -999,6 +1001,10 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
             f_sh[j] = (slot & 7) * 4;
 #pragma unroll
             for (int i = 0; i < NMAX; ++i) f_s[j][i] = (hole && i < N) ? __ldg(p.s_k + (size_t)i * E + f_col[j]) : 0.0f;
+            // (the items' biases with them: fetched in the store phase they would sit between "main_done" and
+            // the release of the stage)
+            f_bh[j] = (HAS_BIAS && on) ? __ldg(p.bias + f_hpcol[j]) : 0.0f;
+            f_bf[j] = (HAS_BIAS && hole) ? __ldg(p.bias + f_col[j]) : 0.0f;
         }
         const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
         for (int it = 0;; ++it) {
@@ -1042,13 +1048,13 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
                 if (f_r[j] >= 0 && f_r[j] < rows) {
                     const int64_t orow = (t0 + f_r[j]) * p.out_stride;
                     if (HAS_BIAS) {
-                        hv[j] = __fadd_rn(hv[j], __ldg(p.bias + f_hpcol[j]));
-                        if (f_col[j] >= 0) fv[j] = __fadd_rn(fv[j], __ldg(p.bias + f_col[j]));
+                        hv[j] = __fadd_rn(hv[j], f_bh[j]);
+                        if (f_col[j] >= 0) fv[j] = __fadd_rn(fv[j], f_bf[j]);
                     }
                     store_one<FP32OUT>(p.out, orow + f_hpcol[j], hv[j]);
                     if (f_col[j] >= 0) store_one<FP32OUT>(p.out, orow + f_col[j], fv[j]);
                 }
-            for (int item = ft + FX_PRE * DR_FIXUP_THREADS; item < rows * k; item += DR_FIXUP_THREADS) {
+            for (int item = ft + FX_PRE * FX; item < rows * k; item += FX) {
                 const int r = item / k, h = item - r * k;  // row of the stage, rank of the selected feature
                 const int64_t orow = (t0 + r) * p.out_stride;
                 float v = 0.0f;
@@ -1090,6 +1096,15 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
     constexpr int ESIZE = FP32OUT ? 4 : 2;
     uint8_t *const out_col = static_cast<uint8_t *>(p.out) + (size_t)8 * g_ld * ESIZE;
     const int64_t out_row_bytes = p.out_stride * ESIZE;
+    float2 b[4];  // the thread's 8 biases (only in the instantiation that adds them)
+#pragma unroll
+    for (int h = 0; h < 4; ++h) b[h] = make_float2(0.0f, 0.0f);
+    if (HAS_BIAS) {
+        const float4 b0 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld));
+        const float4 b1 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld + 4));
+        b[0] = make_float2(b0.x, b0.y); b[1] = make_float2(b0.z, b0.w);
+        b[2] = make_float2(b1.x, b1.y); b[3] = make_float2(b1.z, b1.w);
+    }
     TPQ_DMARK(1);
     for (int it = 0;; ++it) {
         const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
@@ -1123,10 +1138,6 @@ __global__ void __launch_bounds__(MAXT + DR_FIXUP_THREADS + 32, 1) dequant_rows(
             }
             if (live) {
                 if (HAS_BIAS) {  // (a hole's lane gets its own column's bias here and is overwritten by the fix-up)
-                    const float4 b0 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld));
-                    const float4 b1 = __ldg(reinterpret_cast<const float4 *>(p.bias + 8 * g_ld + 4));
-                    const float2 b[4] = {make_float2(b0.x, b0.y), make_float2(b0.z, b0.w), make_float2(b1.x, b1.y),
-                                         make_float2(b1.z, b1.w)};
 #pragma unroll
                     for (int r = 0; r < 2; ++r)
 #pragma unroll
@@ -1189,32 +1200,41 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
 
 namespace {
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
-cudaError_t launch_rows_w(const DRParams &pp, int grid, int threads, size_t smem, cudaStream_t st)
+template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+cudaError_t launch_rows_w(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>,
+    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, HAS_WAIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
-        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(threads), smem, st, pp);
+        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(consumers + FX + 32), smem,
+                           st, pp);
     return e;
 }
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
-cudaError_t launch_rows_v(const DRParams &pp, int grid, int threads, size_t smem, cudaStream_t st)
+template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS>
+cudaError_t launch_rows_v(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, true>(pp, grid, threads, smem, st)
-                          : launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, false>(pp, grid, threads, smem, st);
+    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, true>(pp, grid, consumers, smem, st)
+                          : launch_rows_w<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
 }
 
-template <int NMAX, int MAXT>
-cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int threads, size_t smem, cudaStream_t st)
+template <int NMAX, int MAXT, int FX>
+cudaError_t launch_rows_f(const DRParams &pp, int fp32_out, int grid, int consumers, size_t smem, cudaStream_t st)
 {
     const bool bias = pp.q.bias != nullptr;
     if (fp32_out)
-        return bias ? launch_rows_v<NMAX, MAXT, true, true>(pp, grid, threads, smem, st)
-                    : launch_rows_v<NMAX, MAXT, true, false>(pp, grid, threads, smem, st);
-    return bias ? launch_rows_v<NMAX, MAXT, false, true>(pp, grid, threads, smem, st)
-                : launch_rows_v<NMAX, MAXT, false, false>(pp, grid, threads, smem, st);
+        return bias ? launch_rows_v<NMAX, MAXT, FX, true, true>(pp, grid, consumers, smem, st)
+                    : launch_rows_v<NMAX, MAXT, FX, true, false>(pp, grid, consumers, smem, st);
+    return bias ? launch_rows_v<NMAX, MAXT, FX, false, true>(pp, grid, consumers, smem, st)
+                : launch_rows_v<NMAX, MAXT, FX, false, false>(pp, grid, consumers, smem, st);
+}
+
+template <int NMAX, int MAXT>
+cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int consumers, size_t smem, cudaStream_t st)
+{
+    // two rows per stage: G k items per stage fit three fix-up warps with two items each for k <= 96
+    return (pp.G == 2 && 2 * pp.q.k <= 2 * 96) ? launch_rows_f<NMAX, MAXT, 96>(pp, fp32_out, grid, consumers, smem, st)
+                                               : launch_rows_f<NMAX, MAXT, DR_FIXUP_MAX>(pp, fp32_out, grid, consumers, smem, st);
 }
 
 // Row kernel geometry; returns false if the shape does not admit it.
@@ -1427,10 +1447,9 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             const int L8 = (c->E - c->k) / 8;
             int consumers = ((L8 + 31) / 32) * 32;
             if (consumers < 32) consumers = 32;
-            const int threads = consumers + DR_FIXUP_THREADS + 32;
             cudaError_t e;
-            e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, threads, smem, st)
-                                 : launch_rows<4, 768>(pp, fp32_out, grid, threads, smem, st);
+            e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, consumers, smem, st)
+                                 : launch_rows<4, 768>(pp, fp32_out, grid, consumers, smem, st);
             if (e != cudaSuccess) return e;
             ++*launches;
             return cudaGetLastError();
