@@ -81,7 +81,6 @@ __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
 //   - filler feature filler[tau], tau < n_holes, lives in slot hole[tau]: one code per device;
 //   - selected feature hp_idx[h], h < k: the sum of the devices' BF16 values.
 // ----------------------------------------------------------------------------------------------
-constexpr int DR_WAIT_LIMIT = 1 << 22;
 
 __device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
 
@@ -184,41 +183,6 @@ struct DXParams {           // extras shared by the tiled kernels
     int *status;
 };
 
-// ---- mbarrier / bulk-copy primitives shared by the panel and row kernels
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (int i = 0; i < DR_WAIT_LIMIT; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
 
 // ----------------------------------------------------------------------------------------------
 // Panel kernel (any N, any row length).  A block owns a panel of CG groups of 8 adjacent code slots and
@@ -610,13 +574,6 @@ __host__ __device__ inline size_t dt_smem_bytes(int N, int CG, int nstage)
     return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes() + (size_t)nstage * 16;  // steps, ring, mbarriers
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
-}
 
 template <int CG, bool FP32OUT>
 __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams tp, const __grid_constant__ DTMaps maps)

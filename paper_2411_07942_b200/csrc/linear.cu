@@ -55,15 +55,6 @@ struct LQParams {
     int *status;
 };
 
-__device__ __forceinline__ uint32_t lq_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void lq_mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void lq_mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ bool lq_mbar_wait(uint32_t bar, uint32_t parity)
 {
     unsigned long long t0 = 0;
@@ -85,13 +76,6 @@ __device__ __forceinline__ bool lq_mbar_wait(uint32_t bar, uint32_t parity)
         }
     }
     return false;
-}
-__device__ __forceinline__ void lq_tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
-        : "memory");
 }
 
 // ---- tcgen05
@@ -183,8 +167,8 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
     constexpr int NS = lq_stages(BN);
     constexpr uint32_t STAGE = lq_stage_bytes(BN);
     constexpr uint32_t TCOLS = lq_tmem_cols(BN);
-    const uint32_t base = (lq_smem_u32(lq_raw) + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
-    uint8_t *const gen = lq_raw + (base - lq_smem_u32(lq_raw));
+    const uint32_t base = (smem_u32(lq_raw) + 1023u) & ~1023u;  // swizzled tiles want 1024-byte alignment
+    uint8_t *const gen = lq_raw + (base - smem_u32(lq_raw));
     // after the stages: full[8], empty[8], acc_full[2], acc_empty[2] (8 bytes each), the tensor-memory address,
     // then the reciprocal steps of two tiles
     const uint32_t bars = base + NS * STAGE;
@@ -203,17 +187,17 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) {
-            lq_mbar_init(full(s), 1);
-            lq_mbar_init(empty(s), 1);
+            mbar_init(full(s), 1);
+            mbar_init(empty(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
-            lq_mbar_init(acc_full(b), 1);
-            lq_mbar_init(acc_empty(b), 4);  // one arrival per epilogue warp
+            mbar_init(acc_full(b), 1);
+            mbar_init(acc_empty(b), 4);  // one arrival per epilogue warp
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) tc_alloc(lq_smem_u32(tmem_slot), TCOLS);
+    if (warp == 1) tc_alloc(smem_u32(tmem_slot), TCOLS);
     tc_fence_before();
     tpq_grid_dep_wait();  // the operands and the payload buffer may still be in use by the kernel ahead
     __syncthreads();
@@ -234,9 +218,9 @@ linear_quantize(const LQParams p, const __grid_constant__ CUtensorMap map_x, con
                         ok = false;
                         break;
                     }
-                    lq_mbar_expect_tx(full(s), STAGE);
-                    lq_tma_load_2d(base + s * STAGE, &map_x, kb * LQ_BK, m0, full(s));
-                    lq_tma_load_2d(base + s * STAGE + LQ_A_BYTES, &map_w, kb * LQ_BK, n0, full(s));
+                    mbar_expect_tx(full(s), STAGE);
+                    tma_load_2d(base + s * STAGE, &map_x, kb * LQ_BK, m0, full(s));
+                    tma_load_2d(base + s * STAGE + LQ_A_BYTES, &map_w, kb * LQ_BK, n0, full(s));
                 }
             }
             if (!ok)  // giving up: let the copies already issued land before the block's shared memory is released

@@ -77,7 +77,6 @@ __global__ void __launch_bounds__(256) quantize_generic(const uint16_t *__restri
 // ----------------------------------------------------------------------------------------------
 constexpr int QP_MAX_GPT = 4;          // groups of 8 features per thread
 constexpr int QP_MAX_CONSUMERS = 992;  // 31 consumer warps + 1 producer warp per block
-constexpr int QP_WAIT_LIMIT = 1 << 22; // bounded mbarrier polling
 
 constexpr int QP_MAX_BATCH = 16;  // devices' shards quantised by one launch (each by its own set of blocks)
 
@@ -121,43 +120,6 @@ __host__ __device__ inline QPLayout qp_layout(int E, int G, int nstage)
     return l;
 }
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// bounded wait: false if the phase never completed
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    for (int i = 0; i < QP_WAIT_LIMIT; ++i) {
-        uint32_t ok;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(ok)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (ok) return true;
-    }
-    return false;
-}
-// global -> this block's shared memory, bytes a multiple of 16, both addresses 16-byte aligned
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
 
 // One element: product rounded to binary32, clamped, rounded half-to-even by the magic add; returns the
 // bits of fl(u + 1.5*2^23) = 0x4B400000 + code.
