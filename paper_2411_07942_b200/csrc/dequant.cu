@@ -1268,26 +1268,6 @@ cudaError_t launch_panels(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
 }
 
 // ---- tensor maps of the payloads' code sections
-typedef CUresult (*tpq_encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                        const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-tpq_encode_tiled_fn encode_tiled_fn()
-{
-    static tpq_encode_tiled_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<tpq_encode_tiled_fn>(sym);
-        else
-            (void)cudaGetLastError();
-    }
-    return fn;
-}
 
 // A payload's map depends on its address and on the shape; encoding costs about a microsecond of host time,
 // so the maps of recently seen payloads are kept (callers reuse their communication buffers).
@@ -1315,7 +1295,7 @@ bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC,
                 return true;
             }
         }
-    tpq_encode_tiled_fn fn = encode_tiled_fn();
+    tpq_encode_tiled_fn fn = tpq_tensor_map_encoder();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)L8, (cuuint64_t)T};
     const cuuint64_t strides[1] = {(cuuint64_t)L8 * 4};

@@ -365,31 +365,11 @@ __global__ void __launch_bounds__(256) permute_weight(const uint16_t *__restrict
     }
 }
 
-typedef CUresult (*lq_encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-lq_encode_tiled_fn lq_encode_fn()
-{
-    static lq_encode_tiled_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<lq_encode_tiled_fn>(sym);
-        else
-            (void)cudaGetLastError();
-    }
-    return fn;
-}
 
 // [rows][K] BF16, row-major -> boxes of box_rows x 64 elements with the 128-byte swizzle; out-of-range reads give 0
 bool lq_map(const void *ptr, int64_t rows, int64_t K, int box_rows, CUtensorMap *out)
 {
-    lq_encode_tiled_fn fn = lq_encode_fn();
+    tpq_encode_tiled_fn fn = tpq_tensor_map_encoder();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)K * 2};

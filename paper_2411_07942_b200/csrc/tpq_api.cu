@@ -85,6 +85,23 @@ struct StateHeader {
 
 }  // namespace
 
+tpq_encode_tiled_fn tpq_tensor_map_encoder()
+{
+    static tpq_encode_tiled_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<tpq_encode_tiled_fn>(sym);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
 extern "C" {
 
 const char *tpq_version(void) { return "tpq 0.1 (sm_100a)"; }

@@ -1,6 +1,7 @@
 // Internal declarations shared by the translation units of libtpq (not installed).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -111,6 +112,13 @@ cudaError_t tpq_launch_publish_arrivals(uint32_t *const *arrived, int n_dst, uin
 // Bounded wait until n arrival words equal `epoch`; on expiry the context's device status becomes TPQ_ERR_TIMEOUT.
 cudaError_t tpq_launch_wait_arrivals(const tpq_ctx *c, const uint32_t *arrived, int n, uint32_t epoch,
                                      unsigned long long timeout_ns, cudaStream_t st, int64_t *launches);
+
+// cuTensorMapEncodeTiled, looked up once through the runtime (the library does not link the driver API);
+// NULL if the driver does not provide it.
+typedef CUresult (*tpq_encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                        const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                        CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+tpq_encode_tiled_fn tpq_tensor_map_encoder();
 
 // The pre-synchronisation linear layer fused with the compressor (linear.cu): tensor-core GEMM whose epilogue
 // quantises and packs.  w_slots is the [E][K] weight matrix with its rows in slot order (tpq_launch_permute_weight).
