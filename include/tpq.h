@@ -23,7 +23,10 @@
  *   - Arguments are validated before anything is launched; a non-zero status
  *     means nothing was enqueued.  No entry point throws, aborts or traps.
  *   - A context is bound to the CUDA device that was current at tpq_create and
- *     may be used from one host thread at a time.
+ *     may be used from one host thread at a time.  Work enqueued through one
+ *     context must not overlap on the GPU with itself: use one stream, or
+ *     streams ordered by events (the kernels share the context's status word,
+ *     the calibration scratch and the block counter of tpq_quantize_pack_push).
  *   - One context serves all N simulated devices: the static parameters and
  *     the selected feature set are identical on every device by construction
  *     (Section 3: "fixed across all sequences and devices").
