@@ -130,3 +130,53 @@ def test_fused_layer_argument_checks():
     torch.cuda.synchronize()
     t.close()
     t3.close()
+
+
+def test_fused_layer_and_push_on_random_shapes():
+    """Seeded random shapes (E, k, K multiples of 8; any T): the fused layer's payload against the oracle's
+    quantiser on its own BF16 sums, and the pushing quantiser's three copies of the same payload."""
+    orc = oracle.c()
+    rng = np.random.default_rng(411)
+    for case in range(12):
+        E = int(rng.integers(2, 200)) * 8
+        k = int(rng.integers(0, max(1, E // 32) + 1)) * 8
+        if E - k < 8:
+            k = 0
+        T, K, N = int(rng.integers(1, 400)), int(rng.integers(1, 60)) * 8, int(rng.integers(1, 4))
+        x = bf16_bits(rng.normal(0, 1, (T, K)))
+        gain = np.exp(rng.normal(0, 0.7, E))
+        w = bf16_bits(rng.normal(0, 1, (E, K)) * (gain[:, None] / np.sqrt(K)))
+        y_ref = oracle_np.linear_bf16(x, w)
+        yv = oracle_np.widen(y_ref)
+        t = binding.Tpq(N, E)
+        t.set_ranges(np.tile(0.8 * yv.min(axis=0), (N, 1)), np.tile(0.8 * yv.max(axis=0), (N, 1)), np.ones(N, np.int64))
+        hp = t.select_features(k)
+        _, inv = t.get_scales()
+        order = np.concatenate([oracle_np.lp_index(E, hp), np.asarray(hp, np.int64)]).astype(np.int64)
+        shard = N - 1
+        ws = torch.zeros((E, K), dtype=torch.int16, device="cuda")
+        t.permute_weight(gu.dev_bf16(w).data_ptr(), K, ws.data_ptr())
+        P = t.payload_bytes(T)
+        whole, view = gu.guarded(P)
+        ywhole, yview = gu.guarded(T * E * 2)
+        t.linear_quantize_pack(shard, gu.dev_bf16(x).data_ptr(), ws.data_ptr(), T, K, view.data_ptr(), P,
+                               y_slots_ptr=yview.data_ptr())
+        torch.cuda.synchronize()
+        tag = (case, N, T, K, E, k)
+        assert t.device_status() == 0, tag
+        assert gu.guards_intact(whole, P) and gu.guards_intact(ywhole, T * E * 2), tag
+        y_k = np.empty((T, E), np.uint16)
+        y_k[:, order] = yview.cpu().numpy().view(np.uint16).reshape(T, E)
+        want = orc.quantize_pack(y_k, hp, inv[shard])
+        assert np.array_equal(view.cpu().numpy(), want), tag
+        assert (y_k != y_ref).mean() < 0.02, tag
+        bufs = [gu.guarded(P) for _ in range(3)]
+        words = torch.zeros(3, dtype=torch.int32, device="cuda")
+        t.quantize_pack_push(shard, gu.dev_bf16(y_k).data_ptr(), T, [v.data_ptr() for _, v in bufs],
+                             [words.data_ptr() + 4 * d for d in range(3)], P, 9)
+        torch.cuda.synchronize()
+        assert t.device_status() == 0, tag
+        for wh, v in bufs:
+            assert gu.guards_intact(wh, P) and np.array_equal(v.cpu().numpy(), want), tag
+        assert bool((words == 9).all()), tag
+        t.close()
