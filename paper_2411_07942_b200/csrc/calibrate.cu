@@ -38,7 +38,7 @@ constexpr uint32_t KEY_MAX2 = 0x7FFF7FFFu;  // identity of min
 constexpr uint32_t KEY_MIN2 = 0x80008000u;  // identity of max
 
 // Tiled extremes: thread = 8 adjacent features (one 128-bit load per row), 8 row lanes per block,
-// four independent loads in flight per thread.  grid = (feature chunks of 256, row splits, sequences).
+// eight independent loads in flight per thread.  grid = (feature chunks of 256, row splits, sequences).
 __global__ void __launch_bounds__(256) colminmax_tiled(const uint16_t *__restrict__ y, int64_t S, int64_t stride, int E,
                                                        int n_split, int16_t *__restrict__ part_lo,
                                                        int16_t *__restrict__ part_hi)
@@ -57,6 +57,21 @@ __global__ void __launch_bounds__(256) colminmax_tiled(const uint16_t *__restric
     if (live) {
         const uint16_t *col = y + q * S * stride + 8 * (int64_t)g;
         int64_t r = r0 + ty;
+        for (; r + 56 < r1; r += 64) {  // eight independent 128-bit loads in flight per thread
+            uint4 v[8];
+#pragma unroll
+            for (int a = 0; a < 8; ++a) v[a] = __ldcs(reinterpret_cast<const uint4 *>(col + (r + 8 * a) * stride));
+#pragma unroll
+            for (int a = 0; a < 8; ++a) {
+                const uint32_t w[4] = {v[a].x, v[a].y, v[a].z, v[a].w};
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    uint32_t kk = key2(w[b]);
+                    lo[b] = min_s16x2(lo[b], kk);
+                    hi[b] = max_s16x2(hi[b], kk);
+                }
+            }
+        }
         for (; r + 24 < r1; r += 32) {
             uint4 v0 = __ldcs(reinterpret_cast<const uint4 *>(col + r * stride));
             uint4 v1 = __ldcs(reinterpret_cast<const uint4 *>(col + (r + 8) * stride));
