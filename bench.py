@@ -403,7 +403,37 @@ def main():
 
     wd_ms = time_loop(wd_only, reps)
 
-    # ---- the layer ahead of the synchronisation point fused with the compressor (Section 2): x [T][K] times the
+    # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
+    # what the launch path costs, relevant for the decode-sized workloads
+    graph_ms = None
+    try:
+        gs = torch.cuda.Stream()
+        gs.wait_stream(stream)
+        gsh = gs.cuda_stream
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=gs):
+            for b in range(args.sets):
+                _, _, out, yarr, parr = sets[b]
+                t.quantize_pack_batch(0, yarr, T, parr, P, stream=gsh)
+                t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=gsh)
+        with torch.cuda.stream(gs):
+            for _ in range(3):
+                graph.replay()
+            ga, gz = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            greps = max(5, min(args.steps, 2000) // args.sets)
+            ga.record(gs)
+            for _ in range(greps):
+                graph.replay()
+            gz.record(gs)
+        torch.cuda.synchronize()
+        graph_ms = ga.elapsed_time(gz) / (greps * args.sets)
+    except Exception as exc:  # measurement only: the step itself does not depend on graphs
+        graph_ms = f"unavailable: {type(exc).__name__}: {exc}"[:200]
+        torch.cuda.synchronize()
+    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
+
+    # ---- (after the clock sampler has stopped: this part is tensor-bound and draws far more power than the path)
+    # the layer ahead of the synchronisation point fused with the compressor (Section 2): x [T][K] times the
     # device's slice of the down projection, K = 2.7 E / N rounded to 64 (Llama's 13824 / 4 at E = 5120), against
     # the library GEMM followed by quantize_pack.  Tensor-bound; an extra, not the headline path.
     fused = None
@@ -435,34 +465,6 @@ def main():
         fused = {"shape": f"x [{T}][{Kd}] . w [{E}][{Kd}]^T", "fused_ms": f_ms, "fused_TFLOPs": flops / f_ms / 1e9,
                  "frac_of_" + tkind + "_bf16_peak": flops / f_ms / 1e9 / tpeak, "peak_TFLOPs": tpeak,
                  "library_gemm_then_quantize_pack_ms": u_ms, "library_gemm_alone_ms": g_ms}
-    # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
-    # what the launch path costs, relevant for the decode-sized workloads
-    graph_ms = None
-    try:
-        gs = torch.cuda.Stream()
-        gs.wait_stream(stream)
-        gsh = gs.cuda_stream
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=gs):
-            for b in range(args.sets):
-                _, _, out, yarr, parr = sets[b]
-                t.quantize_pack_batch(0, yarr, T, parr, P, stream=gsh)
-                t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=gsh)
-        with torch.cuda.stream(gs):
-            for _ in range(3):
-                graph.replay()
-            ga, gz = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            greps = max(5, min(args.steps, 2000) // args.sets)
-            ga.record(gs)
-            for _ in range(greps):
-                graph.replay()
-            gz.record(gs)
-        torch.cuda.synchronize()
-        graph_ms = ga.elapsed_time(gz) / (greps * args.sets)
-    except Exception as exc:  # measurement only: the step itself does not depend on graphs
-        graph_ms = f"unavailable: {type(exc).__name__}: {exc}"[:200]
-        torch.cuda.synchronize()
-    clocks = sampler.stop(wall0, wall1) if rank == 0 else None
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
     ys0 = sets[0][0]
