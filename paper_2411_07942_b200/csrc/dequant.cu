@@ -82,28 +82,38 @@ __global__ void __launch_bounds__(256) dequant_generic(const DQParams p)
 //   - selected feature hp_idx[h], h < k: the sum of the devices' BF16 values.
 // ----------------------------------------------------------------------------------------------
 
-__device__ __host__ constexpr int dq_pos(int n) { return n < 5 ? n : n - 5; }
+__device__ __host__ constexpr int dq_pos(int n) { return n & 3; }
 
 // 8 two's-complement codes of `raw` times their steps, accumulated.  The codes are decoded in place:
 // (x & 0xF << 4n) | 0x4B000000 is the float 2^23 + (code+8) 16^n; subtracting 2^23 + 8*16^n leaves
 // code * 16^n exactly, and the step was pre-divided by 16^n (an exact scaling), so
-// fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 5..7 use raw >> 20.
-// Subtractions and FMAs run two at a time (f32x2), one binary32 rounding per element as before.
-// -(2^23 + 8 * 16^pos) for the code pairs (0,1) (2,3) (4,5) (6,7); in constant memory so that the packed
-// subtract can take the pair as an operand instead of rebuilding it in registers
-__constant__ float2 kDecodeBias[4] = {{-8388616.0f, -8388736.0f},      // 16^0, 16^1
-                                      {-8390656.0f, -8421376.0f},      // 16^2, 16^3
-                                      {-8912896.0f, -8388616.0f},      // 16^4, 16^0 (codes 5..7 use raw >> 20)
-                                      {-8388736.0f, -8390656.0f}};     // 16^1, 16^2
-
+// fma(code*16^n, s/16^n, acc) rounds exactly like fma(code, s, acc).  Codes 0..3 are taken from the low
+// half of the word, codes 4..7 from the word shifted down by 16, both at positions 0..3, so that four
+// masks and two bias pairs serve all eight.  Subtractions and FMAs run two at a time (f32x2), one binary32
+// rounding per element as before.
+//
 // Each code costs ONE logic instruction only if the mask and the exponent pattern are both register
-// operands of an explicit lop3 ((x & mask) | magic, truth table 0xEA): written in C with immediates the
-// compiler emits two.  `magic` holds 0x4B000000 (see opaque_magic).
-__device__ __forceinline__ uint32_t opaque_magic()
+// operands of an explicit lop3 ((x & mask) | magic, truth table 0xEA), and the packed subtract takes its
+// bias pair from registers: the constants are made opaque to the compiler once per thread (DecodeConsts),
+// which otherwise rebuilds them from immediates at every use.
+struct DecodeConsts {
+    uint32_t mask[4];  // 0xF << 4n
+    uint32_t magic;    // 0x4B000000
+    float2 bias[2];    // -(2^23 + 8 * 16^n) for positions (0,1) and (2,3)
+};
+__device__ __forceinline__ DecodeConsts decode_consts()
 {
-    uint32_t m;
-    asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(m));
-    return m;
+    DecodeConsts c;
+    asm volatile("mov.u32 %0, 0xF;" : "=r"(c.mask[0]));
+    asm volatile("mov.u32 %0, 0xF0;" : "=r"(c.mask[1]));
+    asm volatile("mov.u32 %0, 0xF00;" : "=r"(c.mask[2]));
+    asm volatile("mov.u32 %0, 0xF000;" : "=r"(c.mask[3]));
+    asm volatile("mov.u32 %0, 0x4B000000;" : "=r"(c.magic));
+    asm volatile("mov.f32 %0, 0fCB000008;" : "=f"(c.bias[0].x));  // -(2^23 + 8)
+    asm volatile("mov.f32 %0, 0fCB000080;" : "=f"(c.bias[0].y));  // -(2^23 + 128)
+    asm volatile("mov.f32 %0, 0fCB000800;" : "=f"(c.bias[1].x));  // -(2^23 + 2048)
+    asm volatile("mov.f32 %0, 0fCB008000;" : "=f"(c.bias[1].y));  // -(2^23 + 32768)
+    return c;
 }
 __device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t mask, uint32_t magic)
 {
@@ -112,19 +122,20 @@ __device__ __forceinline__ uint32_t and_or(uint32_t x, uint32_t mask, uint32_t m
     return d;
 }
 
-__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], uint32_t magic,
-                                        const float2 (&bias)[4] = kDecodeBias)
+// FIRST: the accumulators start here, acc = code * step (what fma(code, step, +0) gives: a product that is
+// zero has a +0 code, except at a hole's lane, whose step is 0 and whose sum is never kept).
+template <bool FIRST = false>
+__device__ __forceinline__ void decode8(uint32_t raw, const float2 (&sc)[4], float2 (&acc)[4], const DecodeConsts &c)
 {
     const uint32_t xa = raw ^ 0x88888888u;
-    const uint32_t xb = xa >> 20;
+    const uint32_t xb = xa >> 16;
 #pragma unroll
     for (int h = 0; h < 4; ++h) {
-        const int n0 = 2 * h, n1 = 2 * h + 1;
-        const uint32_t x0 = (n0 < 5) ? xa : xb, x1 = (n1 < 5) ? xa : xb;
-        const float f0 = __uint_as_float(and_or(x0, 0xFu << (4 * dq_pos(n0)), magic));
-        const float f1 = __uint_as_float(and_or(x1, 0xFu << (4 * dq_pos(n1)), magic));
-        const float2 d = __fadd2_rn(make_float2(f0, f1), bias[h]);
-        acc[h] = __ffma2_rn(d, sc[h], acc[h]);
+        const uint32_t x = (h < 2) ? xa : xb;
+        const float f0 = __uint_as_float(and_or(x, c.mask[2 * (h & 1)], c.magic));
+        const float f1 = __uint_as_float(and_or(x, c.mask[2 * (h & 1) + 1], c.magic));
+        const float2 d = __fadd2_rn(make_float2(f0, f1), c.bias[h & 1]);
+        acc[h] = FIRST ? __fmul2_rn(d, sc[h]) : __ffma2_rn(d, sc[h], acc[h]);
     }
 }
 
@@ -370,13 +381,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
         dp_steps[(2 * i) * CG + c] = make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y);
         dp_steps[(2 * i + 1) * CG + c] = make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y);
     }
-    const uint32_t magic = opaque_magic();
-    float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        bias[h] = kDecodeBias[h];
-        asm volatile("" : "+f"(bias[h].x), "+f"(bias[h].y));
-    }
+    const DecodeConsts dc = decode_consts();
 
     // consume side: word of (device i of the step, this thread's row r) inside a stage
     int wofs[DP_R];
@@ -507,7 +512,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                     const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                           make_float2(b.z, b.w)};
 #pragma unroll
-                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                    for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], dc);
                 }
             } else {
 #pragma unroll
@@ -517,7 +522,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
                         const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                               make_float2(b.z, b.w)};
 #pragma unroll
-                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], dc);
                     }
             }
         }
@@ -607,13 +612,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     const int cg = tid & (CG - 1), rs = tid / CG;
-    const uint32_t magic = opaque_magic();
-    float2 bias[4];  // the decode biases in registers (the packed subtract takes no constant-bank pair)
-#pragma unroll
-    for (int h = 0; h < 4; ++h) {
-        bias[h] = kDecodeBias[h];
-        asm volatile("" : "+f"(bias[h].x), "+f"(bias[h].y));
-    }
+    const DecodeConsts dc = decode_consts();
     const float4 *const my_steps = dp_steps + cg;
     const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R) * CG + cg;
     // ring state: the producer lane and the main warps walk the same sequence of stages across segments
@@ -743,7 +742,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                         const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                               make_float2(b.z, b.w)};
 #pragma unroll
-                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                        for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], dc);
                     }
                 } else {
 #pragma unroll
@@ -753,7 +752,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                             const float2 sc[4] = {make_float2(a.x, a.y), make_float2(a.z, a.w), make_float2(b.x, b.y),
                                                   make_float2(b.z, b.w)};
 #pragma unroll
-                            for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], magic, bias);
+                            for (int r = 0; r < DP_R; ++r) decode8(w[i][r], sc, acc[r], dc);
                         }
                 }
             }
@@ -786,35 +785,44 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 // ----------------------------------------------------------------------------------------------
 // Row kernel for N <= 4 devices and (E-k)/8 <= MAXT main threads.
 //
-// One persistent block per SM with three kinds of warps:
-//   producer (1 warp)  streams groups of G rows of all N payloads (a code-row block and a BF16 block per
-//                      device, 2N 1-D bulk asynchronous copies issued by 2N lanes) into a ring of
-//                      shared-memory stages; completion on "full" mbarriers;
+// One persistent block per SM works on a run of adjacent rows, G at a time, with three kinds of warps:
+//   producer (1 warp)  sets up the barriers, waits for the kernel ahead in the stream and streams the
+//                      stages (a code-row block and a BF16 block per device, 2N 1-D bulk asynchronous
+//                      copies issued by 2N lanes) into a ring of shared-memory stages; "full" mbarriers;
 //   main (MAXT/32)     thread <-> 8 adjacent output features = one aligned word per device and row; its
-//                      N x 8 steps live in registers for the life of the block (0 at holes); pure
-//                      decode + 128-bit row stores, two rows at a time, no hole logic at all; arrives on
-//                      "main_done" (release: its stores are ordered before what follows the barrier);
-//   fix-up (4 warps)   after "main_done": one item per selected feature and row -- the sum of the
-//                      devices' BF16 values goes to the selected feature's column (overwriting the 0 the
-//                      main store left at a hole), and, for a hole, the filler feature whose codes the
-//                      hole's slot holds is decoded and stored to the filler's column.
-// Main and fix-up warps release a stage through the "empty" mbarrier; no block-wide barrier in the loop.
-// G is a multiple of 4/gcd(4, L/8) so that every stage starts 16-byte aligned in the code stream.
+//                      N x 8 steps live in registers for the life of the block (0 at holes); straight-line
+//                      decode + one 128-bit store per row.  A thread whose group contains a selected
+//                      feature then overwrites that lane of its own stores (same thread, same address:
+//                      ordered) with the sum the auxiliary warps left in shared memory;
+//   auxiliary (3)      per stage, from shared memory only: (1) the sums of the devices' BF16 values of every
+//                      (row, selected feature), two adjacent ranks per thread, left in shared memory in
+//                      the output's format ("sums" barrier); (2) the last k columns of the output, which no
+//                      main thread covers: an unselected one is a filler feature, decoded from the hole's
+//                      slot that carries its codes, a selected one takes its sum; lane <-> column, so the
+//                      small stores of a warp are adjacent.
+// No warp ever waits for another one's global stores, and no block-wide barrier follows the prologue.
+// Blocks and stages start on rows at which the code stream is 16-byte aligned (multiples of 4/gcd(4, L/8)).
 // ----------------------------------------------------------------------------------------------
-// fix-up threads: 128, or 96 where that takes the block from 25 warps (allocated as 28: 72 registers per
-// thread) to 24 (80 registers) and two rows per stage leave few items
-constexpr int DR_FIXUP_MAX = 128;
+constexpr int DR_AUX = 96;          // auxiliary threads
+constexpr int DR_PREFETCH_ROWS = 4; // rows whose bytes a block asks L2 for ahead of the dependency wait (measured: 2..8 alike, all: worse)
+
+// main threads (= 32-bit words of a code row a stage leaves room for) for a row of L8 words
+__host__ __device__ inline int dr_row_cap(int L8) { return L8 <= 640 ? 640 : 768; }
 
 struct DRLayout {
-    size_t lp_stage, hp_stage, stage, bars, total;
+    size_t lp_stage, hp_stage, stage, sums, sums_stage, bars, total;
 };
 __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int nstage)
 {
     DRLayout l;
-    l.lp_stage = (((size_t)G * (E - k) / 2) + 15) & ~(size_t)15;
+    // a device's code rows of a stage start at a stride that depends on G only (the widest row the main
+    // threads cover), so that the main loop addresses them with immediate offsets
+    l.lp_stage = (size_t)G * dr_row_cap((E - k) >> 3) * 4;
     l.hp_stage = (size_t)G * k * 2;
     l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
-    l.bars = (size_t)nstage * l.stage;
+    l.sums = (size_t)nstage * l.stage;
+    l.sums_stage = (((size_t)G * k * 4) + 15) & ~(size_t)15;  // one 32-bit slot per (row, rank)
+    l.bars = l.sums + (size_t)nstage * l.sums_stage;
     l.total = l.bars + (size_t)nstage * 24;
     return l;
 }
@@ -823,87 +831,167 @@ struct DRParams {
     DQParams q;
     DXParams x;
     int G, nstage;
-    int64_t ngroups;
-#ifdef TPQ_TRACE
-    long long *trace;
-#endif
+    int first;               // rows of a block's first stage (<= G: a short first stage lands sooner)
+    int64_t rows_per_block;  // a block works on rows_per_block adjacent rows (a multiple of the number of
+                             // rows after which the code stream is 16-byte aligned again)
 };
 
-#ifdef TPQ_TRACE
-static long long *g_dtrace = nullptr;  // 64 slots per block, globaltimer ns
-__device__ __forceinline__ long long tpq_dnow()
+__device__ __forceinline__ uint32_t lds32(uint32_t saddr)
 {
-    long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(saddr) : "memory");
+    return v;
 }
-#define TPQ_DMARK(slot) do { if (threadIdx.x == 0 && pp.trace && (slot) < 64) pp.trace[blockIdx.x * 64 + (slot)] = tpq_dnow(); } while (0)
-#else
-#define TPQ_DMARK(slot) do { } while (0)
-#endif
+__device__ __forceinline__ uint32_t lds16(uint32_t saddr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts64(uint32_t saddr, uint32_t a, uint32_t b)
+{
+    asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(saddr), "r"(a), "r"(b) : "memory");
+}
+__device__ __forceinline__ void sts32(uint32_t saddr, uint32_t a)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(saddr), "r"(a) : "memory");
+}
 
-template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
-__global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams pp)
+// the bits an output element holds for the sum v
+template <bool FP32OUT>
+__device__ __forceinline__ uint32_t out_bits(float v)
+{
+    if (FP32OUT) return __float_as_uint(v);
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
+}
+template <bool FP32OUT>
+__device__ __forceinline__ void store_bits(uint8_t *ptr, uint32_t bits)
+{
+    if (FP32OUT)
+        *reinterpret_cast<uint32_t *>(ptr) = bits;
+    else
+        *reinterpret_cast<uint16_t *>(ptr) = (uint16_t)bits;
+}
+// the code in bits [sh, sh+4) of w, as a float
+__device__ __forceinline__ float code_at(uint32_t w, int sh)
+{
+    return __fsub_rn(__uint_as_float((((w >> sh) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
+}
+
+// GR rows of a stage for one main thread.  sa: shared-memory address of its word of the first row of
+// device 0; device i's copy of a row lies DEVSTEP bytes further on each (a compile-time constant, so the
+// device's word is one load at an immediate offset; 0: dev_step, known at run time only); a row is
+// row_bytes long.  NDEV > 0: the number of devices, known at compile time; 0: n (1 <= n <= NMAX) devices.
+template <int NMAX, int NDEV, int GR, uint32_t DEVSTEP, bool FP32OUT, bool HAS_BIAS>
+__device__ __forceinline__ void rows_stage(uint32_t sa, uint32_t dev_step, uint32_t row_bytes, int n,
+                                           const float2 (&sc)[NMAX][4], const DecodeConsts &dc, const float2 (&b)[4],
+                                           uint8_t *orow, int64_t out_row_bytes, bool live)
+{
+#pragma unroll
+    for (int r = 0; r < GR; ++r) {
+        float2 acc[4];
+        decode8<true>(lds32(sa), sc[0], acc, dc);
+#pragma unroll
+        for (int i = 1; i < NMAX; ++i)
+            if (NDEV ? i < NDEV : i < n) decode8(lds32(sa + (uint32_t)i * (DEVSTEP ? DEVSTEP : dev_step)), sc[i], acc, dc);
+        sa += row_bytes;
+        if (live) {
+            if (HAS_BIAS) {  // (a hole's lane gets its own column's bias here and is overwritten below)
+#pragma unroll
+                for (int h = 0; h < 4; ++h) acc[h] = __fadd2_rn(acc[h], b[h]);
+            }
+            store_group<FP32OUT>(orow, 0, acc, 0u);
+        }
+        orow += out_row_bytes;
+    }
+}
+
+// Marks a value loaded once per thread as opaque: without it the compiler, short of registers, drops the value
+// and repeats its chain of (read-only) table loads at every use inside the stage loop, a trip to L2 each time.
+__device__ __forceinline__ void keep(int &v) { asm volatile("" : "+r"(v)); }
+__device__ __forceinline__ void keep(uint32_t &v) { asm volatile("" : "+r"(v)); }
+__device__ __forceinline__ void keep(float &v) { asm volatile("" : "+f"(v)); }
+
+// first row (within the block's run) of the block's it-th stage
+__device__ __forceinline__ int dr_stage_row(int it, int first, int G) { return it == 0 ? 0 : first + (it - 1) * G; }
+
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+__global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRParams pp)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    TPQ_DMARK(0);
     const DQParams &p = pp.q;
     const DXParams &x = pp.x;
     const int tid = threadIdx.x;
-    const int NT = blockDim.x - FX - 32;  // main threads; then the fix-up warps; then the producer warp
-    const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;  // G rows per stage, even
+    // warp 0 is the producer, then the auxiliary warps, then the main warps: where several warps of a
+    // scheduler can issue, the one launched first goes first, and the few instructions of the producer and of
+    // the auxiliary warps must not wait behind the main warps' many (as last warps they took 3 us per stage)
+    const int NT = blockDim.x - DR_AUX - 32;  // main threads
+    const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;
     const int L = E - k, L8 = L >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
     uint64_t *empty = full + nstage;
-    uint64_t *main_done = empty + nstage;
+    uint64_t *sums_ready = empty + nstage;
+    // this block's rows
+    const int64_t t_begin = blockIdx.x * pp.rows_per_block;
+    const int64_t t_end = (p.T - t_begin < pp.rows_per_block) ? p.T : t_begin + pp.rows_per_block;
+    const int rows_mine = (int)(t_end - t_begin);
+    constexpr int ESIZE = FP32OUT ? 4 : 2;
+    const int64_t out_row_bytes = p.out_stride * ESIZE;
+    const uint32_t smem_s = smem_u32(smem);
+    const uint32_t stage_b = (uint32_t)lay.stage, lp_b = (uint32_t)lay.lp_stage, hp_b = (uint32_t)lay.hp_stage;
+    const uint32_t sums_s = smem_s + (uint32_t)lay.sums, sums_b = (uint32_t)lay.sums_stage;
 
-    // (first thing, with no load of its own in flight: behind the table loads below it would make every
-    // thread wait for them ahead of the barrier that releases the producer; and an instantiation of its
-    // own: even a branch that is never taken costs this prologue a few hundred cycles)
-    if constexpr (HAS_WAIT) tpq_block_wait_arrivals(p.arr);
-    if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) {
-            mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), (NT + FX) / 32);
-            mbar_init(smem_u32(&main_done[s]), NT / 32);
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // Order of the prologue.  The producer warp sets up the barriers, waits for the kernel ahead in the stream
+    // and issues the first stages' copies at once: the other warps' table loads then run in the shadow of the
+    // first stage's flight instead of ahead of it.  Only the producer executes griddepcontrol.wait: every
+    // other access to the payloads, and every store to the output, follows a "full" barrier that one of the
+    // producer's copies completes, i.e. follows that wait.
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue as SMs free up
+    if constexpr (HAS_WAIT) {  // (an instantiation of its own: the plain call's prologue stays short)
+        tpq_block_wait_arrivals(p.arr);
+        __syncthreads();
     }
-
-    // main-thread constants: loads issued before the barrier that releases the producer (so that they
-    // are not queued behind the bulk copies)
-    const int g = tid;
-    const bool is_main = tid < NT;
-    const bool live = is_main && g < L8;
-    const int g_ld = live ? g : 0;
-    float2 sc[NMAX][4];
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) {
-#pragma unroll
-        for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
-        if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
-    }
-    tpq_grid_dep_wait();    // the payloads and the output buffer may still be in use by the kernel ahead
-    __syncthreads();
-    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
-
-    if (tid >= NT + FX) {
+    if (tid < 32) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
         // copies of the stage are issued by 2N lanes at once
-        const int pl = tid - NT - FX;
+        const int pl = tid;
+        if (pl == 0) {
+            for (int s = 0; s < nstage; ++s) {
+                mbar_init(smem_u32(&full[s]), 1);
+                mbar_init(smem_u32(&empty[s]), (NT + DR_AUX) / 32);
+                mbar_init(smem_u32(&sums_ready[s]), DR_AUX / 32);
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncwarp();
+        asm volatile("bar.arrive 1, %0;" ::"r"(blockDim.x) : "memory");  // the barriers exist
+        if (pl < 2 * N) {
+            // the block's first rows may start their way from HBM to L2 while it waits (a hint only: L2 is the
+            // point of coherence, so whatever the kernel ahead still writes is what the copies will read)
+            const int rows = rows_mine < DR_PREFETCH_ROWS ? rows_mine : DR_PREFETCH_ROWS;
+            const int i = pl >> 1;
+            if ((pl & 1) == 0)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.pl[i] + t_begin * ((E - k) / 2)),
+                             "r"((uint32_t)((((size_t)rows * (E - k) / 2) + 15) & ~(size_t)15)) : "memory");
+            else if (k)
+                asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p.pl[i] + p.lp_bytes + t_begin * k * 2),
+                             "r"((uint32_t)rows * k * 2u) : "memory");
+        }
+        tpq_grid_dep_wait();  // the payloads and the output buffer may still be in use by the kernel ahead
         int st = 0;
         uint32_t parity = 1;  // parity of the "empty" phase to wait for
         for (int it = 0;; ++it) {
-            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-            if (gi >= pp.ngroups) break;
-            const int64_t t0 = gi * G;
-            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+            const int r0 = dr_stage_row(it, pp.first, G);
+            if (r0 >= rows_mine) break;
+            const int cap = it == 0 ? pp.first : G;
+            const int rows = rows_mine - r0 < cap ? rows_mine - r0 : cap;
+            const int64_t t0 = t_begin + r0;
             const uint32_t lp_bytes = (uint32_t)((((size_t)rows * (E - k) / 2) + 15) & ~(size_t)15);
             const uint32_t hp_bytes = (uint32_t)rows * k * 2u;
             const uint32_t bar = smem_u32(&full[st]);
-            uint8_t *stage = smem + (size_t)st * lay.stage;
+            const uint32_t stage = smem_s + (uint32_t)st * stage_b;
             int ok = 1;
             if (pl == 0) {
                 if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
@@ -918,10 +1006,9 @@ __global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams
             for (int c = pl; c < 2 * N; c += 32) {
                 const int i = c >> 1;
                 if ((c & 1) == 0)
-                    bulk_g2s(smem_u32(stage + (size_t)i * lay.lp_stage), p.pl[i] + t0 * ((E - k) / 2), lp_bytes, bar);
+                    bulk_g2s(stage + (uint32_t)i * lp_b, p.pl[i] + t0 * ((E - k) / 2), lp_bytes, bar);
                 else if (hp_bytes)
-                    bulk_g2s(smem_u32(stage + (size_t)N * lay.lp_stage + (size_t)i * lay.hp_stage),
-                             p.pl[i] + p.lp_bytes + t0 * k * 2, hp_bytes, bar);
+                    bulk_g2s(stage + (uint32_t)N * lp_b + (uint32_t)i * hp_b, p.pl[i] + p.lp_bytes + t0 * k * 2, hp_bytes, bar);
             }
             if (++st == nstage) {
                 st = 0;
@@ -931,107 +1018,119 @@ __global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams
         return;
     }
 
-    const int lane = tid & 31;
     int st = 0;
     uint32_t parity = 0;
+    const int lane = tid & 31;
 
-    if (!is_main) {
-        // ---------------- fix-up warps
-        // A thread's items of a stage are the same (row of the stage, rank) pairs in every stage, so their
-        // columns, slots and steps are loaded once; sums are formed as soon as the stage has landed (they
-        // read shared memory only) and stored once the main warps' row stores are done.
-        const int ft = tid - NT;
-        constexpr int FX_PRE = 2;  // items per thread kept in registers (more: the plain loop below)
-        int f_r[FX_PRE], f_h[FX_PRE], f_hpcol[FX_PRE], f_col[FX_PRE], f_word[FX_PRE], f_sh[FX_PRE];
-        float f_s[FX_PRE][NMAX], f_bh[FX_PRE], f_bf[FX_PRE];
+    if (tid < 32 + DR_AUX) {
+        // ---------------- auxiliary warps
+        // Thread c works on the c-th selected feature (its sum) and on column L + c of the output, row by
+        // row, in short rolled loops: these warps run code that nobody else runs, once per stage, so
+        // straight-line code would pay an instruction fetch for every few instructions it executes.
+        // What a thread needs from the tables is loaded once (feature sets with more than DR_AUX selected
+        // features: further chunks of DR_AUX, with the tables read where they are used).
+        const int at = tid - 32;
+        const bool on = at < k;
+        const int col = L + (on ? at : 0);
+        const int ps = on ? __ldg(p.pos + col) : 0;
+        // the column's code sits at bits [sh, sh + 4) of a word of the hole's slot that carries it; it is
+        // decoded in place like the main threads' codes (mask, exponent pattern, bias and a step divided by
+        // the code's position), from the word shifted down by 16 for the upper four positions
+        const int slot = ps >= 0 ? ps : 0;
+        int sel = ps < 0;
+        uint32_t c_off = (uint32_t)(slot >> 3) * 4u;                    // the word inside a code row
+        uint32_t c_sum = ps < 0 ? (uint32_t)(-ps - 1) * 4u : 0u;        // a selected column's sum inside a row of sums
+        const int sh = (slot & 7) * 4, shl = sh & 15;
+        uint32_t c_hi = sh >= 16 ? 16u : 0u, c_mask = 0xFu << shl;
+        float c_nb = -(8388608.0f + (float)(8 << shl));
+        float c_s[NMAX];
 #pragma unroll
-        for (int j = 0; j < FX_PRE; ++j) {
-            const int item = ft + j * FX;
-            const bool on = item < G * k;
-            f_r[j] = on ? item / k : -1;
-            f_h[j] = on ? item - f_r[j] * k : 0;
-            f_hpcol[j] = on ? __ldg(x.hp_idx + f_h[j]) : 0;
-            const bool hole = on && f_h[j] < x.n_holes;
-            f_col[j] = hole ? __ldg(x.filler + f_h[j]) : -1;
-            const int slot = hole ? __ldg(x.hole + f_h[j]) : 0;
-            f_word[j] = f_r[j] * L8 + (slot >> 3);
-            f_sh[j] = (slot & 7) * 4;
+        for (int i = 0; i < NMAX; ++i)
+            c_s[i] = (on && ps >= 0 && i < N) ? __ldg(p.s_k + (size_t)i * E + col) * (1.0f / (float)(1 << shl)) : 0.0f;
+        float c_b = (HAS_BIAS && on && ps >= 0) ? __ldg(p.bias + col) : 0.0f;
+        float h_b = (HAS_BIAS && on) ? __ldg(p.bias + __ldg(x.hp_idx + at)) : 0.0f;
+        keep(sel); keep(c_off); keep(c_sum); keep(c_hi); keep(c_mask); keep(c_nb); keep(c_b); keep(h_b);
 #pragma unroll
-            for (int i = 0; i < NMAX; ++i) f_s[j][i] = (hole && i < N) ? __ldg(p.s_k + (size_t)i * E + f_col[j]) : 0.0f;
-            // (the items' biases with them: fetched in the store phase they would sit between "main_done" and
-            // the release of the stage)
-            f_bh[j] = (HAS_BIAS && on) ? __ldg(p.bias + f_hpcol[j]) : 0.0f;
-            f_bf[j] = (HAS_BIAS && hole) ? __ldg(p.bias + f_col[j]) : 0.0f;
-        }
-        const int hp_dev = (int)(lay.hp_stage / 2);  // BF16 elements between two devices' blocks
+        for (int i = 0; i < NMAX; ++i) keep(c_s[i]);
+        uint32_t magic = 0x4B000000u;
+        keep(magic);
+        const uint32_t kb2 = (uint32_t)k * 2u, kb4 = (uint32_t)k * 4u, row_b = (uint32_t)L8 * 4u;
+        asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");
         for (int it = 0;; ++it) {
-            const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-            if (gi >= pp.ngroups) break;
+            const int r0 = dr_stage_row(it, pp.first, G);
+            if (r0 >= rows_mine) break;
+            const int cap = it == 0 ? pp.first : G;
+            const int rows = rows_mine - r0 < cap ? rows_mine - r0 : cap;
             if (!mbar_wait(smem_u32(&full[st]), parity)) {
                 atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
                 break;
             }
-            const int64_t t0 = gi * G;
-            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-            const uint8_t *stage = smem + (size_t)st * lay.stage;
-            const uint16_t *hp = reinterpret_cast<const uint16_t *>(stage + (size_t)N * lay.lp_stage);
-            float hv[FX_PRE], fv[FX_PRE];
-#pragma unroll
-            for (int j = 0; j < FX_PRE; ++j) {
-                hv[j] = 0.0f;
-                fv[j] = 0.0f;
-                if (f_r[j] >= 0 && f_r[j] < rows) {
+            const uint32_t stage = smem_s + (uint32_t)st * stage_b;
+            const uint32_t hp_s = stage + (uint32_t)N * lp_b;  // device 0's BF16 rows
+            const uint32_t sums = sums_s + (uint32_t)st * sums_b;
+            // (1) the sums of the selected features
+            if (on) {
+                uint32_t a = hp_s + (uint32_t)at * 2u, o = sums + (uint32_t)at * 4u;
+#pragma unroll 1
+                for (int r = 0; r < rows; ++r, a += kb2, o += kb4) {
+                    float v = 0.0f;
 #pragma unroll
                     for (int i = 0; i < NMAX; ++i)
-                        if (i < N) hv[j] = __fadd_rn(hv[j], __uint_as_float((uint32_t)hp[i * hp_dev + f_r[j] * k + f_h[j]] << 16));
-                    if (f_col[j] >= 0) {  // the hole's slot holds the codes of filler feature f_h
-#pragma unroll
-                        for (int i = 0; i < NMAX; ++i)
-                            if (i < N) {
-                                const uint32_t w = reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[f_word[j]];
-                                const float code =
-                                    __fsub_rn(__uint_as_float((((w >> f_sh[j]) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
-                                fv[j] = __fmaf_rn(code, f_s[j][i], fv[j]);
-                            }
-                    }
+                        if (i < N) v = __fadd_rn(v, __uint_as_float(lds16(a + (uint32_t)i * hp_b) << 16));
+                    if (HAS_BIAS) v = __fadd_rn(v, h_b);
+                    sts32(o, out_bits<FP32OUT>(v));
                 }
             }
-            if (!mbar_wait(smem_u32(&main_done[st]), parity)) {
+            for (int c = at + DR_AUX; c < k; c += DR_AUX) {  // (more selected features than threads)
+                const float hb = HAS_BIAS ? __ldg(p.bias + __ldg(x.hp_idx + c)) : 0.0f;
+                for (int r = 0; r < rows; ++r) {
+                    float v = 0.0f;
+                    for (int i = 0; i < N; ++i)
+                        v = __fadd_rn(v, __uint_as_float(lds16(hp_s + (uint32_t)i * hp_b + (uint32_t)(r * k + c) * 2u) << 16));
+                    if (HAS_BIAS) v = __fadd_rn(v, hb);
+                    sts32(sums + (uint32_t)(r * k + c) * 4u, out_bits<FP32OUT>(v));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sums_ready[st]));  // (release: the sums above are visible to whoever waits)
+            if (!mbar_wait(smem_u32(&sums_ready[st]), parity)) {    // the other auxiliary warps' sums
                 atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
                 break;
             }
+            // (2) the last k columns
+            uint8_t *const obase = static_cast<uint8_t *>(p.out) + (t_begin + r0) * out_row_bytes;
+            if (on) {
+                uint32_t a = stage + c_off, sa = sums + c_sum;
+                uint8_t *o = obase + (int64_t)col * ESIZE;
+#pragma unroll 1
+                for (int r = 0; r < rows; ++r, a += row_b, sa += kb4, o += out_row_bytes) {
+                    float v = 0.0f;
 #pragma unroll
-            for (int j = 0; j < FX_PRE; ++j)
-                if (f_r[j] >= 0 && f_r[j] < rows) {
-                    const int64_t orow = (t0 + f_r[j]) * p.out_stride;
-                    if (HAS_BIAS) {
-                        hv[j] = __fadd_rn(hv[j], f_bh[j]);
-                        if (f_col[j] >= 0) fv[j] = __fadd_rn(fv[j], f_bf[j]);
-                    }
-                    store_one<FP32OUT>(p.out, orow + f_hpcol[j], hv[j]);
-                    if (f_col[j] >= 0) store_one<FP32OUT>(p.out, orow + f_col[j], fv[j]);
+                    for (int i = 0; i < NMAX; ++i)
+                        if (i < N) {
+                            const uint32_t w = (lds32(a + (uint32_t)i * lp_b) ^ 0x88888888u) >> c_hi;
+                            v = __fmaf_rn(__fadd_rn(__uint_as_float(and_or(w, c_mask, magic)), c_nb), c_s[i], v);
+                        }
+                    if (HAS_BIAS) v = __fadd_rn(v, c_b);
+                    const uint32_t sum = lds32(sa);
+                    store_bits<FP32OUT>(o, sel ? sum : out_bits<FP32OUT>(v));
                 }
-            for (int item = ft + FX_PRE * FX; item < rows * k; item += FX) {
-                const int r = item / k, h = item - r * k;  // row of the stage, rank of the selected feature
-                const int64_t orow = (t0 + r) * p.out_stride;
-                float v = 0.0f;
-                for (int i = 0; i < N; ++i)
-                    v = __fadd_rn(v, __uint_as_float((uint32_t)hp[i * hp_dev + r * k + h] << 16));
-                {
-                    const int hc = __ldg(x.hp_idx + h);
-                    store_one<FP32OUT>(p.out, orow + hc, HAS_BIAS ? __fadd_rn(v, __ldg(p.bias + hc)) : v);
-                }
-                if (h < x.n_holes) {
-                    const int slot = __ldg(x.hole + h), col = __ldg(x.filler + h);
-                    float u = 0.0f;
-                    for (int i = 0; i < N; ++i) {
-                        const uint32_t w =
-                            reinterpret_cast<const uint32_t *>(stage + (size_t)i * lay.lp_stage)[r * L8 + (slot >> 3)];
-                        const float code = __fsub_rn(
-                            __uint_as_float((((w >> ((slot & 7) * 4)) & 0xFu) ^ 8u) | 0x4B000000u), 8388616.0f);
-                        u = __fmaf_rn(code, __ldg(p.s_k + (size_t)i * E + col), u);
+            }
+            for (int c = at + DR_AUX; c < k; c += DR_AUX) {  // (more columns than threads)
+                const int cl = L + c, pc = __ldg(p.pos + cl);
+                for (int r = 0; r < rows; ++r) {
+                    uint32_t bits;
+                    if (pc >= 0) {
+                        float v = 0.0f;
+                        for (int i = 0; i < N; ++i)
+                            v = __fmaf_rn(code_at(lds32(stage + (uint32_t)i * lp_b + (uint32_t)(r * L8 + (pc >> 3)) * 4u), (pc & 7) * 4),
+                                          __ldg(p.s_k + (size_t)i * E + cl), v);
+                        if (HAS_BIAS) v = __fadd_rn(v, __ldg(p.bias + cl));
+                        bits = out_bits<FP32OUT>(v);
+                    } else {
+                        bits = lds32(sums + (uint32_t)(r * k + (-pc - 1)) * 4u);
                     }
-                    store_one<FP32OUT>(p.out, orow + col, HAS_BIAS ? __fadd_rn(u, __ldg(p.bias + col)) : u);
+                    store_bits<FP32OUT>(obase + r * out_row_bytes + (int64_t)cl * ESIZE, bits);
                 }
             }
             __syncwarp();
@@ -1045,14 +1144,24 @@ __global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams
     }
 
     // ---------------- main warps
-    const uint32_t magic = opaque_magic();
-    // 32-bit word indices into shared memory and a per-thread output pointer keep the loop's address
-    // arithmetic short
-    const uint32_t *const smem32 = reinterpret_cast<const uint32_t *>(smem);
-    const int stage_w = (int)(lay.stage >> 2), lp_w = (int)(lay.lp_stage >> 2);
-    constexpr int ESIZE = FP32OUT ? 4 : 2;
-    uint8_t *const out_col = static_cast<uint8_t *>(p.out) + (size_t)8 * g_ld * ESIZE;
-    const int64_t out_row_bytes = p.out_stride * ESIZE;
+    const int g = tid - 32 - DR_AUX;
+    const bool live = g < L8;
+    const int g_ld = live ? g : 0;
+    float2 sc[NMAX][4];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) {
+#pragma unroll
+        for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
+        if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
+    }
+    // the selected features among the thread's 8 ("holes": their lanes are overwritten with the sums)
+    const uint32_t gd = live ? __ldg(p.grp + g) : 0u;
+    const uint32_t hmask = gd & 0xFFu;
+    const int hrank = (int)(gd >> 8);  // rank of the group's first selected feature
+    const int nh = __popc(hmask);
+    const int hl0 = nh > 0 ? __ffs(hmask) - 1 : 0;
+    const int hl1 = nh > 1 ? __ffs(hmask & (hmask - 1)) - 1 : 0;
+    const bool warp_holes = __any_sync(0xffffffffu, nh > 0);
     float2 b[4];  // the thread's 8 biases (only in the instantiation that adds them)
 #pragma unroll
     for (int h = 0; h < 4; ++h) b[h] = make_float2(0.0f, 0.0f);
@@ -1062,55 +1171,60 @@ __global__ void __launch_bounds__(MAXT + FX + 32, 1) dequant_rows(const DRParams
         b[0] = make_float2(b0.x, b0.y); b[1] = make_float2(b0.z, b0.w);
         b[2] = make_float2(b1.x, b1.y); b[3] = make_float2(b1.z, b1.w);
     }
-    TPQ_DMARK(1);
+    const DecodeConsts dc = decode_consts();
+    const uint32_t word_s = smem_s + (uint32_t)g_ld * 4u;  // this thread's word of row 0, device 0, stage 0
+    const uint32_t row_b = (uint32_t)L8 * 4u;
+    uint8_t *orow = static_cast<uint8_t *>(p.out) + (size_t)8 * g_ld * ESIZE + t_begin * out_row_bytes;
+    asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");
+
     for (int it = 0;; ++it) {
-        const int64_t gi = blockIdx.x + it * (int64_t)gridDim.x;
-        if (gi >= pp.ngroups) break;
+        const int r0 = dr_stage_row(it, pp.first, G);
+        if (r0 >= rows_mine) break;
+        const int cap = it == 0 ? pp.first : G;
+        const int rows = rows_mine - r0 < cap ? rows_mine - r0 : cap;
         if (!mbar_wait(smem_u32(&full[st]), parity)) {
             atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
-        TPQ_DMARK(2 + 2 * it);
-        const int64_t t0 = gi * G;
-        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
-        const uint32_t *const sw = smem32 + st * stage_w + g_ld;  // this thread's word of row 0, device 0
-        uint8_t *orow = out_col + t0 * out_row_bytes;
-        for (int r0 = 0; r0 < rows; r0 += 2) {
-            const bool two = r0 + 1 < rows;
-            const int d1 = two ? L8 : 0;  // a ragged last stage decodes its last row twice, stores it once
-            const uint32_t *const w = sw + r0 * L8;
-            float2 acc[2][4];
-#pragma unroll
-            for (int r = 0; r < 2; ++r)
-#pragma unroll
-                for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-#pragma unroll
-            for (int i = 0; i < NMAX; ++i) {
-                if (i < N) {  // uniform
-                    const uint32_t w0 = w[i * lp_w];
-                    const uint32_t w1 = w[i * lp_w + d1];
-                    decode8(w0, sc[i], acc[0], magic);
-                    decode8(w1, sc[i], acc[1], magic);
-                }
-            }
-            if (live) {
-                if (HAS_BIAS) {  // (a hole's lane gets its own column's bias here and is overwritten by the fix-up)
-#pragma unroll
-                    for (int r = 0; r < 2; ++r)
-#pragma unroll
-                        for (int h = 0; h < 4; ++h) acc[r][h] = __fadd2_rn(acc[r][h], b[h]);
-                }
-                store_group<FP32OUT>(orow, 0, acc[0], 0u);
-                if (two) store_group<FP32OUT>(orow + out_row_bytes, 0, acc[1], 0u);
-            }
-            orow += 2 * out_row_bytes;
+        const uint32_t sa = word_s + (uint32_t)st * stage_b;
+        // whole stages run as straight-line code (rows per stage and device count known at compile time)
+        if (G == 4 && rows == 4) {
+            if (N == NMAX) rows_stage<NMAX, NMAX, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            else rows_stage<NMAX, 0, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+        } else if (G == 4 && rows == 2) {
+            rows_stage<NMAX, 0, 2, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+        } else if (G == 2 && rows == 2) {
+            if (N == NMAX) rows_stage<NMAX, NMAX, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            else rows_stage<NMAX, 0, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+        } else {
+#pragma unroll 1
+            for (int r = 0; r < rows; ++r)
+                rows_stage<NMAX, 0, 1, 0, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                                                             orow + r * out_row_bytes, out_row_bytes, live);
         }
+        if (warp_holes) {  // (uniform over the warp)
+            if (!mbar_wait(smem_u32(&sums_ready[st]), parity)) {
+                atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
+                break;
+            }
+            if (nh > 0) {
+                const uint32_t sums = sums_s + (uint32_t)st * sums_b + (uint32_t)hrank * 4u;
+                for (int r = 0; r < rows; ++r) {
+                    uint8_t *const o = orow + r * out_row_bytes;
+                    const uint32_t sr = sums + (uint32_t)(r * k) * 4u;
+                    store_bits<FP32OUT>(o + hl0 * ESIZE, lds32(sr));
+                    if (nh > 1) store_bits<FP32OUT>(o + hl1 * ESIZE, lds32(sr + 4u));
+                    if (nh > 2) {
+                        uint32_t m = hmask & (hmask - 1);
+                        m &= m - 1;
+                        for (int j = 2; m; ++j, m &= m - 1) store_bits<FP32OUT>(o + (__ffs(m) - 1) * ESIZE, lds32(sr + 4u * j));
+                    }
+                }
+            }
+        }
+        orow += rows * out_row_bytes;
         __syncwarp();
-        if (lane == 0) {
-            mbar_arrive(smem_u32(&main_done[st]));  // release: the row stores above precede the fix-up stores
-            mbar_arrive(smem_u32(&empty[st]));
-        }
-        TPQ_DMARK(3 + 2 * it);
+        if (lane == 0) mbar_arrive(smem_u32(&empty[st]));
         if (++st == nstage) {
             st = 0;
             parity ^= 1u;
@@ -1157,68 +1271,67 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
 
 namespace {
 
-template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
 cudaError_t launch_rows_w(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, HAS_WAIT>,
+    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
-        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(consumers + FX + 32), smem,
+        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(consumers + DR_AUX + 32), smem,
                            st, pp);
     return e;
 }
 
-template <int NMAX, int MAXT, int FX, bool FP32OUT, bool HAS_BIAS>
+template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
 cudaError_t launch_rows_v(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, true>(pp, grid, consumers, smem, st)
-                          : launch_rows_w<NMAX, MAXT, FX, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
-}
-
-template <int NMAX, int MAXT, int FX>
-cudaError_t launch_rows_f(const DRParams &pp, int fp32_out, int grid, int consumers, size_t smem, cudaStream_t st)
-{
-    const bool bias = pp.q.bias != nullptr;
-    if (fp32_out)
-        return bias ? launch_rows_v<NMAX, MAXT, FX, true, true>(pp, grid, consumers, smem, st)
-                    : launch_rows_v<NMAX, MAXT, FX, true, false>(pp, grid, consumers, smem, st);
-    return bias ? launch_rows_v<NMAX, MAXT, FX, false, true>(pp, grid, consumers, smem, st)
-                : launch_rows_v<NMAX, MAXT, FX, false, false>(pp, grid, consumers, smem, st);
+    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, true>(pp, grid, consumers, smem, st)
+                          : launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
 }
 
 template <int NMAX, int MAXT>
 cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    // two rows per stage: G k items per stage fit three fix-up warps with two items each for k <= 96
-    return (pp.G == 2 && 2 * pp.q.k <= 2 * 96) ? launch_rows_f<NMAX, MAXT, 96>(pp, fp32_out, grid, consumers, smem, st)
-                                               : launch_rows_f<NMAX, MAXT, DR_FIXUP_MAX>(pp, fp32_out, grid, consumers, smem, st);
+    const bool bias = pp.q.bias != nullptr;
+    if (fp32_out)
+        return bias ? launch_rows_v<NMAX, MAXT, true, true>(pp, grid, consumers, smem, st)
+                    : launch_rows_v<NMAX, MAXT, true, false>(pp, grid, consumers, smem, st);
+    return bias ? launch_rows_v<NMAX, MAXT, false, true>(pp, grid, consumers, smem, st)
+                : launch_rows_v<NMAX, MAXT, false, false>(pp, grid, consumers, smem, st);
+}
+
+// rows after which the code stream is 16-byte aligned again: blocks and stages start on multiples of it
+int g0_of(const tpq_ctx *c)
+{
+    const int L8 = (c->E - c->k) / 8;
+    return L8 % 4 == 0 ? 1 : (L8 % 2 == 0 ? 2 : 4);
 }
 
 // Row kernel geometry; returns false if the shape does not admit it.
-bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *ngroups_out, int *grid_out)
+bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t *rows_per_block_out, int *grid_out)
 {
-
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
     // measured against the panel kernels: the row kernel wins with up to 4 devices at every input length
     // (the panel kernels scale better with N)
     if (N > 4) return false;
     if (L8 > 768) return false;  // consumer threads (register budget per thread)
-    int g0 = 4;
-    if (L8 % 4 == 0) g0 = 1;
-    else if (L8 % 2 == 0) g0 = 2;
-    int G = g0 < 2 ? 2 : g0;  // 2 or 4 rows per stage (a multiple of g0), walked two rows at a time
-    // long inputs: 4-row stages amortise the per-stage work (measured faster from about 32 rows per block)
-    if (G == 2 && T >= 32LL * c->sm_count && dr_layout(N, E, k, 4, 3).total <= (size_t)c->smem_optin) G = 4;
+    const int g0 = g0_of(c);
+    // every block takes the same number of adjacent rows (a multiple of g0), so no block has more than g0 - 1
+    // rows above the mean; it walks them four at a time where a ring of three such stages fits, else two
+    int64_t rpb = (T + c->sm_count - 1) / c->sm_count;
+    rpb = (rpb + g0 - 1) / g0 * g0;
+    int G = 4;
+    if (rpb < 4 || dr_layout(N, E, k, 4, 3).total > (size_t)c->smem_optin) G = 2;
+    if (G < g0) G = g0;
     if (dr_layout(N, E, k, G, 2).total > (size_t)c->smem_optin) return false;
-    const int64_t ngroups = (T + G - 1) / G;
-    const int grid = (int)(ngroups < c->sm_count ? ngroups : c->sm_count);
-    const int64_t per_block = (ngroups + grid - 1) / grid;
+    const int grid = (int)((T + rpb - 1) / rpb);
+    const int64_t per_block = (rpb + G - 1) / G;
     int nstage = (int)(per_block < 4 ? per_block : 4);  // deeper rings measured no faster (often slower)
     if (G == 4 && nstage > 3) nstage = 3;
     if (nstage < 2) nstage = 2;
     while (nstage > 2 && dr_layout(N, E, k, G, nstage).total > (size_t)c->smem_optin) --nstage;
-    *G_out = G; *nstage_out = nstage; *ngroups_out = ngroups; *grid_out = grid;
+    *G_out = G; *nstage_out = nstage; *rows_per_block_out = rpb; *grid_out = grid;
     return true;
 }
 
@@ -1374,12 +1487,11 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
     if (want == 0 || want == 1) {
         DRParams pp;
         int grid = 0;
-        if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.ngroups, &grid)) {
+        if (rows_plan(c, T, &pp.G, &pp.nstage, &pp.rows_per_block, &grid)) {
             pp.q = p;
             pp.x = x;
-#ifdef TPQ_TRACE
-            pp.trace = g_dtrace;
-#endif
+            // a short first stage lands sooner (measured at 2048 x 5120: 11.0 -> 10.9 us, 12.3 -> 11.6 us without the prefetch)
+            pp.first = (pp.G == 4 && pp.rows_per_block > 4 && (g0_of(c) <= 2)) ? 2 : pp.G;
             const size_t smem = dr_layout(c->N, c->E, c->k, pp.G, pp.nstage).total;
             const int L8 = (c->E - c->k) / 8;
             int consumers = ((L8 + 31) / 32) * 32;

@@ -102,9 +102,6 @@ struct QPParams {
     uint32_t epoch;                     // value written to every arrival word once the payload is complete
     uint32_t *arrived[QP_MAX_BATCH];    // arrival word beside destination d (same memory as payload[d])
     unsigned int *done;                 // blocks that have finished their stores (returns to 0)
-#ifdef TPQ_TRACE
-    long long *trace;
-#endif
 };
 
 // Dynamic shared memory layout (byte offsets).
@@ -153,26 +150,12 @@ __device__ __forceinline__ uint32_t quant8(const uint4 v, const float2 (&inv)[4]
     return (acc - K0 + 0x88888888u) ^ 0x88888888u;
 }
 
-#ifdef TPQ_TRACE
-static long long *g_trace = nullptr;  // 64 slots per block, globaltimer ns
-__device__ __forceinline__ long long tpq_now()
-{
-    long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-#define TPQ_MARK(slot) do { if (threadIdx.x == 0 && p.trace && (slot) < 64) p.trace[blockIdx.x * 64 + (slot)] = tpq_now(); } while (0)
-#else
-#define TPQ_MARK(slot) do { } while (0)
-#endif
-
 // PUSH: every payload store goes to n_dst destinations (plain stores; a destination may be a peer's
 // memory), and the block that finishes last publishes the arrival words.
 template <int GPT, int G, int TB, bool PUSH>  // TB: upper bound of the block size (register budget)
 __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
-    TPQ_MARK(0);
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
     // this block's shard of the batch, its index among the shard's blocks, and the shard's buffers
@@ -234,7 +217,6 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     tpq_grid_dep_wait();    // the input and the payload buffer may still be in use by the kernel ahead
     __syncthreads();
     tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
-    TPQ_MARK(40);
 
     if (tid >= NT) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier; a contiguous
@@ -314,7 +296,6 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
             m &= m - 1;
         }
     }
-    TPQ_MARK(1);
 
     int st = 0;
     uint32_t parity = 0;
@@ -325,7 +306,6 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
             atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
-        TPQ_MARK(2 + 2 * it);
         const int64_t t0 = gi * G;
         const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
         const uint4 *stage = reinterpret_cast<const uint4 *>(ring + (size_t)st * stage_bytes);
@@ -406,7 +386,6 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         }
         __syncwarp();
         if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty[st]));
-        TPQ_MARK(3 + 2 * it);
         if (++st == nstage) {
             st = 0;
             parity ^= 1u;
@@ -570,9 +549,6 @@ cudaError_t launch_tiled(const tpq_ctx *c, int shard0, int n, const void *const 
     p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
     p.inv_s = c->t.inv_s + (size_t)shard0 * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
     p.lp_words = lpb / 4; p.status = c->t.status;
-#ifdef TPQ_TRACE
-    p.trace = g_trace;
-#endif
     const size_t smem = qp_smem_bytes(E, G, nstage);
 
     cudaError_t e = cudaSuccess;
