@@ -5,6 +5,8 @@
 // The two roundings are kept separate (__fmul_rn, then the magic-constant add).
 #include "tpq_internal.h"
 
+#include <type_traits>
+
 namespace {
 
 // ----------------------------------------------------------------------------------------------
@@ -78,6 +80,8 @@ __global__ void __launch_bounds__(256) quantize_generic(const uint16_t *__restri
 constexpr int QP_MAX_GPT = 4;          // groups of 8 features per thread
 constexpr int QP_MAX_CONSUMERS = 992;  // 31 consumer warps + 1 producer warp per block
 
+constexpr int QP_PREFETCH_ROWS = 4;  // rows whose bytes a block asks L2 for ahead of the dependency wait
+
 constexpr int QP_MAX_BATCH = 16;  // devices' shards quantised by one launch (each by its own set of blocks)
 
 struct QPParams {
@@ -89,8 +93,9 @@ struct QPParams {
     int64_t T;
     int E, k;
     int G;        // rows per stage
+    int first;    // rows of a block's first stage (<= G: a short first stage lands sooner)
+    int64_t rows_per_block;  // a block quantises rows_per_block adjacent rows of its shard
     int nstage;
-    int64_t ngroups;
     const float *inv_s;     // [E] of the batch's first device; device d of the batch at inv_s + d*E
     const uint32_t *grp;    // [E/8]
     const int32_t *filler;  // [n_holes]
@@ -174,61 +179,50 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
     uint64_t *full = reinterpret_cast<uint64_t *>(smem + lay.bars);
     uint64_t *empty = full + nstage;
 
-    if (tid == 0) {
-        for (int s = 0; s < nstage; ++s) {
-            mbar_init(smem_u32(&full[s]), 1);
-            mbar_init(smem_u32(&empty[s]), NT / 32);
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
+    // this block's rows
+    const int64_t t_begin = (int64_t)bx * p.rows_per_block;
+    const int64_t t_end = (p.T - t_begin < p.rows_per_block) ? p.T : t_begin + p.rows_per_block;
+    const int rows_mine = (int)(t_end - t_begin);
+    // first row (within the block's run) and row count of the block's it-th stage
+    auto stage_row = [&](int it) { return it == 0 ? 0 : p.first + (it - 1) * G; };
+    auto stage_rows = [&](int it, int r0) {
+        const int cap = it == 0 ? p.first : G;
+        return rows_mine - r0 < cap ? rows_mine - r0 : cap;
+    };
 
-    // ---- consumer constants: their loads are issued BEFORE the block-wide barrier that releases the
-    // producer, so they are not queued behind the bulk copies in the memory system.
-    float2 inv[GPT][4];
-    uint32_t mask[GPT];      // selected features among the thread's 8 (only where the group is below L)
-    int hb[GPT];             // holes before the group
-    // the first two holes of the group: bit position of the hole's nibble in the word and its mask
-    uint32_t f_sh[GPT][2], hmask[GPT][2];
-    int my_hp = 0;
-    if (tid < NT) {
-#pragma unroll
-        for (int a = 0; a < GPT; ++a) {
-            const int g = tid + a * NT;
-            mask[a] = 0; hb[a] = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
-            f_sh[a][0] = f_sh[a][1] = 0;
-            hmask[a][0] = hmask[a][1] = 0;
-            if (g < L8) {
-                const float4 i0 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g));
-                const float4 i1 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g + 4));
-                const uint32_t gd = __ldg(p.grp + g);
-                inv[a][0] = make_float2(i0.x, i0.y);
-                inv[a][1] = make_float2(i0.z, i0.w);
-                inv[a][2] = make_float2(i1.x, i1.y);
-                inv[a][3] = make_float2(i1.z, i1.w);
-                mask[a] = gd & 0xFFu;
-                hb[a] = (int)(gd >> 8);
-            }
-        }
-        if (tid < k) my_hp = __ldg(p.hp_idx + tid);
-    }
-    tpq_grid_dep_wait();    // the input and the payload buffer may still be in use by the kernel ahead
-    __syncthreads();
-    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue
-
+    // Order of the prologue.  The producer warp sets up the barriers, waits for the kernel ahead in the stream
+    // and issues the first stages' copies at once; the consumers' table loads run in the shadow of the first
+    // stage's flight.  Only the producer executes griddepcontrol.wait: every store of a consumer follows a
+    // "full" barrier that one of the producer's copies completes, i.e. follows that wait.
+    tpq_grid_dep_launch();  // the next kernel in the stream may start its own prologue as SMs free up
     if (tid >= NT) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier; a contiguous
         // input is one copy per stage, a strided one is one copy per row, issued by as many lanes at once
         const int pl = tid - NT;
+        if (pl == 0) {
+            for (int s = 0; s < nstage; ++s) {
+                mbar_init(smem_u32(&full[s]), 1);
+                mbar_init(smem_u32(&empty[s]), NT / 32);
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncwarp();
+        asm volatile("bar.arrive 1, %0;" ::"r"(blockDim.x) : "memory");  // the barriers exist
+        if (pl == 0 && p.stride == E) {
+            // the block's first rows may start their way from HBM to L2 while it waits (a hint only: L2 is the
+            // point of coherence, so whatever the kernel ahead still writes is what the copies will read)
+            const int rows = rows_mine < QP_PREFETCH_ROWS ? rows_mine : QP_PREFETCH_ROWS;
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(y_in + t_begin * p.stride), "r"(rows * row_bytes) : "memory");
+        }
+        tpq_grid_dep_wait();  // the input and the payload buffer may still be in use by the kernel ahead
         int st = 0;
         uint32_t parity = 1;  // parity of the "empty" phase to wait for
         for (int it = 0;; ++it) {
-            const int64_t gi = bx + it * (int64_t)p.cps;
-            if (gi >= p.ngroups) break;
-            const int64_t t0 = gi * G;
-            const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+            const int r0 = stage_row(it);
+            if (r0 >= rows_mine) break;
+            const int rows = stage_rows(it, r0);
+            const int64_t t0 = t_begin + r0;
             const uint32_t bar = smem_u32(&full[st]);
             const uint32_t dst = smem_u32(ring + (size_t)st * stage_bytes);
             int ok = 1;
@@ -256,6 +250,36 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         return;
     }
 
+    // ---- consumer constants
+    float2 inv[GPT][4];
+    uint32_t mask[GPT];      // selected features among the thread's 8 (only where the group is below L)
+    int hb[GPT];             // holes before the group
+    // the first two holes of the group: bit position of the hole's nibble in the word and its mask
+    uint32_t f_sh[GPT][2], hmask[GPT][2];
+    int my_hp = 0;
+    {
+#pragma unroll
+        for (int a = 0; a < GPT; ++a) {
+            const int g = tid + a * NT;
+            mask[a] = 0; hb[a] = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) inv[a][i] = make_float2(0.0f, 0.0f);
+            f_sh[a][0] = f_sh[a][1] = 0;
+            hmask[a][0] = hmask[a][1] = 0;
+            if (g < L8) {
+                const float4 i0 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g));
+                const float4 i1 = __ldg(reinterpret_cast<const float4 *>(inv_s + 8 * g + 4));
+                const uint32_t gd = __ldg(p.grp + g);
+                inv[a][0] = make_float2(i0.x, i0.y);
+                inv[a][1] = make_float2(i0.z, i0.w);
+                inv[a][2] = make_float2(i1.x, i1.y);
+                inv[a][3] = make_float2(i1.z, i1.w);
+                mask[a] = gd & 0xFFu;
+                hb[a] = (int)(gd >> 8);
+            }
+        }
+        if (tid < k) my_hp = __ldg(p.hp_idx + tid);
+    }
     // ---------------- consumers
     // Holes are patched warp-cooperatively.  The holes of a warp's 32 groups are consecutive in the
     // global hole order, so lane i quantises the filler element of the warp's i-th hole (w_off / w_inv)
@@ -297,41 +321,43 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         }
     }
 
+    asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");  // the producer has set up the barriers
+
     int st = 0;
     uint32_t parity = 0;
     for (int it = 0;; ++it) {
-        const int64_t gi = bx + it * (int64_t)p.cps;
-        if (gi >= p.ngroups) break;
+        const int r0s = stage_row(it);
+        if (r0s >= rows_mine) break;
+        const int rows = stage_rows(it, r0s);
         if (!mbar_wait(smem_u32(&full[st]), parity)) {
             atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
             break;
         }
-        const int64_t t0 = gi * G;
-        const int rows = (int)((p.T - t0 < G) ? p.T - t0 : G);
+        const int64_t t0 = t_begin + r0s;
         const uint4 *stage = reinterpret_cast<const uint4 *>(ring + (size_t)st * stage_bytes);
         const uint16_t *stage16 = reinterpret_cast<const uint16_t *>(stage);
+        const uint8_t *stage8 = reinterpret_cast<const uint8_t *>(stage);
 #pragma unroll
         for (int a = 0; a < GPT; ++a) {
             const int g = tid + a * NT;
             const bool live = g < L8;
             const int g_ld = live ? g : 0;  // idle lanes load something harmless: straight-line code below
-            const uint32_t nh = __popc(mask[a]);
-            const uint8_t *stage8 = reinterpret_cast<const uint8_t *>(stage);
-            if (!serial[a] && rows == G) {
-                // full stage: all shared loads of the G rows first, then G independent chains, no branches
-                uint4 v[G];
-                uint32_t fx[G];
+            // GR rows from row rb of the stage on: all shared loads first, then GR independent chains, no branches
+            auto rows_fast = [&](auto gr_tag, int rb) {
+                constexpr int GR = decltype(gr_tag)::value;
+                uint4 v[GR];
+                uint32_t fx[GR];
 #pragma unroll
-                for (int r = 0; r < G; ++r) {
-                    v[r] = stage[r * E8 + g_ld];
-                    fx[r] = *reinterpret_cast<const uint16_t *>(stage8 + (size_t)r * row_bytes + w_off[a]);
+                for (int r = 0; r < GR; ++r) {
+                    v[r] = stage[(rb + r) * E8 + g_ld];
+                    fx[r] = *reinterpret_cast<const uint16_t *>(stage8 + (size_t)(rb + r) * row_bytes + w_off[a]);
                 }
-                uint32_t word[G];
+                uint32_t word[GR];
 #pragma unroll
-                for (int r = 0; r < G; ++r) word[r] = quant8(v[r], inv[a]);
+                for (int r = 0; r < GR; ++r) word[r] = quant8(v[r], inv[a]);
                 if (n_wh[a]) {  // uniform over the warp
 #pragma unroll
-                    for (int r = 0; r < G; ++r) {
+                    for (int r = 0; r < GR; ++r) {
                         const uint32_t qv = quant_bits(fx[r], w_inv[a]) & 0xFu;
                         const uint32_t q0 = __shfl_sync(0xffffffffu, qv, src0[a]) << f_sh[a][0];
                         const uint32_t q1 = __shfl_sync(0xffffffffu, qv, src0[a] + 1) << f_sh[a][1];
@@ -341,17 +367,23 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                 if (live) {
                     if constexpr (PUSH) {
                         for (int d = 0; d < p.n_dst; ++d) {
-                            uint32_t *const o = reinterpret_cast<uint32_t *>(p.payload[d]) + t0 * L8 + g;
+                            uint32_t *const o = reinterpret_cast<uint32_t *>(p.payload[d]) + (t0 + rb) * L8 + g;
 #pragma unroll
-                            for (int r = 0; r < G; ++r) o[r * L8] = word[r];
+                            for (int r = 0; r < GR; ++r) o[r * L8] = word[r];
                         }
                     } else {
 #pragma unroll
-                        for (int r = 0; r < G; ++r) lp_out[(t0 + r) * L8 + g] = word[r];
+                        for (int r = 0; r < GR; ++r) lp_out[(t0 + rb + r) * L8 + g] = word[r];
                     }
                 }
+            };
+            if (!serial[a]) {  // (uniform over the warp, like the row counts below)
+                int rb = 0;
+                if (G >= 4 && rows - rb >= 4) { rows_fast(std::integral_constant<int, 4>(), rb); rb += 4; }
+                if (G >= 2 && rows - rb >= 2) { rows_fast(std::integral_constant<int, 2>(), rb); rb += 2; }
+                if (rows - rb >= 1) rows_fast(std::integral_constant<int, 1>(), rb);
             } else if (live) {
-                // ragged last stage, or a warp on the serial path: every hole patched by its owner
+                // a warp on the serial path: every hole patched by its owner
                 for (int r = 0; r < rows; ++r) {
                     uint32_t word = quant8(stage[r * E8 + g], inv[a]);
                     uint32_t m = mask[a];
@@ -371,7 +403,6 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
                     }
                 }
             }
-            (void)nh;
         }
         for (int h = tid; h < k; h += NT) {
             const int j = (h == tid) ? my_hp : __ldg(p.hp_idx + h);
@@ -392,7 +423,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         }
     }
     // zero padding of the code section (at most 3 words), by the block that owned the last rows
-    if ((p.ngroups - 1) % p.cps == bx) {
+    if (t_begin < p.T && p.T <= t_end) {
         const int64_t valid = p.T * L8;
         for (int64_t w = valid + tid; w < p.lp_words; w += NT) {
             if constexpr (PUSH) {
@@ -519,13 +550,17 @@ cudaError_t launch_tiled(const tpq_ctx *c, int shard0, int n, const void *const 
     // blocks per shard: the SMs are divided among the shards of the batch (one persistent block per SM)
     int cps = c->sm_count / n;
     if (cps < 1) cps = 1;
-    // rows per stage (= independent chains per thread): small enough that every block gets work
+    // every block takes the same number of adjacent rows of its shard, so none has more than a row above the
+    // mean; it walks them four at a time where a ring of three such stages fits (else two, else one), and a
+    // short first stage lands sooner
+    if (T < cps) cps = (int)T;
+    const int64_t rpb = (T + cps - 1) / cps;
+    cps = (int)((T + rpb - 1) / rpb);
     int G = 4;
-    while (G > 1 && ((T + G - 1) / G < 2 * (int64_t)cps || qp_smem_bytes(E, G, 3) > (size_t)c->smem_optin)) G >>= 1;
-    const int64_t ngroups = (T + G - 1) / G;
-    if (ngroups < cps) cps = (int)ngroups;
+    while (G > 1 && (rpb < G || qp_smem_bytes(E, G, 3) > (size_t)c->smem_optin)) G >>= 1;
+    const int first = (G == 4 && rpb > 4) ? 2 : G;
     const int64_t grid = (int64_t)cps * n;
-    const int64_t per_block = (ngroups + cps - 1) / cps;
+    const int64_t per_block = (rpb + G - 1) / G + (first < G ? 1 : 0);
     int nstage = (int)(per_block < 8 ? per_block : 8);
     if (nstage < 2) nstage = 2;
     while (nstage > 2 && qp_smem_bytes(E, G, nstage) > (size_t)c->smem_optin) --nstage;
@@ -546,7 +581,7 @@ cudaError_t launch_tiled(const tpq_ctx *c, int shard0, int n, const void *const 
         }
     }
     p.cps = cps; p.lp_bytes = lpb;
-    p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.nstage = nstage; p.ngroups = ngroups;
+    p.stride = stride; p.T = T; p.E = E; p.k = k; p.G = G; p.first = first; p.rows_per_block = rpb; p.nstage = nstage;
     p.inv_s = c->t.inv_s + (size_t)shard0 * E; p.grp = c->t.grp; p.filler = c->t.filler; p.hp_idx = c->t.hp_idx;
     p.lp_words = lpb / 4; p.status = c->t.status;
     const size_t smem = qp_smem_bytes(E, G, nstage);
