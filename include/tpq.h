@@ -29,7 +29,7 @@
  *     the calibration scratch and the block counter of tpq_quantize_pack_push).
  *   - One context serves all N simulated devices: the static parameters and
  *     the selected feature set are identical on every device by construction
- *     (Section 3: "fixed across all sequences and devices").
+ *     (Section 3: the set is static and shared by every sequence and device).
  */
 #ifndef TPQ_H
 #define TPQ_H
@@ -86,7 +86,7 @@ typedef struct tpq_comm_report {
 /* Create a context for n_shards (N >= 1) devices and n_features (E >= 1)
  * features on the current CUDA device.  bits is the code width: 4 is the
  * paper's Int4 (Section 3) and the width the tiled kernels serve; 2..8 are
- * accepted (the method "at lower and higher precision", Section 4 / Figure 3:
+ * accepted (other code widths, as evaluated in Section 4 / Figure 3:
  * step R/(2^bits - 1), codes -2^(bits-1) .. 2^(bits-1)-1, one little-endian
  * stream of bits-wide codes) and run on the shape-generic kernels.  gamma is
  * the moving-average constant of Eq. (1)-(2) (the paper uses 0.01),
@@ -164,17 +164,41 @@ tpq_status tpq_get_scales(tpq_ctx *ctx, float *s_host, float *inv_s_host);
 int tpq_num_selected(const tpq_ctx *ctx);
 /* The selected indices, ascending (capacity >= k).  BAD_STATE before a feature set. */
 tpq_status tpq_get_features(tpq_ctx *ctx, int32_t *hp_idx_out_host);
+/* The slot order of the payload's code section (see "Wire format" below): slot_feature_out_host[c],
+ * 0 <= c < E-k, is the feature whose code slot c of every token carries (capacity >= E-k int32).
+ * The order is this library's choice (the paper gives only the bit count, Section 4).
+ * BAD_STATE before a feature set; synchronises. */
+tpq_status tpq_get_slot_order(tpq_ctx *ctx, int32_t *slot_feature_out_host);
 
 /* ------------------------------------------------------------- the payload */
 
 /* Payload size in bytes for T tokens with the current feature set:
  *   roundup16(ceil(T*(E-k)/2)) + 2*T*k
- * (Section 4 counts (E-k) 4-bit codes and k BF16 values per token).
- * Layout: one flat stream of 4-bit two's-complement codes in (token, feature
- * with the selected ones removed) order, low nibble first, zero padded to a
- * multiple of 16 bytes; then T*k BF16 values, token-major, selected features
- * ascending.  No header; the static steps are never transmitted.
- * Returns 0 before a feature set exists or for T <= 0. */
+ * (Section 4 counts (E-k) 4-bit codes and k BF16 values per token; the byte
+ * layout below is this library's: the paper fixes only the bit count).
+ *
+ * Wire format.  With L = E-k:
+ *   bytes [0, roundup16(ceil(T*L/2)))  the code section: one flat stream of
+ *       4-bit two's-complement codes; code p = t*L + c (token t, slot c) is
+ *       the low nibble of byte p/2 if p is even, the high nibble if p is odd;
+ *       unused nibbles and the padding up to a multiple of 16 bytes are 0;
+ *   then T*k BF16 values, token-major: value t*k + h is the h-th selected
+ *       feature (ascending feature index) of token t, its bits unchanged.
+ * No header; the static steps are never transmitted.
+ *
+ * Slot order ("hole filling"): which feature slot c of a token carries.
+ * Let S be the selected set.  The holes are the selected features below L,
+ * ascending: h_0 < h_1 < ...; the fillers are the unselected features at or
+ * above L, ascending: f_0 < f_1 < ... (there are equally many of both).
+ *   slot c, 0 <= c < L, carries feature c        if c is not selected,
+ *                               feature f_i      if c = h_i.
+ * So every unselected feature below L keeps its own index as slot, and the
+ * i-th filler takes the i-th hole.  Example: E = 8, S = {1, 6}, L = 6: the
+ * hole is 1, the filler is 7, the slots carry features 0 7 2 3 4 5 and the
+ * BF16 values are features 1 and 6.  tpq_get_slot_order returns the table.
+ * For code widths other than 4 bits the stream is the same with bits-wide
+ * codes: code p occupies bits [p*bits, (p+1)*bits) of the little-endian stream.
+ * tpq_payload_bytes returns 0 before a feature set exists or for T <= 0. */
 size_t tpq_payload_bytes(const tpq_ctx *ctx, int64_t T);
 /* The same closed form without a context (Int4), and for a code width of
  * 2..8 bits: roundup16(ceil(T*(E-k)*bits / 8)) + 2*T*k. */
@@ -240,8 +264,8 @@ tpq_status tpq_dequant_reduce_bias(tpq_ctx *ctx, const void *const *payloads_dev
  * FP32 accumulation, one rounding to BF16 (the layer's output type), then exactly tpq_quantize_pack.
  *
  * tpq_permute_weight: once per weight matrix and feature set, gather the rows of w_bf16_dev ([E][K],
- * row-major, 16-byte aligned) into the payload's slot order: row c < E-k is the feature that code slot c
- * carries, row E-k+h the h-th selected feature.  w_slots_dev: [E][K], 16-byte aligned, not aliasing w.
+ * row-major, 16-byte aligned) into the payload's slot order ("Wire format" above; tpq_get_slot_order): row
+ * c < E-k is the feature that code slot c carries, row E-k+h the h-th selected feature.  w_slots_dev: [E][K], 16-byte aligned, not aliasing w.
  * Errors: BAD_STATE (no feature set), INVALID_ARG, ALIGN, CUDA. */
 tpq_status tpq_permute_weight(tpq_ctx *ctx, const void *w_bf16_dev, int64_t K, void *w_slots_dev, void *cuda_stream);
 

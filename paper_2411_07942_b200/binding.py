@@ -45,6 +45,7 @@ SIGNATURES = {
     "tpq_get_scales": (c_int, [c_void_p, POINTER(c_float), POINTER(c_float)]),
     "tpq_num_selected": (c_int, [c_void_p]),
     "tpq_get_features": (c_int, [c_void_p, POINTER(c_int32)]),
+    "tpq_get_slot_order": (c_int, [c_void_p, POINTER(c_int32)]),
     "tpq_payload_bytes": (c_size_t, [c_void_p, c_int64]),
     "tpq_payload_bytes_for": (c_size_t, [c_int64, c_int64, c_int64]),
     "tpq_payload_bytes_for_bits": (c_size_t, [c_int64, c_int64, c_int64, c_int]),
@@ -188,6 +189,13 @@ class Tpq:
         out = np.zeros(max(k, 1), np.int32)
         self._check(lib().tpq_get_features(self._h, out.ctypes.data_as(POINTER(c_int32))))
         return out[:k].copy()
+
+    def get_slot_order(self) -> np.ndarray:
+        """Feature carried by each code slot of a token (length E - k)."""
+        L = self.E - max(self.num_selected(), 0)
+        out = np.zeros(max(L, 1), np.int32)
+        self._check(lib().tpq_get_slot_order(self._h, out.ctypes.data_as(POINTER(c_int32))))
+        return out[:L].copy()
 
     def payload_bytes(self, T: int) -> int:
         return int(lib().tpq_payload_bytes(self._h, T))

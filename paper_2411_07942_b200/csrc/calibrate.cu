@@ -5,6 +5,8 @@
 // (sign-magnitude -> two's complement, so -0 sorts below +0 and the result does
 // not depend on the order in which rows are visited); min / max of the keys are
 // exact, so any reduction tree gives the same bits.
+#include <mutex>
+
 #include "tpq_internal.h"
 
 namespace {
@@ -266,14 +268,22 @@ namespace {
 constexpr int kMaxDevices = 64;
 void *g_static_scratch_ptr[kMaxDevices];  // device address of the array, per device ordinal (set-up once)
 bool g_static_scratch_ready[kMaxDevices];
+std::mutex g_static_scratch_mutex;
 }  // namespace
 
 cudaError_t tpq_static_scratch_address(int device, void **ptr_out)
 {
     if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+    // The look-up answers for the CURRENT device: a caller on another device would cache a wrong address.
+    int current = -1;
+    cudaError_t e = cudaGetDevice(&current);
+    if (e != cudaSuccess) return e;
+    if (current != device) return cudaErrorInvalidDevice;
+    // One look-up per device; contexts on several host threads may get here together.
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
     if (!g_static_scratch_ready[device]) {
         void *ptr = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);  // for the CURRENT device
+        e = cudaGetSymbolAddress(&ptr, g_calib_static_scratch);
         if (e != cudaSuccess) return e;
         g_static_scratch_ptr[device] = ptr;
         g_static_scratch_ready[device] = true;

@@ -618,6 +618,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     // ring state: the producer lane and the main warps walk the same sequence of stages across segments
     int st = 0, it = 0;
     uint32_t parity = (tid >= DT_MAIN) ? 1u : 0u;  // producer: parity of the "empty" phase to wait for
+    bool dead = false;  // a wait of this thread ran out (TPQ_ERR_TIMEOUT is recorded)
 
     for (int64_t f = f0; f < f1;) {
         const int panel = (int)(f / pp.n_chunks);
@@ -647,14 +648,16 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                     for (int i0 = 0; i0 < N; i0 += DT_NB, ++it) {
                         const int nb = (N - i0 < DT_NB) ? N - i0 : DT_NB;
                         const uint32_t bar = smem_u32(&full[st]);
-                        if (it >= nstage && !mbar_wait(smem_u32(&empty[st]), parity)) {
+                        if (it >= nstage && !dead && !mbar_wait(smem_u32(&empty[st]), parity)) {
                             atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
-                            return;
+                            dead = true;  // nothing more is issued; the loops go on so that every barrier is still met
                         }
-                        mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
-                        const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
-                        for (int i = 0; i < nb; ++i)
-                            tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
+                        if (!dead) {
+                            mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
+                            const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
+                            for (int i = 0; i < nb; ++i)
+                                tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
+                        }
                         if (++st == nstage) {
                             st = 0;
                             parity ^= 1u;
@@ -719,9 +722,9 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                     for (int i = 0; i < DT_NB; ++i)
                         if (i0 + i < N) hvv[i] = __ldcs(reinterpret_cast<const uint16_t *>(p.pl[i0 + i] + it_off));
                 }
-                if (!mbar_wait(smem_u32(&full[st]), parity)) {
+                if (!dead && !mbar_wait(smem_u32(&full[st]), parity)) {
                     atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
-                    return;
+                    dead = true;  // no more waits and no more stores; the loops go on so that every barrier is still met
                 }
                 const uint32_t *const sw = ring_w + (size_t)st * (STAGE_BYTES / 4);
                 uint32_t w[DT_NB][DP_R];
@@ -762,12 +765,12 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                 for (int i = 0; i < DT_NB; ++i)
                     if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
             }
-            if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+            if (live && !dead) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
             if (n_it > 0) {
                 asm volatile("bar.sync 1, %0;" ::"n"(DT_MAIN) : "memory");  // the chunk's rows are stored
-                if (it_on) item_done(tc + my_r, my_col, my_fcol, hv);
+                if (it_on && !dead) item_done(tc + my_r, my_col, my_fcol, hv);
                 // panels with more items than threads (many selected features in one panel): the rest, unpipelined
-                for (int a = tid + DT_MAIN; a < items; a += DT_MAIN) {
+                for (int a = tid + DT_MAIN; a < items && !dead; a += DT_MAIN) {
                     const int r = a / n_it, h = hs + (a - r * n_it);
                     if (tc + r >= p.T) break;
                     const int64_t off = p.lp_bytes + ((tc + r) * k + h) * 2;

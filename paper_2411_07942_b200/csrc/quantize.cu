@@ -163,8 +163,10 @@ template <int GPT, int G, int TB, bool PUSH>  // TB: upper bound of the block si
 __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
 {
     extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ int s_failed;  // (push mode) a wait of this block ran out
     const int tid = threadIdx.x;
     const int NT = blockDim.x - 32;  // consumer threads
+    if (PUSH && tid == 0) s_failed = 0;  // (ordered before any use by the named barrier of the prologue)
     // this block's shard of the batch, its index among the shard's blocks, and the shard's buffers
     const int sb = blockIdx.x / p.cps;
     const int bx = blockIdx.x - sb * p.cps;
@@ -333,6 +335,7 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         const int rows = stage_rows(it, r0s);
         if (!mbar_wait(smem_u32(&full[st]), parity)) {
             atomicExch(p.status, (int)TPQ_ERR_TIMEOUT);
+            if constexpr (PUSH) s_failed = 1;  // this block's part of the payload is incomplete
             break;
         }
         const int64_t t0 = t_begin + r0s;
@@ -442,14 +445,18 @@ __global__ void __launch_bounds__(TB, 1) quantize_tiled(const QPParams p)
         asm volatile("bar.sync 2, %0;" ::"r"(NT) : "memory");
         if (tid == 0) {
             __threadfence_system();
-            const unsigned int prev = atomicAdd(p.done, 1u);
-            if (prev == gridDim.x - 1) {
+            // a block whose waits ran out counts in the upper half as well: the payload is then incomplete,
+            // the words are not written, and the receivers' own bounded waits flag the step
+            const unsigned int prev = atomicAdd(p.done, s_failed ? 0x10001u : 1u);
+            if ((prev & 0xFFFFu) == gridDim.x - 1) {
                 *p.done = 0u;  // the next launch in the stream starts from zero
-                // one fence (acquire side of the counts above, release side of the words below), then the
-                // words as relaxed system-scope stores: together a release of everything observed so far
-                __threadfence_system();
-                for (int d = 0; d < p.n_dst; ++d)
-                    asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p.arrived[d]), "r"(p.epoch) : "memory");
+                if ((prev >> 16) == 0 && !s_failed) {
+                    // one fence (acquire side of the counts above, release side of the words below), then the
+                    // words as relaxed system-scope stores: together a release of everything observed so far
+                    __threadfence_system();
+                    for (int d = 0; d < p.n_dst; ++d)
+                        asm volatile("st.relaxed.sys.global.u32 [%0], %1;" ::"l"(p.arrived[d]), "r"(p.epoch) : "memory");
+                }
             }
         }
     }

@@ -249,6 +249,8 @@ tpq_status tpq_calibrate_ranges_noalloc(tpq_ctx *c, int shard, const void *y, in
                     (unsigned)(TPQ_NOALLOC_SCRATCH_BYTES / 4));
     void *scratch = nullptr;
     cudaError_t e = tpq_static_scratch_address(c->device, &scratch);  // first call on a device: symbol look-up
+    if (e == cudaErrorInvalidDevice)
+        return fail(c, TPQ_ERR_BAD_STATE, "the context's device (%d) must be the current CUDA device", c->device);
     if (e != cudaSuccess) return cuda_fail(c, e, "cudaGetSymbolAddress(static scratch)");
     float *m = c->t.m + (size_t)shard * c->E, *M = c->t.M + (size_t)shard * c->E;
     e = tpq_launch_calibrate(static_cast<const uint16_t *>(y), n_seq, S, stride, c->E, m, M, c->counts[shard], c->gamma,
@@ -339,6 +341,18 @@ tpq_status tpq_get_features(tpq_ctx *c, int32_t *hp_out)
     if (c->k > 0) {
         if (!hp_out) return fail(c, TPQ_ERR_INVALID_ARG, "NULL output");
         TPQ_CUDA(c, cudaMemcpy(hp_out, c->t.hp_idx, (size_t)c->k * sizeof(int32_t), cudaMemcpyDeviceToHost));
+    }
+    return TPQ_OK;
+}
+
+tpq_status tpq_get_slot_order(tpq_ctx *c, int32_t *slot_out)
+{
+    if (!c) return TPQ_ERR_INVALID_ARG;
+    c->err[0] = 0;
+    if (c->k < 0) return fail(c, TPQ_ERR_BAD_STATE, "no feature set yet");
+    if (c->E - c->k > 0) {
+        if (!slot_out) return fail(c, TPQ_ERR_INVALID_ARG, "NULL output");
+        TPQ_CUDA(c, cudaMemcpy(slot_out, c->t.lp_idx, (size_t)(c->E - c->k) * sizeof(int32_t), cudaMemcpyDeviceToHost));
     }
     return TPQ_OK;
 }

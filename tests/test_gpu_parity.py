@@ -62,7 +62,7 @@ def test_generic_path_odd_shapes(N, T, E, k):
 @pytest.mark.parametrize("N,T,E,k", [(2, 16, 256, 4), (3, 17, 130, 2), (2, 5, 253, 9), (4, 67, 512, 8), (2, 3, 64, 0),
                                      (8, 33, 1024, 16), (2, 129, 5120, 80), (3, 50, 520, 16)])
 def test_other_code_widths(bits, N, T, E, k):
-    """The method at lower and higher precision (Section 4 / Figure 3): b-bit codes, step R/(2^b - 1),
+    """Other code widths (Section 4 / Figure 3): b-bit codes, step R/(2^b - 1),
     payloads bit-exact against the oracle (codes straddle bytes and words for b = 3, 5, 6, 7), sums in
     tolerance, bits per value b + (16-b)k/E up to the pad."""
     _full_pipeline(_workload(N, T, E, 19 * E + T + bits), k, binding.PATH_AUTO, bits=bits)

@@ -1,5 +1,4 @@
-"""Pins for the oracle at code widths other than 4 bits (the method "at lower and higher precision",
-Section 4 / Figure 3): closed-form bit count, brute-force nearest level, a bit stream written out with
+"""Pins for the oracle at code widths other than 4 bits (Section 4 / Figure 3): closed-form bit count, brute-force nearest level, a bit stream written out with
 Python integers, the error bound of a symmetric quantiser, and the two oracles against each other."""
 from fractions import Fraction
 

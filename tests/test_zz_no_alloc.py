@@ -5,7 +5,8 @@ belongs to a pool, a framework that forbids allocation after start-up, or code t
 device-wide synchronisation hidden in cudaFree.  tpq_calibrate_ranges may grow its scratch buffer; the
 variant tested here keeps that scratch in a fixed array inside the library instead.  The test drives it
 through the C ABI and checks, on two calls in a row, that it leaves exactly the state the ordinary entry
-point leaves (bit for bit, the tolerance every calibration test uses), that the array's stale contents
+point leaves and the state the CPU oracle computes from the same sequences (Eq. 1-2; bit for bit, the
+tolerance every calibration test uses), that the array's stale contents
 from the first call do not leak into the second, and that an oversized call is refused with a clear
 error and launches nothing.  It is collected last so that a run that stops at the first failure has
 already run everything else."""
@@ -16,6 +17,8 @@ import torch
 pytestmark = pytest.mark.gpu
 
 from paper_2411_07942_b200 import binding, synth  # noqa: E402
+
+import oracle  # noqa: E402
 
 import gpu_util as gu  # noqa: E402
 
@@ -35,6 +38,8 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
     first, second = _cal(E, 5, 300, 11), _cal(E, 3, 77, 12)      # different shapes: different scratch layouts
     ref = binding.Tpq(2, E)
     na = binding.Tpq(2, E)
+    orc = oracle.c()
+    state = {0: (None, None, 0), 1: (None, None, 0)}      # the oracle's (m, M, count) per shard
     for shard, cal in ((0, first), (0, second), (1, second)):
         d = gu.dev_bf16(cal)
         n_seq, S, _ = cal.shape
@@ -43,6 +48,8 @@ def test_noalloc_matches_the_allocating_entry_point_twice_in_a_row():
         torch.cuda.synchronize()
         a, b = ref.get_ranges(with_R=False), na.get_ranges(with_R=False)
         assert gu.bits_equal(a[0], b[0]) and gu.bits_equal(a[1], b[1])
+        state[shard] = orc.calibrate(*state[shard], cal, 0.01)
+        assert gu.bits_equal(b[0][shard], state[shard][0]) and gu.bits_equal(b[1][shard], state[shard][1])
     assert na.device_status() == 0
     # the two contexts now select the same features and steps
     assert ref.select_features(-1).tolist() == na.select_features(-1).tolist()
@@ -65,6 +72,23 @@ def test_noalloc_strided_and_generic_shapes():
         assert gu.bits_equal(a[0], b[0]) and gu.bits_equal(a[1], b[1])
         ref.close()
         na.close()
+
+
+def test_noalloc_near_its_limit_against_the_oracle():
+    """100 sequences x 8192 features fill 78 % of the array; the result is the oracle's.  (The branch that
+    lowers the row-split count to fit the array needs more than 512 SMs' worth of splits and is not
+    reachable on this GPU: 8 x 148 x 256 partial extremes always fit.)"""
+    E, n_seq, S = 8192, 100, 24
+    cal = _cal(E, n_seq, S, 31)
+    d = gu.dev_bf16(cal)
+    na = binding.Tpq(1, E)
+    na.calibrate_ranges_noalloc(0, d.data_ptr(), n_seq, S)
+    torch.cuda.synchronize()
+    m, M = na.get_ranges(with_R=False)
+    om, oM, _ = oracle.c().calibrate(None, None, 0, cal, 0.01)
+    assert gu.bits_equal(m[0], om) and gu.bits_equal(M[0], oM)
+    assert na.device_status() == 0
+    na.close()
 
 
 def test_noalloc_rejects_what_does_not_fit():
