@@ -127,42 +127,79 @@ class AllGatherExchange:
                            bias_ptr=bias_ptr)
 
 
-class PushExchange:
-    """The fused exchange.  Receive buffers live in symmetric memory when there is more than one rank
-    (every rank maps every peer's buffer); with one rank the buffer is a plain device tensor."""
+@dataclass
+class PeerBuffers:
+    """One receive buffer per rank, each mapped by every rank: peer_ptrs[p] is the address at which THIS rank
+    reaches rank p's buffer (peer_ptrs[rank] is its own).  `keep` holds whatever owns the memory."""
+    rank: int
+    peer_ptrs: list
+    keep: object = None
 
-    def __init__(self, tpq, T: int, group=None, device=None, timeout_ns: int = 1_000_000_000):
+
+def open_peer_buffers(total_bytes: int, group=None, device=None) -> PeerBuffers:
+    """Allocate this rank's receive buffer, zero it and exchange the mappings: symmetric memory when there is
+    more than one rank (every rank maps every peer's buffer), a plain device tensor otherwise."""
+    rank, world = _world(group)
+    device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+    if world == 1:
+        buf = torch.zeros(total_bytes, dtype=torch.uint8, device=device)
+        return PeerBuffers(0, [buf.data_ptr()], buf)
+    import torch.distributed._symmetric_memory as symm_mem
+    buf = symm_mem.empty(total_bytes, dtype=torch.uint8, device=device)
+    buf.zero_()
+    g = group if group is not None else dist.group.WORLD
+    hdl = symm_mem.rendezvous(buf, g)
+    ptrs = [int(p) for p in hdl.buffer_ptrs]
+    torch.cuda.synchronize(device)
+    dist.barrier(group=group)  # every buffer is zeroed before anyone pushes
+    return PeerBuffers(rank, ptrs, (buf, hdl))
+
+
+class PushExchange:
+    """The fused exchange.  Per step s, rank r stores its payload into slot (s & 1, r) of EVERY rank's receive
+    buffer and then the step's tag into the arrival word beside each copy; the reduction on rank r waits for
+    the N words of set s & 1 in its OWN buffer and reads its own N slots.  Peers are only ever stored to.
+
+    `buffers` (a PeerBuffers) may be handed in by the caller, e.g. addresses obtained from another
+    allocator, or host-made integers in a test of this bookkeeping; by default open_peer_buffers is used."""
+
+    def __init__(self, tpq, T: int, group=None, device=None, timeout_ns: int = 1_000_000_000, buffers=None,
+                 world: int | None = None):
         self.tpq = tpq
         self.T = T
         self.group = group
         self.rank, self.world = _world(group)
+        if buffers is not None:
+            self.rank = buffers.rank
+            self.world = world if world is not None else len(buffers.peer_ptrs)
         if self.world != tpq.N:
             raise ValueError(f"context has {tpq.N} shards, the group {self.world} ranks")
         self.layout = ReceiveLayout(self.world, tpq.payload_bytes(T))
         self.timeout_ns = timeout_ns
         self.step_no = 0
-        device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
-        if self.world == 1:
-            self.buf = torch.zeros(self.layout.total_bytes, dtype=torch.uint8, device=device)
-            self.peer_ptrs = [self.buf.data_ptr()]
-        else:
-            import torch.distributed._symmetric_memory as symm_mem
-            self.buf = symm_mem.empty(self.layout.total_bytes, dtype=torch.uint8, device=device)
-            self.buf.zero_()
-            g = group if group is not None else dist.group.WORLD
-            self._hdl = symm_mem.rendezvous(self.buf, g)
-            self.peer_ptrs = [int(p) for p in self._hdl.buffer_ptrs]
-            torch.cuda.synchronize(device)
-            dist.barrier(group=group)  # every buffer is zeroed before anyone pushes
+        self.buffers = buffers if buffers is not None else open_peer_buffers(self.layout.total_bytes, group, device)
+        if len(self.buffers.peer_ptrs) != self.world:
+            raise ValueError(f"{len(self.buffers.peer_ptrs)} peer mappings for {self.world} ranks")
+        self.peer_ptrs = list(self.buffers.peer_ptrs)
+
+    def push_args(self, step: int):
+        """(destinations, arrival words, tag) of this rank's push in `step`: one pair per rank, in rank order."""
+        L, r = self.layout, self.rank
+        return ([p + L.slot(step, r) for p in self.peer_ptrs], [p + L.word(step, r) for p in self.peer_ptrs],
+                L.epoch(step))
+
+    def reduce_args(self, step: int):
+        """(payload addresses in device order, first arrival word, tag) of this rank's reduction in `step`:
+        all in its own buffer; the N words of a set are adjacent, one wait covers them."""
+        L, mine = self.layout, self.peer_ptrs[self.rank]
+        return [mine + L.slot(step, i) for i in range(self.world)], mine + L.word(step, 0), L.epoch(step)
 
     def step(self, y_ptr: int, out_ptr: int, out_dtype: int, stream: int = 0, bias_ptr: int | None = None) -> None:
         """One synchronisation: push own shard to every rank, wait for all N arrivals, reduce locally."""
-        L, r, s = self.layout, self.rank, self.step_no
-        epoch = L.epoch(s)
-        self.tpq.quantize_pack_push(r, y_ptr, self.T, [p + L.slot(s, r) for p in self.peer_ptrs],
-                                    [p + L.word(s, r) for p in self.peer_ptrs], L.slot_bytes, epoch, stream=stream)
-        mine = self.peer_ptrs[r]
-        self.tpq.dequant_reduce([mine + L.slot(s, i) for i in range(self.world)], self.T, out_ptr, out_dtype,
-                                stream=stream, bias_ptr=bias_ptr, arrived_ptr=mine + L.word(s, 0), epoch=epoch,
-                                timeout_ns=self.timeout_ns)
+        s = self.step_no
+        dst, words, epoch = self.push_args(s)
+        self.tpq.quantize_pack_push(self.rank, y_ptr, self.T, dst, words, self.layout.slot_bytes, epoch, stream=stream)
+        payloads, first_word, epoch = self.reduce_args(s)
+        self.tpq.dequant_reduce(payloads, self.T, out_ptr, out_dtype, stream=stream, bias_ptr=bias_ptr,
+                                arrived_ptr=first_word, epoch=epoch, timeout_ns=self.timeout_ns)
         self.step_no += 1
