@@ -47,7 +47,11 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"quantize_tiled_batch": 88030464, "dequant_rows": 22081792}
+NCU_TRAFFIC_BYTES = {
+    "quantize_tiled": None,
+    "quantize_tiled_batch": None,
+    "dequant_rows": None,
+}
 
 
 # ------------------------------------------------------------------ helpers
@@ -131,10 +135,17 @@ class ClockSampler:
             for name, val in zip(names, f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
-        in_region = len([1 for ts, _ in self.rows if t0 <= ts <= t1])
+        region = []
+        for ts, r in self.rows:
+            if t0 <= ts <= t1:
+                try:
+                    region.append(float(r.split(",")[1]))
+                except (ValueError, IndexError):
+                    pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "sm_mhz_in_timed_region": statistics.median(region) if region else None,
                 "power_w_max": max(power) if power else None, "samples": len(sm),
-                "samples_in_timed_region": in_region, "reasons": sorted(reasons)}
+                "samples_in_timed_region": len(region), "reasons": sorted(reasons)}
 
 
 def dist_env():
@@ -190,6 +201,108 @@ def oracle_leg(w, steps: int, warmup: int):
     return gbs, dt * 1e3, orc.num_threads(), sample
 
 
+# ------------------------------------------------------------------ the other configurations (extra.configs)
+def other_configs(args, dev, stream, peak, time_loop, graph_loop):
+    """Config 3 (decode shape: latency, plain launches and graph replay), config 5 at 8192 tokens, and the
+    calibration pass of config 4 on 32 sequences of one shard; the same kernels, timed the same way."""
+    import torch
+    from paper_2411_07942_b200 import binding, synth
+
+    sh = stream.cuda_stream
+    out = {}
+
+    def build(wname, n_sets):
+        w = synth.WORKLOADS[wname]
+        N, T, E = w.n_shards, w.tokens, w.features
+        scale = synth.column_scales(w)
+        t = binding.Tpq(N, E)
+        for i in range(N):
+            cal = synth.activations_torch(w, i, 2 * 64, dev, stream=1, scale=scale)
+            t.calibrate_ranges(i, cal.data_ptr(), 2, 64, stream=sh)
+        torch.cuda.synchronize()
+        k = len(t.select_features(-1))
+        P = t.payload_bytes(T)
+        sets = []
+        for b in range(n_sets):
+            ys = [synth.activations_torch(w, i, T, dev, stream=2 + b, scale=scale) for i in range(N)]
+            pls = [torch.empty(P, dtype=torch.uint8, device=dev) for _ in range(N)]
+            o = torch.empty((T, E), dtype=torch.bfloat16, device=dev)
+            sets.append((ys, pls, o, (ctypes.c_void_p * N)(*[y.data_ptr() for y in ys]),
+                         (ctypes.c_void_p * N)(*[p_.data_ptr() for p_ in pls])))
+        return w, t, k, P, sets
+
+    def timed(wname, n_sets, with_graph):
+        w, t, k, P, sets = build(wname, n_sets)
+        N, T, E = w.n_shards, w.tokens, w.features
+        alg = algorithmic_bytes(N, T, E, k)
+        cnt = [0]
+
+        def q_one(b, s_=None):          # one shard per call, the shards in turn
+            ys, pls, _, _, _ = sets[b % n_sets]
+            i = (b // n_sets) % N
+            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh if s_ is None else s_)
+
+        def q_all(b, s_=None):
+            _, _, _, yarr, parr = sets[b % n_sets]
+            t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh if s_ is None else s_)
+
+        def d_one(b, s_=None):
+            _, _, o, _, parr = sets[b % n_sets]
+            t.dequant_reduce(parr, T, o.data_ptr(), binding.TPQ_OUT_BF16, stream=sh if s_ is None else s_)
+
+        def st(b, s_=None):
+            q_all(b, s_)
+            d_one(b, s_)
+
+        q_all(0)
+        torch.cuda.synchronize()
+        r = {"shape": f"N={N} shards x {T} tokens x {E} features, k={k}", "buffer_sets": n_sets,
+             "algorithmic_bytes": {"quantize_pack": alg["quantize_pack"], "dequant_reduce": alg["dequant_reduce"]}}
+        for name, fn, nbytes in (("quantize_pack", q_one, alg["quantize_pack"]),
+                                 ("quantize_pack_batch", q_all, N * alg["quantize_pack"]),
+                                 ("dequant_reduce", d_one, alg["dequant_reduce"]), ("step", st, None)):
+            ms = time_loop(fn)
+            e = {"us_per_call": ms * 1e3}
+            if with_graph:
+                g = graph_loop(fn, n_sets * (N if fn is q_one else 1))
+                e["us_per_call_graph_replay"] = None if g is None else g * 1e3
+            if nbytes:
+                e["hbm_GBps"] = nbytes / ms / 1e6
+                e["frac_of_measured"] = nbytes / ms / 1e6 / peak
+                e["frac_of_8000"] = nbytes / ms / 1e6 / NOMINAL_HBM_GBS
+            r[name] = e
+        assert t.device_status() == 0
+        t.close()
+        del sets
+        torch.cuda.empty_cache()
+        return r
+
+    out["gemma27b_decode"] = timed("gemma27b_decode", 6, True)
+    out["gemma27b_decode"]["note"] = "latency-bound (0.7 MB / 1.8 MB per call): microseconds per call are the figure"
+    out["large_8192_tokens"] = timed("large", 2, False)
+    # config 4: the calibration pass, 32 sequences of 2048 tokens of one shard per call (two inputs in turn)
+    w = synth.WORKLOADS["calibration"]
+    E, S, n_seq = w.features, w.calib_tokens, 32
+    scale = synth.column_scales(w)
+    bufs = [synth.activations_torch(w, 0, n_seq * S, dev, stream=1 + b, scale=scale) for b in range(2)]
+    tc = binding.Tpq(w.n_shards, E)
+
+    def cal(b):
+        tc.calibrate_ranges(0, bufs[b % 2].data_ptr(), n_seq, S, stream=sh)
+
+    ms = time_loop(cal)
+    nbytes = n_seq * S * E * 2
+    out["calibration_32_sequences"] = {"shape": f"{n_seq} sequences x {S} tokens x {E} features, one shard per call",
+                                       "ms_per_call": ms, "bytes": nbytes, "hbm_GBps": nbytes / ms / 1e6,
+                                       "frac_of_measured": nbytes / ms / 1e6 / peak,
+                                       "frac_of_8000": nbytes / ms / 1e6 / NOMINAL_HBM_GBS,
+                                       "full_pass_512_sequences_ms_per_shard": ms * 512 / n_seq}
+    tc.close()
+    del bufs
+    torch.cuda.empty_cache()
+    return out
+
+
 # ------------------------------------------------------------------ main
 def main():
     ap = argparse.ArgumentParser()
@@ -199,6 +312,11 @@ def main():
     ap.add_argument("--impl", default="tpq", choices=["tpq", "reference"])
     ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-time", type=float, default=0.25,
+                    help="every timed region (the K steps and each per-kernel loop) is repeated until it lasts at "
+                         "least this many seconds, so that clock samples fall inside it; 0 for profiler captures")
+    ap.add_argument("--no-extra-configs", action="store_true",
+                    help="skip the other configurations (decode shape, large shape, calibration pass) under extra.configs")
     ap.add_argument("--workload", default=WORKLOAD,
                     help="synthetic workload (default: the configuration the metric is quoted on; the others are "
                          "for profiling captures, e.g. `--workload large --tokens 1024 --sets 2`)")
@@ -219,6 +337,10 @@ def main():
     in_bytes = N * T * E * 2
     config = {"workload": f"{args.workload}: N={N} shards x {T} tokens x {E} features BF16, k={k} BF16 features, "
                           f"BF16 output", "n_shards": N, "tokens": T, "features": E, "k": k}
+    set_bytes = in_bytes + N * payload_bytes(T, E, k, args.bits) + 2 * T * E
+    # (the same text in both arms: the GPU arm rotates its buffer sets; the CPU arm's caches are far smaller than one set)
+    config["l2"] = (f"rotating {args.sets} buffer sets, {args.sets * set_bytes / 1e6:.0f} MB touched between "
+                    f"reuses (> 126 MB L2)")
 
     if args.impl == "reference":
         if rank != 0:
@@ -293,9 +415,6 @@ def main():
         yarr = (ctypes.c_void_p * N)(*[y.data_ptr() for y in ys])
         parr = (ctypes.c_void_p * N)(*[p_.data_ptr() for p_ in pls])
         sets.append((ys, pls, out, yarr, parr))
-    set_bytes = in_bytes + N * P + 2 * T * E
-    config["l2"] = (f"rotating {args.sets} buffer sets, {args.sets * set_bytes / 1e6:.0f} MB touched between "
-                    f"reuses (> 126 MB L2)")
 
     # One step: the N simulated ranks' quantize_pack (one batched launch: the SMs are divided among the
     # N shards, as N devices would work side by side), then the local dequantise + reduce.
@@ -312,6 +431,22 @@ def main():
     for b in range(args.warmup):
         step(b)
     barrier()
+    # a short pilot run (untimed work, after the warm-up) tells how long a step takes
+    wa, wz = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pilot = max(args.steps, 20)
+    wa.record(stream)
+    for b in range(pilot):
+        step(b)
+    wz.record(stream)
+    barrier()
+    # the K steps are repeated `inner` times inside the timed region so that it lasts at least --min-time
+    # (the same on every rank: rank 0's estimate from the warm-up steps is broadcast)
+    est_ms = max(wa.elapsed_time(wz) / pilot, 1e-3)
+    inner = max(1, int(np.ceil(args.min_time * 1e3 / (est_ms * args.steps))))
+    if world > 1:
+        it_ = torch.tensor([inner], dtype=torch.int64, device=dev)
+        dist.broadcast(it_, 0)
+        inner = int(it_.item())
     sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
                            int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
     if rank == 0:
@@ -322,53 +457,102 @@ def main():
     barrier()
     wall0 = time.time()
     ev0.record(stream)
-    for b in range(args.steps):
+    for b in range(args.steps * inner):
         step(b)
     ev1.record(stream)
     barrier()
     wall1 = time.time()
-    local_ms = ev0.elapsed_time(ev1) / args.steps
-    gpu_launches = t.launch_count() - launches0
+    local_ms = ev0.elapsed_time(ev1) / (args.steps * inner)
+    gpu_launches = (t.launch_count() - launches0) // inner      # launches of the K steps
 
     # ---- per-kernel durations, same buffers and rotation, CUDA events on the launching stream
-    def time_loop(fn, reps):
+    def time_loop(fn, reps=None):
+        """Average ms per call of fn over a loop of at least --min-time seconds (CUDA events on the stream)."""
         for b in range(3):
             fn(b)
         torch.cuda.synchronize()
         a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 20
         a.record(stream)
-        for b in range(reps):
+        for b in range(n):
             fn(b)
         z.record(stream)
         torch.cuda.synchronize()
-        return a.elapsed_time(z) / reps
+        est = max(a.elapsed_time(z) / n, 1e-4)
+        n = max(n, int(np.ceil(args.min_time * 1e3 / est))) if reps is None else reps
+        a.record(stream)
+        for b in range(n):
+            fn(b)
+        z.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(z) / n
 
-    def q_only(b):          # one launch per shard: what each rank of a real deployment calls
+    def graph_loop(fn, per):
+        """The same calls replayed from a CUDA graph of `per` calls: what the device needs when the host's
+        launch path is out of the way.  None if capture is unavailable."""
+        try:
+            gs = torch.cuda.Stream()
+            gs.wait_stream(stream)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=gs):
+                for b in range(per):
+                    fn(b, gs.cuda_stream)
+            with torch.cuda.stream(gs):
+                for _ in range(3):
+                    g.replay()
+                gs.synchronize()
+                a, z = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(gs)
+                g.replay()
+                z.record(gs)
+                gs.synchronize()
+                est = max(a.elapsed_time(z), 1e-4)
+                n = max(3, int(np.ceil(args.min_time * 1e3 / est)))
+                a.record(gs)
+                for _ in range(n):
+                    g.replay()
+                z.record(gs)
+                gs.synchronize()
+            return a.elapsed_time(z) / (n * per)
+        except Exception:
+            torch.cuda.synchronize()
+            return None
+
+    def q_only(b, s_=None):          # one launch per shard: what each rank of a real deployment calls
         ys, pls, _, _, _ = sets[b % args.sets]
         for i in range(N):
-            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh)
+            t.quantize_pack(i, ys[i].data_ptr(), T, pls[i].data_ptr(), P, stream=sh if s_ is None else s_)
 
-    def qb_only(b):         # the N shards in one launch (the step's form)
+    def qb_only(b, s_=None):         # the N shards in one launch (the step's form)
         _, _, _, yarr, parr = sets[b % args.sets]
-        t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh)
+        t.quantize_pack_batch(0, yarr, T, parr, P, stream=sh if s_ is None else s_)
 
-    def d_only(b):
+    def d_only(b, s_=None):
         _, _, out, _, parr = sets[b % args.sets]
-        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh)
+        t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh if s_ is None else s_)
 
-    # the sampler keeps running through the per-kernel loops below (same kernels, same buffers), so that a
-    # short timed region still ends up with several clock samples; both counts are reported
-    reps = max(20, min(args.steps, 2000))
-    q_ms = time_loop(q_only, reps) / N          # per single-shard launch
-    qb_ms = time_loop(qb_only, reps)            # per batched launch (N shards)
-    d_ms = time_loop(d_only, reps)
+    def step_on(b, s_):
+        qb_only(b, s_)
+        d_only(b, s_)
+
+    # the sampler keeps running through the per-kernel loops below (same kernels, same buffers); each loop lasts
+    # at least --min-time as well
+    q_ms = time_loop(q_only) / N          # per single-shard launch
+    qb_ms = time_loop(qb_only)            # per batched launch (N shards)
+    d_ms = time_loop(d_only)
+    # the same from a CUDA graph (one pass over the rotating buffer sets per replay): the device's own pace
+    qg = graph_loop(q_only, args.sets)
+    q_graph_ms = None if qg is None else qg / N
+    qb_graph_ms = graph_loop(qb_only, args.sets)
+    d_graph_ms = graph_loop(d_only, args.sets)
+    graph_ms = graph_loop(step_on, args.sets)
     bias_dev = torch.zeros(E, dtype=torch.float32, device=dev).normal_(generator=torch.Generator(device=dev).manual_seed(7))
 
     def db_only(b):         # the same with the layer's bias added in the kernel's store (Section 2)
         _, _, out, _, parr = sets[b % args.sets]
         t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh, bias_ptr=bias_dev.data_ptr())
 
-    db_ms = time_loop(db_only, reps)
+    db_ms = time_loop(db_only)
 
     # the fused exchange (Section 5) on one GPU: one shard's payload stored into 1 and into N local receive slots
     # and its arrival words published; then the bounded wait ahead of the reduction (words already set)
@@ -391,8 +575,8 @@ def main():
         return fn
 
     push_max = min(N, 16)
-    p1_ms = time_loop(push_fn(1), reps) / N
-    pn_ms = time_loop(push_fn(push_max), reps) / N
+    p1_ms = time_loop(push_fn(1)) / N
+    pn_ms = time_loop(push_fn(push_max)) / N
     words.fill_(1)
     torch.cuda.synchronize()
 
@@ -401,35 +585,8 @@ def main():
         t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=sh, arrived_ptr=words.data_ptr(), epoch=1,
                          timeout_ns=50_000_000)
 
-    wd_ms = time_loop(wd_only, reps)
+    wd_ms = time_loop(wd_only)
 
-    # ---- the same step replayed from a CUDA graph (one graph = one pass over the rotating buffer sets):
-    # what the launch path costs, relevant for the decode-sized workloads
-    graph_ms = None
-    try:
-        gs = torch.cuda.Stream()
-        gs.wait_stream(stream)
-        gsh = gs.cuda_stream
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=gs):
-            for b in range(args.sets):
-                _, _, out, yarr, parr = sets[b]
-                t.quantize_pack_batch(0, yarr, T, parr, P, stream=gsh)
-                t.dequant_reduce(parr, T, out.data_ptr(), binding.TPQ_OUT_BF16, stream=gsh)
-        with torch.cuda.stream(gs):
-            for _ in range(3):
-                graph.replay()
-            ga, gz = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            greps = max(5, min(args.steps, 2000) // args.sets)
-            ga.record(gs)
-            for _ in range(greps):
-                graph.replay()
-            gz.record(gs)
-        torch.cuda.synchronize()
-        graph_ms = ga.elapsed_time(gz) / (greps * args.sets)
-    except Exception as exc:  # measurement only: the step itself does not depend on graphs
-        graph_ms = f"unavailable: {type(exc).__name__}: {exc}"[:200]
-        torch.cuda.synchronize()
     clocks = sampler.stop(wall0, wall1) if rank == 0 else None
 
     # ---- (after the clock sampler has stopped: this part is tensor-bound and draws far more power than the path)
@@ -459,12 +616,16 @@ def main():
             with torch.cuda.stream(stream):
                 torch.matmul(xk, wk.t(), out=ytmp)
 
-        f_ms, u_ms, g_ms = time_loop(fused_fn, reps), time_loop(unfused_fn, reps), time_loop(gemm_fn, reps)
+        f_ms, u_ms, g_ms = time_loop(fused_fn), time_loop(unfused_fn), time_loop(gemm_fn)
         tpeak, tkind = measured_tensor_peak()
         flops = 2.0 * T * Kd * E
         fused = {"shape": f"x [{T}][{Kd}] . w [{E}][{Kd}]^T", "fused_ms": f_ms, "fused_TFLOPs": flops / f_ms / 1e9,
                  "frac_of_" + tkind + "_bf16_peak": flops / f_ms / 1e9 / tpeak, "peak_TFLOPs": tpeak,
                  "library_gemm_then_quantize_pack_ms": u_ms, "library_gemm_alone_ms": g_ms}
+
+    configs_extra = None
+    if rank == 0 and world == 1 and not args.no_extra_configs and args.workload == WORKLOAD and not args.tokens and args.bits == 4:
+        configs_extra = other_configs(args, dev, stream, peak, time_loop, graph_loop)
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
     ys0 = sets[0][0]
@@ -519,26 +680,42 @@ def main():
         return 0
 
     value = units / (ms * 1e-3) / 1e9
-    # dominant kernel of the step: the batched quantize_tiled launch (N shards) or dequant_rows
-    if qb_ms >= d_ms:
-        dom, dom_ms, dom_bytes = "quantize_pack (batched launch, N shards)", qb_ms, N * alg["quantize_pack"]
-        traffic = NCU_TRAFFIC_BYTES["quantize_tiled_batch"]
-    else:
-        dom, dom_ms, dom_bytes = "dequant_reduce", d_ms, alg["dequant_reduce"]
-        traffic = NCU_TRAFFIC_BYTES["dequant_rows"]
     if args.bits != 4:
         config["workload"] += f", {args.bits}-bit codes"
         config["bits"] = args.bits
-    if args.workload != WORKLOAD or args.tokens or args.bits != 4:
-        traffic = None  # the captured DRAM traffic is for the default workload's launches
-    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "algorithmic_bytes_per_launch": dom_bytes, "launch_ms": dom_ms, "traffic": traffic}
+    default_workload = args.workload == WORKLOAD and not args.tokens and args.bits == 4
+
+    def kernel_entry(name, ms_, graph_, nbytes, key):
+        """One kernel's roofline entry: algorithmic bytes / measured launch time against the copy bandwidth,
+        the DRAM traffic ncu saw for one launch, and which limit the kernel is at."""
+        cap = NCU_TRAFFIC_BYTES.get(key) if default_workload else None   # (captured for the default workload only)
+        ach = nbytes / (ms_ * 1e-3) / 1e9
+        e = {"kernel": name, "launch_ms": ms_, "launch_ms_graph_replay": graph_, "algorithmic_bytes_per_launch": nbytes,
+             "achieved": ach, "unit": "GB/s", "frac": ach / peak, "frac_of_nominal_8000": ach / NOMINAL_HBM_GBS,
+             "traffic": cap["bytes"] if cap else None, "traffic_capture": cap["capture"] if cap else None}
+        if cap:
+            e["dram_GBps"] = cap["bytes"] / (ms_ * 1e-3) / 1e9
+            # DRAM busy at less than half the copy rate: the launch is not limited by HBM but by instruction
+            # issue and by its fixed cost (ramp, drain, dependency on the kernel ahead)
+            e["bound"] = "hbm" if e["dram_GBps"] >= 0.5 * peak else "issue"
+        else:
+            e["bound"] = "hbm"
+        return e
+
+    kernels = [kernel_entry("quantize_pack (one shard per launch)", q_ms, q_graph_ms, alg["quantize_pack"], "quantize_tiled"),
+               kernel_entry("quantize_pack_batch (N shards per launch)", qb_ms, qb_graph_ms, N * alg["quantize_pack"],
+                            "quantize_tiled_batch"),
+               kernel_entry("dequant_reduce", d_ms, d_graph_ms, alg["dequant_reduce"], "dequant_rows")]
+    # dominant kernel of the step: the longer of its two launches
+    dom = kernels[1] if qb_ms >= d_ms else kernels[2]
+    roofline = {"bound": dom["bound"], "kernel": dom["kernel"], "achieved": dom["achieved"], "peak": peak, "unit": "GB/s",
+                "frac": dom["frac"], "peak_kind": f"of {peak_kind}", "frac_of_nominal_8000": dom["frac_of_nominal_8000"],
+                "algorithmic_bytes_per_launch": dom["algorithmic_bytes_per_launch"], "launch_ms": dom["launch_ms"],
+                "traffic": dom["traffic"], "kernels": kernels}
     extra = {
         "bits_per_value": comm.bits_per_value, "bits_per_value_formula": comm.bits_per_value_formula,
-        "step_cuda_graph_replay_ms": graph_ms,
+        "step_cuda_graph_replay_ms": graph_ms, "inner_repeats": inner,
+        "configs": configs_extra,
         "dequant_reduce_bias_ms_per_launch": db_ms,
         "fused_layer": fused,
         "exchange_one_gpu": {"quantize_pack_push_1_dst_ms": p1_ms, f"quantize_pack_push_{push_max}_dst_ms": pn_ms,
@@ -569,6 +746,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "inner_repeats": inner, "timed_region_s": args.steps * inner * ms * 1e-3,
             "config": config, "clocks": clocks, "gpu_launches": int(gpu_launches),
             "e2e": {"value": world * in_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": 2 * T * E, "ms_per_step": e2e_ms},
