@@ -48,9 +48,9 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 NCU_TRAFFIC_BYTES = {
-    "quantize_tiled": None,
-    "quantize_tiled_batch": None,
-    "dequant_rows": None,
+    "quantize_tiled": {"bytes": 21025024, "capture": "profiles/dram_traffic_llama13b_prefill.md"},
+    "quantize_tiled_batch": {"bytes": 84600000, "capture": "profiles/dram_traffic_llama13b_prefill.md"},
+    "dequant_rows": {"bytes": 22106624, "capture": "profiles/dram_traffic_llama13b_prefill.md"},
 }
 
 
