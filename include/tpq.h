@@ -63,7 +63,7 @@ typedef enum {
      * multiples of 8, 4-bit codes). */
     TPQ_OPT_KERNEL_PATH = 0,
     /* Which tiled kernel tpq_dequant_reduce uses when the tiled path is taken: 0 = chosen from the
-     * shape (default); 1 = row kernel (needs N <= 4 and (E-k)/8 <= 768); 2 = tensor-map panel kernel
+     * shape (default); 1 = row kernel (needs N <= 4 and (E-k)/8 <= 768, or N <= 8 and (E-k)/8 <= 640); 2 = tensor-map panel kernel
      * (needs N <= 16 and E-k a multiple of 32); 3 = copy-ring panel kernel.  A kernel that the shape
      * does not admit makes the call return TPQ_ERR_INVALID_ARG.  For tests and measurements: all
      * kernels give identical results. */

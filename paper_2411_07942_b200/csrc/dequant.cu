@@ -786,14 +786,15 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 }
 
 // ----------------------------------------------------------------------------------------------
-// Row kernel for N <= 4 devices and (E-k)/8 <= MAXT main threads.
+// Row kernel for N <= 8 devices and (E-k)/8 <= MAXT main threads.
 //
 // One persistent block per SM works on a run of adjacent rows, G at a time, with three kinds of warps:
 //   producer (1 warp)  sets up the barriers, waits for the kernel ahead in the stream and streams the
 //                      stages (a code-row block and a BF16 block per device, 2N 1-D bulk asynchronous
 //                      copies issued by 2N lanes) into a ring of shared-memory stages; "full" mbarriers;
-//   main (MAXT/32)     thread <-> 8 adjacent output features = one aligned word per device and row; its
-//                      N x 8 steps live in registers for the life of the block (0 at holes); straight-line
+//   main (MAXT/32)     thread <-> 8 adjacent output features = one aligned word per device and row; the
+//                      8 steps of each of the first four devices live in registers for the life of the block
+//                      (0 at holes), those of devices five to eight in the thread's own shared-memory slots; straight-line
 //                      decode + one 128-bit store per row.  A thread whose group contains a selected
 //                      feature then overwrites that lane of its own stores (same thread, same address:
 //                      ordered) with the sum the auxiliary warps left in shared memory;
@@ -807,13 +808,14 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 // Blocks and stages start on rows at which the code stream is 16-byte aligned (multiples of 4/gcd(4, L/8)).
 // ----------------------------------------------------------------------------------------------
 constexpr int DR_AUX = 96;          // auxiliary threads
+constexpr int DR_NREG = 4;          // devices whose steps a main thread keeps in registers
 constexpr int DR_PREFETCH_ROWS = 4; // rows whose bytes a block asks L2 for ahead of the dependency wait (measured: 2..8 alike, all: worse)
 
 // main threads (= 32-bit words of a code row a stage leaves room for) for a row of L8 words
 __host__ __device__ inline int dr_row_cap(int L8) { return L8 <= 640 ? 640 : 768; }
 
 struct DRLayout {
-    size_t lp_stage, hp_stage, stage, sums, sums_stage, bars, total;
+    size_t lp_stage, hp_stage, stage, sums, sums_stage, hi, hi_plane, bars, total;
 };
 __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int nstage)
 {
@@ -825,7 +827,11 @@ __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int ns
     l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
     l.sums = (size_t)nstage * l.stage;
     l.sums_stage = (((size_t)G * k * 4) + 15) & ~(size_t)15;  // one 32-bit slot per (row, rank)
-    l.bars = l.sums + (size_t)nstage * l.sums_stage;
+    // devices beyond the fourth: their steps do not fit a main thread's registers and live here, two planes of
+    // 16 bytes per (device, main thread); a thread reads back only what it wrote itself
+    l.hi = l.sums + (size_t)nstage * l.sums_stage;
+    l.hi_plane = (size_t)dr_row_cap((E - k) >> 3) * 16;
+    l.bars = l.hi + (size_t)(N > DR_NREG ? N - DR_NREG : 0) * 2 * l.hi_plane;
     l.total = l.bars + (size_t)nstage * 24;
     return l;
 }
@@ -906,6 +912,53 @@ __device__ __forceinline__ void rows_stage(uint32_t sa, uint32_t dev_step, uint3
             store_group<FP32OUT>(orow, 0, acc, 0u);
         }
         orow += out_row_bytes;
+    }
+}
+
+__device__ __forceinline__ float4 lds128f(uint32_t saddr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts128f(uint32_t saddr, float4 v)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// The same for more than DR_NREG devices (n of them, n <= 8): the first DR_NREG as above, the steps of the
+// others come from the thread's own slots in shared memory (hi: address of device DR_NREG's first plane, the
+// second plane hi_plane further, the next device 2 hi_plane further), loaded once per GR rows.
+template <int GR, uint32_t DEVSTEP, bool FP32OUT, bool HAS_BIAS>
+__device__ __forceinline__ void rows_stage_hi(uint32_t sa, uint32_t row_bytes, int n, const float2 (&sc)[DR_NREG][4],
+                                              uint32_t hi, uint32_t hi_plane, const DecodeConsts &dc, const float2 (&b)[4],
+                                              uint8_t *orow, int64_t out_row_bytes, bool live)
+{
+    float2 acc[GR][4];
+#pragma unroll
+    for (int r = 0; r < GR; ++r) {
+        decode8<true>(lds32(sa + (uint32_t)r * row_bytes), sc[0], acc[r], dc);
+#pragma unroll
+        for (int i = 1; i < DR_NREG; ++i) decode8(lds32(sa + (uint32_t)r * row_bytes + (uint32_t)i * DEVSTEP), sc[i], acc[r], dc);
+    }
+#pragma unroll
+    for (int i = DR_NREG; i < 8; ++i)
+        if (i < n) {
+            const float4 s0 = lds128f(hi + (uint32_t)(i - DR_NREG) * 2u * hi_plane);
+            const float4 s1 = lds128f(hi + (uint32_t)(i - DR_NREG) * 2u * hi_plane + hi_plane);
+            const float2 s[4] = {make_float2(s0.x, s0.y), make_float2(s0.z, s0.w), make_float2(s1.x, s1.y), make_float2(s1.z, s1.w)};
+#pragma unroll
+            for (int r = 0; r < GR; ++r) decode8(lds32(sa + (uint32_t)r * row_bytes + (uint32_t)i * DEVSTEP), s, acc[r], dc);
+        }
+    if (live) {
+#pragma unroll
+        for (int r = 0; r < GR; ++r) {
+            if (HAS_BIAS) {
+#pragma unroll
+                for (int h = 0; h < 4; ++h) acc[r][h] = __fadd2_rn(acc[r][h], b[h]);
+            }
+            store_group<FP32OUT>(orow + r * out_row_bytes, 0, acc[r], 0u);
+        }
     }
 }
 
@@ -1150,12 +1203,24 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     const int g = tid - 32 - DR_AUX;
     const bool live = g < L8;
     const int g_ld = live ? g : 0;
-    float2 sc[NMAX][4];
+    float2 sc[DR_NREG][4];
 #pragma unroll
-    for (int i = 0; i < NMAX; ++i) {
+    for (int i = 0; i < DR_NREG; ++i) {
 #pragma unroll
         for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
+    }
+    const uint32_t hi_plane = (uint32_t)lay.hi_plane;
+    const uint32_t hi_s = smem_s + (uint32_t)lay.hi + (uint32_t)g * 16u;  // this thread's slot of device DR_NREG
+    if constexpr (NMAX > DR_NREG) {
+        for (int i = DR_NREG; i < N; ++i) {
+            float2 s4[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
+            if (live) load_steps(p.s_k + (size_t)i * E, g, s4);
+            sts128f(hi_s + (uint32_t)(i - DR_NREG) * 2u * hi_plane, make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y));
+            sts128f(hi_s + (uint32_t)(i - DR_NREG) * 2u * hi_plane + hi_plane, make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y));
+        }
     }
     // the selected features among the thread's 8 ("holes": their lanes are overwritten with the sums)
     const uint32_t gd = live ? __ldg(p.grp + g) : 0u;
@@ -1191,19 +1256,33 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
         }
         const uint32_t sa = word_s + (uint32_t)st * stage_b;
         // whole stages run as straight-line code (rows per stage and device count known at compile time)
-        if (G == 4 && rows == 4) {
-            if (N == NMAX) rows_stage<NMAX, NMAX, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
-            else rows_stage<NMAX, 0, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+        if constexpr (NMAX > DR_NREG) {
+            // more devices than a thread holds steps for: row by row (two rows side by side would share the steps
+            // read from shared memory, but their sixteen sums do not fit the registers: measured 2.6 times slower)
+            if (G == 2) {
+#pragma unroll 1
+                for (int r = 0; r < rows; ++r)
+                    rows_stage_hi<1, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, row_b, N, sc, hi_s, hi_plane, dc, b,
+                                                                      orow + r * out_row_bytes, out_row_bytes, live);
+            } else {
+#pragma unroll 1
+                for (int r = 0; r < rows; ++r)
+                    rows_stage_hi<1, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, row_b, N, sc, hi_s, hi_plane, dc, b,
+                                                                      orow + r * out_row_bytes, out_row_bytes, live);
+            }
+        } else if (G == 4 && rows == 4) {
+            if (N == DR_NREG) rows_stage<DR_NREG, DR_NREG, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            else rows_stage<DR_NREG, 0, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
         } else if (G == 4 && rows == 2) {
-            rows_stage<NMAX, 0, 2, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            rows_stage<DR_NREG, 0, 2, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
         } else if (G == 2 && rows == 2) {
-            if (N == NMAX) rows_stage<NMAX, NMAX, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
-            else rows_stage<NMAX, 0, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            if (N == DR_NREG) rows_stage<DR_NREG, DR_NREG, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            else rows_stage<DR_NREG, 0, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
         } else {
 #pragma unroll 1
             for (int r = 0; r < rows; ++r)
-                rows_stage<NMAX, 0, 1, 0, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
-                                                             orow + r * out_row_bytes, out_row_bytes, live);
+                rows_stage<DR_NREG, 0, 1, 0, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                                                                orow + r * out_row_bytes, out_row_bytes, live);
         }
         if (warp_holes) {  // (uniform over the warp)
             if (!mbar_wait(smem_u32(&sums_ready[st]), parity)) {
@@ -1315,15 +1394,18 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
 {
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
-    // measured against the panel kernels: the row kernel wins with up to 4 devices at every input length
-    // (the panel kernels scale better with N)
-    if (N > 4) return false;
-    if (L8 > 768) return false;  // consumer threads (register budget per thread)
+    // up to 8 devices: the steps of the first four live in the main threads' registers, those of the others in
+    // shared memory (beyond that the panel kernels, whose registers do not grow with N, take over)
+    if (N > 8) return false;
+    if (L8 > (N > DR_NREG ? 640 : 768)) return false;  // consumer threads (register budget per thread)
     const int g0 = g0_of(c);
     // every block takes the same number of adjacent rows (a multiple of g0), so no block has more than g0 - 1
     // rows above the mean; it walks them four at a time where a ring of three such stages fits, else two
     int64_t rpb = (T + c->sm_count - 1) / c->sm_count;
     rpb = (rpb + g0 - 1) / g0 * g0;
+    // more than four devices: measured ahead of the copy-ring panel kernel on short inputs only (8 devices,
+    // 2048 x 5120: 22.9 against 24.7 us; level at 4096 tokens, behind from 8192 on)
+    if (N > DR_NREG && rpb > 16 && c->dq_kernel != 1) return false;
     int G = 4;
     if (rpb < 4 || dr_layout(N, E, k, 4, 3).total > (size_t)c->smem_optin) G = 2;
     if (G < g0) G = g0;
@@ -1500,8 +1582,11 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             int consumers = ((L8 + 31) / 32) * 32;
             if (consumers < 32) consumers = 32;
             cudaError_t e;
-            e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, consumers, smem, st)
-                                 : launch_rows<4, 768>(pp, fp32_out, grid, consumers, smem, st);
+            if (c->N > DR_NREG)
+                e = launch_rows<8, 640>(pp, fp32_out, grid, consumers, smem, st);
+            else
+                e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, consumers, smem, st)
+                                     : launch_rows<4, 768>(pp, fp32_out, grid, consumers, smem, st);
             if (e != cudaSuccess) return e;
             ++*launches;
             return cudaGetLastError();

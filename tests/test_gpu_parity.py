@@ -183,7 +183,8 @@ def test_row_kernel_equals_generic_on_clustered_feature_sets():
         t.close()
 
 
-@pytest.mark.parametrize("N,T,E,k", [(4, 37, 512, 32), (2, 301, 1024, 32), (3, 16, 4096, 64), (4, 2, 256, 0), (1, 65, 6144, 96)])
+@pytest.mark.parametrize("N,T,E,k", [(4, 37, 512, 32), (2, 301, 1024, 32), (3, 16, 4096, 64), (4, 2, 256, 0), (1, 65, 6144, 96),
+                                     (8, 70, 1056, 32), (5, 33, 4096, 64), (7, 130, 520, 8)])
 def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
     """The row, tensor-map panel and copy-ring panel kernels forced in turn on shapes that admit all three
     (short inputs included, where the automatic choice would not pick them): FP32 and BF16 outputs are
@@ -218,12 +219,12 @@ def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
         assert np.array_equal(outs[name][0], outs["generic"][0]), name
         assert np.array_equal(outs[name][1], outs["generic"][1]), name
     # a kernel the shape does not admit is refused, not silently replaced
-    t2 = binding.Tpq(5, 512)
-    gu.calibrate_both(t2, [synth.calibration_np(_workload(5, 4, 512, 3, calib=(2, 8)), i) for i in range(5)])
+    t2 = binding.Tpq(9, 512)
+    gu.calibrate_both(t2, [synth.calibration_np(_workload(9, 4, 512, 3, calib=(2, 8)), i) for i in range(9)])
     t2.select_features(8)
     t2.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, binding.DQ_ROWS)
     with pytest.raises(binding.TpqError):
-        t2.dequant_reduce([pls[0].data_ptr()] * 5, 1, torch.empty((1, 512), dtype=torch.bfloat16, device="cuda").data_ptr())
+        t2.dequant_reduce([pls[0].data_ptr()] * 9, 1, torch.empty((1, 512), dtype=torch.bfloat16, device="cuda").data_ptr())
     t.close()
     t2.close()
 
