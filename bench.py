@@ -442,7 +442,7 @@ def main():
     # the K steps are repeated `inner` times inside the timed region so that it lasts at least --min-time
     # (the same on every rank: rank 0's estimate from the warm-up steps is broadcast)
     est_ms = max(wa.elapsed_time(wz) / pilot, 1e-3)
-    inner = max(1, int(np.ceil(args.min_time * 1e3 / (est_ms * args.steps))))
+    inner = max(1, int(np.ceil(1.2 * args.min_time * 1e3 / (est_ms * args.steps))))
     if world > 1:
         it_ = torch.tensor([inner], dtype=torch.int64, device=dev)
         dist.broadcast(it_, 0)
