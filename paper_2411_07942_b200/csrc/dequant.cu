@@ -801,29 +801,34 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 //                      stages (a code-row block and a BF16 block per device, 2N 1-D bulk asynchronous
 //                      copies issued by 2N lanes) into a ring of shared-memory stages; "full" mbarriers;
 //   main (MAXT/32)     thread <-> 8 adjacent output features = one aligned word per device and row; the
-//                      8 steps of each of the first four devices live in registers for the life of the block
-//                      (0 at holes), those of devices five to eight in the thread's own shared-memory slots; straight-line
-//                      decode + one 128-bit store per row.  A thread whose group contains a selected
-//                      feature then overwrites that lane of its own stores (same thread, same address:
-//                      ordered) with the sum the auxiliary warps left in shared memory;
-//   auxiliary (3)      per stage, from shared memory only: (1) the sums of the devices' BF16 values of every
-//                      (row, selected feature), two adjacent ranks per thread, left in shared memory in
-//                      the output's format ("sums" barrier); (2) the last k columns of the output, which no
-//                      main thread covers: an unselected one is a filler feature, decoded from the hole's
-//                      slot that carries its codes, a selected one takes its sum; lane <-> column, so the
-//                      small stores of a warp are adjacent.
+//                      8 steps of every device live in registers for the life of the block (0 at holes);
+//                      straight-line decode + one 128-bit store per row.  A thread whose group contains a
+//                      selected feature then overwrites that lane of its own stores (same thread, same
+//                      address: ordered) with the sum the auxiliary warps left in shared memory;
+//   auxiliary (3 or 5) per stage, from shared memory only: (1) the sums of the devices' BF16 values of every
+//                      (row, selected feature), left in shared memory in the output's format ("sums"
+//                      barrier); (2) the last k columns of the output, which no main thread covers: an
+//                      unselected one is a filler feature, decoded from the hole's slot that carries its
+//                      codes, a selected one takes its sum; lane <-> column, so the small stores of a warp
+//                      are adjacent.
 // No warp ever waits for another one's global stores, and no block-wide barrier follows the prologue.
 // Blocks and stages start on rows at which the code stream is 16-byte aligned (multiples of 4/gcd(4, L/8)).
+//
+// Up to four devices (NMAX = 4) a block has a main thread for every group of the row.  With five to eight
+// (NMAX = the device count, 40 to 64 registers of steps per thread) the register file holds half as many
+// threads, so two blocks (on two SMs) share a run of rows: both stage the whole rows, each decodes one half
+// of the groups, adds up the selected features its own main threads overwrite and stores one half of the
+// last k columns; its auxiliary threads take one item (a sum or a column) each and, where they outnumber the
+// items, several rows of a stage side by side.
 // ----------------------------------------------------------------------------------------------
 constexpr int DR_AUX = 96;          // auxiliary threads
-constexpr int DR_NREG = 4;          // devices whose steps a main thread keeps in registers
 constexpr int DR_PREFETCH_ROWS = 4; // rows whose bytes a block asks L2 for ahead of the dependency wait (measured: 2..8 alike, all: worse)
 
 // main threads (= 32-bit words of a code row a stage leaves room for) for a row of L8 words
 __host__ __device__ inline int dr_row_cap(int L8) { return L8 <= 640 ? 640 : 768; }
 
 struct DRLayout {
-    size_t lp_stage, hp_stage, stage, sums, sums_stage, hi, hi_plane, bars, total;
+    size_t lp_stage, hp_stage, stage, sums, sums_stage, bars, total;
 };
 __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int nstage)
 {
@@ -835,11 +840,7 @@ __host__ __device__ inline DRLayout dr_layout(int N, int E, int k, int G, int ns
     l.stage = (size_t)N * (l.lp_stage + l.hp_stage);
     l.sums = (size_t)nstage * l.stage;
     l.sums_stage = (((size_t)G * k * 4) + 15) & ~(size_t)15;  // one 32-bit slot per (row, rank)
-    // devices beyond the fourth: their steps do not fit a main thread's registers and live here, two planes of
-    // 16 bytes per (device, main thread); a thread reads back only what it wrote itself
-    l.hi = l.sums + (size_t)nstage * l.sums_stage;
-    l.hi_plane = (size_t)dr_row_cap((E - k) >> 3) * 16;
-    l.bars = l.hi + (size_t)(N > DR_NREG ? N - DR_NREG : 0) * 2 * l.hi_plane;
+    l.bars = l.sums + (size_t)nstage * l.sums_stage;
     l.total = l.bars + (size_t)nstage * 24;
     return l;
 }
@@ -850,6 +851,7 @@ struct DRParams {
     int G, nstage;
     int first;               // rows of a block's first stage (<= G: a short first stage lands sooner)
     int pairs;               // main threads walk a stage two rows at a time in a rolled loop
+    int half_groups;         // (more than four devices) groups per block: two blocks share a run of rows
     int64_t rows_per_block;  // a block works on rows_per_block adjacent rows (a multiple of the number of
                              // rows after which the code stream is 16-byte aligned again)
 };
@@ -924,53 +926,6 @@ __device__ __forceinline__ void rows_stage(uint32_t sa, uint32_t dev_step, uint3
     }
 }
 
-__device__ __forceinline__ float4 lds128f(uint32_t saddr)
-{
-    float4 v;
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(saddr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts128f(uint32_t saddr, float4 v)
-{
-    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
-}
-
-// The same for more than DR_NREG devices (n of them, n <= 8): the first DR_NREG as above, the steps of the
-// others come from the thread's own slots in shared memory (hi: address of device DR_NREG's first plane, the
-// second plane hi_plane further, the next device 2 hi_plane further), loaded once per GR rows.
-template <int GR, uint32_t DEVSTEP, bool FP32OUT, bool HAS_BIAS>
-__device__ __forceinline__ void rows_stage_hi(uint32_t sa, uint32_t row_bytes, int n, const float2 (&sc)[DR_NREG][4],
-                                              uint32_t hi, uint32_t hi_plane, const DecodeConsts &dc, const float2 (&b)[4],
-                                              uint8_t *orow, int64_t out_row_bytes, bool live)
-{
-    float2 acc[GR][4];
-#pragma unroll
-    for (int r = 0; r < GR; ++r) {
-        decode8<true>(lds32(sa + (uint32_t)r * row_bytes), sc[0], acc[r], dc);
-#pragma unroll
-        for (int i = 1; i < DR_NREG; ++i) decode8(lds32(sa + (uint32_t)r * row_bytes + (uint32_t)i * DEVSTEP), sc[i], acc[r], dc);
-    }
-#pragma unroll
-    for (int i = DR_NREG; i < 8; ++i)
-        if (i < n) {
-            const float4 s0 = lds128f(hi + (uint32_t)(i - DR_NREG) * 2u * hi_plane);
-            const float4 s1 = lds128f(hi + (uint32_t)(i - DR_NREG) * 2u * hi_plane + hi_plane);
-            const float2 s[4] = {make_float2(s0.x, s0.y), make_float2(s0.z, s0.w), make_float2(s1.x, s1.y), make_float2(s1.z, s1.w)};
-#pragma unroll
-            for (int r = 0; r < GR; ++r) decode8(lds32(sa + (uint32_t)r * row_bytes + (uint32_t)i * DEVSTEP), s, acc[r], dc);
-        }
-    if (live) {
-#pragma unroll
-        for (int r = 0; r < GR; ++r) {
-            if (HAS_BIAS) {
-#pragma unroll
-                for (int h = 0; h < 4; ++h) acc[r][h] = __fadd2_rn(acc[r][h], b[h]);
-            }
-            store_group<FP32OUT>(orow + r * out_row_bytes, 0, acc[r], 0u);
-        }
-    }
-}
-
 // Marks a value loaded once per thread as opaque: without it the compiler, short of registers, drops the value
 // and repeats its chain of (read-only) table loads at every use inside the stage loop, a trip to L2 each time.
 __device__ __forceinline__ void keep(int &v) { asm volatile("" : "+r"(v)); }
@@ -980,9 +935,10 @@ __device__ __forceinline__ void keep(float &v) { asm volatile("" : "+f"(v)); }
 // first row (within the block's run) of the block's it-th stage
 __device__ __forceinline__ int dr_stage_row(int it, int first, int G) { return it == 0 ? 0 : first + (it - 1) * G; }
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
-__global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRParams pp)
+template <int NMAX, int ROWCAP, int MAXT, int DAUX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+__global__ void __launch_bounds__(MAXT + DAUX + 32, 1) dequant_rows(const DRParams pp)
 {
+    constexpr bool SPLIT = NMAX > 4;  // two blocks share a run of rows, each decoding one half of the groups
     extern __shared__ __align__(128) uint8_t smem[];
     const DQParams &p = pp.q;
     const DXParams &x = pp.x;
@@ -990,7 +946,7 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     // warp 0 is the producer, then the auxiliary warps, then the main warps: where several warps of a
     // scheduler can issue, the one launched first goes first, and the few instructions of the producer and of
     // the auxiliary warps must not wait behind the main warps' many (as last warps they took 3 us per stage)
-    const int NT = blockDim.x - DR_AUX - 32;  // main threads
+    const int NT = blockDim.x - DAUX - 32;  // main threads
     const int N = p.N, E = p.E, k = p.k, G = pp.G, nstage = pp.nstage;
     const int L = E - k, L8 = L >> 3;
     const DRLayout lay = dr_layout(N, E, k, G, nstage);
@@ -998,7 +954,8 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     uint64_t *empty = full + nstage;
     uint64_t *sums_ready = empty + nstage;
     // this block's rows
-    const int64_t t_begin = blockIdx.x * pp.rows_per_block;
+    const int half = SPLIT ? (int)(blockIdx.x & 1u) : 0;
+    const int64_t t_begin = (int64_t)(SPLIT ? blockIdx.x >> 1 : blockIdx.x) * pp.rows_per_block;
     const int64_t t_end = (p.T - t_begin < pp.rows_per_block) ? p.T : t_begin + pp.rows_per_block;
     const int rows_mine = (int)(t_end - t_begin);
     constexpr int ESIZE = FP32OUT ? 4 : 2;
@@ -1016,6 +973,11 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     if constexpr (HAS_WAIT) {  // (an instantiation of its own: the plain call's prologue stays short)
         tpq_block_wait_arrivals(p.arr);
         __syncthreads();
+    } else if constexpr (SPLIT) {  // (one instantiation per device count already: decided at run time here)
+        if (p.arr.words != nullptr) {
+            tpq_block_wait_arrivals(p.arr);
+            __syncthreads();
+        }
     }
     if (tid < 32) {
         // ---------------- producer warp: lane 0 waits for the stage and arms its barrier, then the 2N
@@ -1024,8 +986,8 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
         if (pl == 0) {
             for (int s = 0; s < nstage; ++s) {
                 mbar_init(smem_u32(&full[s]), 1);
-                mbar_init(smem_u32(&empty[s]), (NT + DR_AUX) / 32);
-                mbar_init(smem_u32(&sums_ready[s]), DR_AUX / 32);
+                mbar_init(smem_u32(&empty[s]), (NT + DAUX) / 32);
+                mbar_init(smem_u32(&sums_ready[s]), DAUX / 32);
             }
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1087,8 +1049,134 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     uint32_t parity = 0;
     const int lane = tid & 31;
 
-    if (tid < 32 + DR_AUX) {
+    if (tid < 32 + DAUX) {
         // ---------------- auxiliary warps
+        if constexpr (SPLIT) {
+            // Two blocks share the rows.  Each adds up only the selected features that its own main threads
+            // overwrite (its holes, ranks [hs, he)) and stores one half of the last k columns, a selected one
+            // straight from the devices' BF16 values.  One item (a rank or a column) per thread and row; where
+            // the threads outnumber the items, RP rows of a stage are worked on side by side.  What a thread
+            // needs from the tables is loaded once.  Short rolled loops: this code runs once per stage, so
+            // straight-line code would pay an instruction fetch for every few instructions it executes.
+            const int at = tid - 32;
+            const int gfirst = half * pp.half_groups;
+            const int hs = half == 0 ? 0 : (gfirst < L8 ? (int)(__ldg(p.grp + gfirst) >> 8) : x.n_holes);
+            const int he = (half == 0 && pp.half_groups < L8) ? (int)(__ldg(p.grp + pp.half_groups) >> 8) : x.n_holes;
+            const int nr = he - hs;
+            const int c0 = half == 0 ? 0 : k / 2, nc = half == 0 ? k / 2 : k - k / 2;
+            const int W = nr + nc;  // items per row
+            const bool fast = W > 0 && W <= DAUX;
+            int RP = 1;
+            while (RP * 2 <= G && W * RP * 2 <= DAUX) RP *= 2;
+            const int rp = fast ? at / W : 0, idx = fast ? at - rp * W : 0;
+            const bool on = fast && rp < RP;
+            const bool is_col = idx < nc;
+            const int col = L + c0 + (is_col ? idx : 0);
+            const int ps = (on && is_col) ? __ldg(p.pos + col) : -1;
+            int do_sum = on && (!is_col || ps < 0), do_dec = on && is_col && ps >= 0;
+            // the selected feature whose values this thread adds up, and where the sum goes
+            const int rank = is_col ? (ps < 0 ? -ps - 1 : 0) : hs + idx - nc;
+            int to_out = is_col;
+            // a filler column's code sits at bits [sh, sh + 4) of a word of the hole's slot that carries it; it is
+            // decoded in place like the main threads' codes (mask, exponent pattern, bias and a step divided by
+            // the code's position), from the word shifted down by 16 for the upper four positions
+            const int slot = do_dec ? ps : 0;
+            uint32_t c_off = (uint32_t)(slot >> 3) * 4u;
+            const int sh = (slot & 7) * 4, shl = sh & 15;
+            uint32_t c_hi = sh >= 16 ? 16u : 0u, c_mask = 0xFu << shl;
+            float c_nb = -(8388608.0f + (float)(8 << shl));
+            float c_s[NMAX];
+#pragma unroll
+            for (int i = 0; i < NMAX; ++i)
+                c_s[i] = (do_dec && i < N) ? __ldg(p.s_k + (size_t)i * E + col) * (1.0f / (float)(1 << shl)) : 0.0f;
+            float c_b = 0.0f;  // the column's bias
+            if (HAS_BIAS && do_dec) c_b = __ldg(p.bias + col);
+            if (HAS_BIAS && do_sum) c_b = __ldg(p.bias + __ldg(x.hp_idx + rank));
+            uint32_t h_off = (uint32_t)rank * 2u, s_off = (uint32_t)rank * 4u;
+            keep(do_sum); keep(do_dec); keep(to_out); keep(c_off); keep(c_hi); keep(c_mask); keep(c_nb); keep(c_b);
+            keep(h_off); keep(s_off);
+#pragma unroll
+            for (int i = 0; i < NMAX; ++i) keep(c_s[i]);
+            uint32_t magic = 0x4B000000u;
+            keep(magic);
+            const uint32_t kb2 = (uint32_t)k * 2u, kb4 = (uint32_t)k * 4u, row_b = (uint32_t)L8 * 4u;
+            asm volatile("bar.sync 1, %0;" ::"r"(blockDim.x) : "memory");
+            for (int it = 0;; ++it) {
+                const int r0 = dr_stage_row(it, pp.first, G);
+                if (r0 >= rows_mine) break;
+                const int cap = it == 0 ? pp.first : G;
+                const int rows = rows_mine - r0 < cap ? rows_mine - r0 : cap;
+                if (!mbar_wait(smem_u32(&full[st]), parity)) {
+                    atomicExch(x.status, (int)TPQ_ERR_TIMEOUT);
+                    break;
+                }
+                const uint32_t stage = smem_s + (uint32_t)st * stage_b;
+                const uint32_t hp_s = stage + (uint32_t)N * lp_b;  // device 0's BF16 rows
+                const uint32_t sums = sums_s + (uint32_t)st * sums_b;
+                uint8_t *const obase = static_cast<uint8_t *>(p.out) + (t_begin + r0) * out_row_bytes;
+                if (do_sum) {
+                    uint32_t a = hp_s + h_off + (uint32_t)rp * kb2, o = sums + s_off + (uint32_t)rp * kb4;
+                    uint8_t *og = obase + rp * out_row_bytes + (int64_t)col * ESIZE;
+#pragma unroll 1
+                    for (int r = rp; r < rows; r += RP, a += RP * kb2, o += RP * kb4, og += RP * out_row_bytes) {
+                        float v = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < NMAX; ++i)
+                            if (i < N) v = __fadd_rn(v, __uint_as_float(lds16(a + (uint32_t)i * hp_b) << 16));
+                        if (HAS_BIAS) v = __fadd_rn(v, c_b);
+                        if (to_out) store_bits<FP32OUT>(og, out_bits<FP32OUT>(v));
+                        else sts32(o, out_bits<FP32OUT>(v));
+                    }
+                }
+                if (do_dec) {
+                    uint32_t a = stage + c_off + (uint32_t)rp * row_b;
+                    uint8_t *og = obase + rp * out_row_bytes + (int64_t)col * ESIZE;
+#pragma unroll 1
+                    for (int r = rp; r < rows; r += RP, a += RP * row_b, og += RP * out_row_bytes) {
+                        float v = 0.0f;
+#pragma unroll
+                        for (int i = 0; i < NMAX; ++i)
+                            if (i < N) {
+                                const uint32_t w = (lds32(a + (uint32_t)i * lp_b) ^ 0x88888888u) >> c_hi;
+                                v = __fmaf_rn(__fadd_rn(__uint_as_float(and_or(w, c_mask, magic)), c_nb), c_s[i], v);
+                            }
+                        if (HAS_BIAS) v = __fadd_rn(v, c_b);
+                        store_bits<FP32OUT>(og, out_bits<FP32OUT>(v));
+                    }
+                }
+                if (!fast) {  // (more items than threads: every item with its tables read where they are used)
+                    for (int q = at; q < W; q += DAUX) {
+                        const int cl = L + c0 + q, pc = q < nc ? __ldg(p.pos + cl) : -1;
+                        const int rk = q < nc ? -pc - 1 : hs + q - nc;
+                        for (int r = 0; r < rows; ++r) {
+                            float v = 0.0f;
+                            if (pc >= 0) {
+                                for (int i = 0; i < N; ++i)
+                                    v = __fmaf_rn(code_at(lds32(stage + (uint32_t)i * lp_b + (uint32_t)(r * L8 + (pc >> 3)) * 4u), (pc & 7) * 4),
+                                                  __ldg(p.s_k + (size_t)i * E + cl), v);
+                                if (HAS_BIAS) v = __fadd_rn(v, __ldg(p.bias + cl));
+                            } else {
+                                for (int i = 0; i < N; ++i)
+                                    v = __fadd_rn(v, __uint_as_float(lds16(hp_s + (uint32_t)i * hp_b + (uint32_t)(r * k + rk) * 2u) << 16));
+                                if (HAS_BIAS) v = __fadd_rn(v, __ldg(p.bias + __ldg(x.hp_idx + rk)));
+                            }
+                            if (q < nc) store_bits<FP32OUT>(obase + r * out_row_bytes + (int64_t)cl * ESIZE, out_bits<FP32OUT>(v));
+                            else sts32(sums + (uint32_t)(r * k + rk) * 4u, out_bits<FP32OUT>(v));
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&sums_ready[st]));  // (release: the sums above are visible to whoever waits)
+                    mbar_arrive(smem_u32(&empty[st]));
+                }
+                if (++st == nstage) {
+                    st = 0;
+                    parity ^= 1u;
+                }
+            }
+            return;
+        }
         // Thread c works on the c-th selected feature (its sum) and on column L + c of the output, row by
         // row, in short rolled loops: these warps run code that nobody else runs, once per stage, so
         // straight-line code would pay an instruction fetch for every few instructions it executes.
@@ -1163,8 +1251,10 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
                 break;
             }
             // (2) the last k columns
+            // (of two blocks that share the rows, the second one stores them)
+            const bool tail = !SPLIT || half == 1;
             uint8_t *const obase = static_cast<uint8_t *>(p.out) + (t_begin + r0) * out_row_bytes;
-            if (on) {
+            if (on && tail) {
                 uint32_t a = stage + c_off, sa = sums + c_sum;
                 uint8_t *o = obase + (int64_t)col * ESIZE;
 #pragma unroll 1
@@ -1181,7 +1271,7 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
                     store_bits<FP32OUT>(o, sel ? sum : out_bits<FP32OUT>(v));
                 }
             }
-            for (int c = at + DR_AUX; c < k; c += DR_AUX) {  // (more columns than threads)
+            for (int c = at + DR_AUX; tail && c < k; c += DR_AUX) {  // (more columns than threads)
                 const int cl = L + c, pc = __ldg(p.pos + cl);
                 for (int r = 0; r < rows; ++r) {
                     uint32_t bits;
@@ -1209,27 +1299,16 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
     }
 
     // ---------------- main warps
-    const int g = tid - 32 - DR_AUX;
-    const bool live = g < L8;
+    const int gl = tid - 32 - DAUX;
+    const int g = SPLIT ? half * pp.half_groups + gl : gl;
+    const bool live = SPLIT ? (gl < pp.half_groups && g < L8) : g < L8;
     const int g_ld = live ? g : 0;
-    float2 sc[DR_NREG][4];
+    float2 sc[NMAX][4];
 #pragma unroll
-    for (int i = 0; i < DR_NREG; ++i) {
+    for (int i = 0; i < NMAX; ++i) {
 #pragma unroll
         for (int h = 0; h < 4; ++h) sc[i][h] = make_float2(0.0f, 0.0f);
         if (live && i < N) load_steps(p.s_k + (size_t)i * E, g, sc[i]);
-    }
-    const uint32_t hi_plane = (uint32_t)lay.hi_plane;
-    const uint32_t hi_s = smem_s + (uint32_t)lay.hi + (uint32_t)g * 16u;  // this thread's slot of device DR_NREG
-    if constexpr (NMAX > DR_NREG) {
-        for (int i = DR_NREG; i < N; ++i) {
-            float2 s4[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) s4[h] = make_float2(0.0f, 0.0f);
-            if (live) load_steps(p.s_k + (size_t)i * E, g, s4);
-            sts128f(hi_s + (uint32_t)(i - DR_NREG) * 2u * hi_plane, make_float4(s4[0].x, s4[0].y, s4[1].x, s4[1].y));
-            sts128f(hi_s + (uint32_t)(i - DR_NREG) * 2u * hi_plane + hi_plane, make_float4(s4[2].x, s4[2].y, s4[3].x, s4[3].y));
-        }
     }
     // the selected features among the thread's 8 ("holes": their lanes are overwritten with the sums)
     const uint32_t gd = live ? __ldg(p.grp + g) : 0u;
@@ -1265,54 +1344,40 @@ __global__ void __launch_bounds__(MAXT + DR_AUX + 32, 1) dequant_rows(const DRPa
         }
         const uint32_t sa = word_s + (uint32_t)st * stage_b;
         // whole stages run as straight-line code (rows per stage and device count known at compile time)
-        if constexpr (NMAX > DR_NREG) {
-            // more devices than a thread holds steps for: row by row (two rows side by side would share the steps
-            // read from shared memory, but their sixteen sums do not fit the registers: measured 2.6 times slower)
-            if (G == 2) {
-#pragma unroll 1
-                for (int r = 0; r < rows; ++r)
-                    rows_stage_hi<1, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, row_b, N, sc, hi_s, hi_plane, dc, b,
-                                                                      orow + r * out_row_bytes, out_row_bytes, live);
-            } else {
-#pragma unroll 1
-                for (int r = 0; r < rows; ++r)
-                    rows_stage_hi<1, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, row_b, N, sc, hi_s, hi_plane, dc, b,
-                                                                      orow + r * out_row_bytes, out_row_bytes, live);
-            }
-        } else if (G == 4 && rows == 4 && !pp.pairs) {
-            if (N == DR_NREG) rows_stage<DR_NREG, DR_NREG, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
-            else rows_stage<DR_NREG, 0, 4, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+        if (G == 4 && rows == 4 && !pp.pairs) {
+            if (N == NMAX) rows_stage<NMAX, NMAX, 4, 4 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+            else rows_stage<NMAX, 0, 4, 4 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
         } else if (G == 4 || G == 2) {
             // two rows at a time in a rolled loop (long runs: measured 3 % ahead of four rows as one straight line
             // at 8192 x 5120, 4 % behind at 2048 rows, where the straight line is used for whole stages)
             int r = 0;
             if (G == 4) {
-                if (N == DR_NREG) {
+                if (N == NMAX) {
 #pragma unroll 1
                     for (; r + 2 <= rows; r += 2)
-                        rows_stage<DR_NREG, DR_NREG, 2, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                        rows_stage<NMAX, NMAX, 2, 4 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
                                                                                         orow + r * out_row_bytes, out_row_bytes, live);
                 } else {
 #pragma unroll 1
                     for (; r + 2 <= rows; r += 2)
-                        rows_stage<DR_NREG, 0, 2, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                        rows_stage<NMAX, 0, 2, 4 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
                                                                                   orow + r * out_row_bytes, out_row_bytes, live);
                 }
                 if (r < rows)
-                    rows_stage<DR_NREG, 0, 1, 4 * MAXT * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                    rows_stage<NMAX, 0, 1, 4 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
                                                                               orow + r * out_row_bytes, out_row_bytes, live);
             } else {
                 if (rows == 2) {
-                    if (N == DR_NREG) rows_stage<DR_NREG, DR_NREG, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
-                    else rows_stage<DR_NREG, 0, 2, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+                    if (N == NMAX) rows_stage<NMAX, NMAX, 2, 2 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+                    else rows_stage<NMAX, 0, 2, 2 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
                 } else {
-                    rows_stage<DR_NREG, 0, 1, 2 * MAXT * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
+                    rows_stage<NMAX, 0, 1, 2 * ROWCAP * 4, FP32OUT, HAS_BIAS>(sa, lp_b, row_b, N, sc, dc, b, orow, out_row_bytes, live);
                 }
             }
         } else {
 #pragma unroll 1
             for (int r = 0; r < rows; ++r)
-                rows_stage<DR_NREG, 0, 1, 0, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
+                rows_stage<NMAX, 0, 1, 0, FP32OUT, HAS_BIAS>(sa + (uint32_t)r * row_b, lp_b, row_b, N, sc, dc, b,
                                                                 orow + r * out_row_bytes, out_row_bytes, live);
         }
         if (warp_holes) {  // (uniform over the warp)
@@ -1384,33 +1449,34 @@ cudaError_t tpq_launch_dequant_generic(const tpq_ctx *c, const void *const *payl
 
 namespace {
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
+template <int NMAX, int ROWCAP, int MAXT, int DAUX, bool FP32OUT, bool HAS_BIAS, bool HAS_WAIT>
 cudaError_t launch_rows_w(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>,
+    cudaError_t e = cudaFuncSetAttribute(dequant_rows<NMAX, ROWCAP, MAXT, DAUX, FP32OUT, HAS_BIAS, HAS_WAIT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e == cudaSuccess)
-        e = tpq_launch_pdl(dequant_rows<NMAX, MAXT, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(consumers + DR_AUX + 32), smem,
-                           st, pp);
+        e = tpq_launch_pdl(dequant_rows<NMAX, ROWCAP, MAXT, DAUX, FP32OUT, HAS_BIAS, HAS_WAIT>, dim3(grid), dim3(consumers + DAUX + 32),
+                           smem, st, pp);
     return e;
 }
 
-template <int NMAX, int MAXT, bool FP32OUT, bool HAS_BIAS>
+template <int NMAX, int ROWCAP, int MAXT, int DAUX, bool FP32OUT, bool HAS_BIAS>
 cudaError_t launch_rows_v(const DRParams &pp, int grid, int consumers, size_t smem, cudaStream_t st)
 {
-    return pp.q.arr.words ? launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, true>(pp, grid, consumers, smem, st)
-                          : launch_rows_w<NMAX, MAXT, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
+    if constexpr (NMAX > 4) return launch_rows_w<NMAX, ROWCAP, MAXT, DAUX, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
+    return pp.q.arr.words ? launch_rows_w<NMAX, ROWCAP, MAXT, DAUX, FP32OUT, HAS_BIAS, true>(pp, grid, consumers, smem, st)
+                          : launch_rows_w<NMAX, ROWCAP, MAXT, DAUX, FP32OUT, HAS_BIAS, false>(pp, grid, consumers, smem, st);
 }
 
-template <int NMAX, int MAXT>
+template <int NMAX, int ROWCAP, int MAXT, int DAUX>
 cudaError_t launch_rows(const DRParams &pp, int fp32_out, int grid, int consumers, size_t smem, cudaStream_t st)
 {
     const bool bias = pp.q.bias != nullptr;
     if (fp32_out)
-        return bias ? launch_rows_v<NMAX, MAXT, true, true>(pp, grid, consumers, smem, st)
-                    : launch_rows_v<NMAX, MAXT, true, false>(pp, grid, consumers, smem, st);
-    return bias ? launch_rows_v<NMAX, MAXT, false, true>(pp, grid, consumers, smem, st)
-                : launch_rows_v<NMAX, MAXT, false, false>(pp, grid, consumers, smem, st);
+        return bias ? launch_rows_v<NMAX, ROWCAP, MAXT, DAUX, true, true>(pp, grid, consumers, smem, st)
+                    : launch_rows_v<NMAX, ROWCAP, MAXT, DAUX, true, false>(pp, grid, consumers, smem, st);
+    return bias ? launch_rows_v<NMAX, ROWCAP, MAXT, DAUX, false, true>(pp, grid, consumers, smem, st)
+                : launch_rows_v<NMAX, ROWCAP, MAXT, DAUX, false, false>(pp, grid, consumers, smem, st);
 }
 
 // rows after which the code stream is 16-byte aligned again: blocks and stages start on multiples of it
@@ -1425,23 +1491,31 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
 {
     const int N = c->N, E = c->E, k = c->k;
     const int L8 = (E - k) / 8;
-    // up to 8 devices: the steps of the first four live in the main threads' registers, those of the others in
-    // shared memory (beyond that the panel kernels, whose registers do not grow with N, take over)
+    // up to 8 devices: a main thread keeps the steps of all of them in registers.  Up to four, a block has one
+    // main thread per group; from five on that many registers leave room for half as many threads, so two
+    // blocks share a run of rows (each stages whole rows and decodes one half of the groups).  Beyond 8 the
+    // panel kernels, whose registers do not grow with N, take over.
     if (N > 8) return false;
-    if (L8 > (N > DR_NREG ? 640 : 768)) return false;  // consumer threads (register budget per thread)
+    const bool split = N > 4;
+    if (L8 > (split ? 640 : 768)) return false;  // main threads (two blocks per run: measured behind the panel kernels on wider rows)
+    const int runs = split ? c->sm_count / 2 : c->sm_count;
+    if (runs < 1) return false;
     const int g0 = g0_of(c);
     // every block takes the same number of adjacent rows (a multiple of g0), so no block has more than g0 - 1
     // rows above the mean; it walks them four at a time where a ring of three such stages fits, else two
-    int64_t rpb = (T + c->sm_count - 1) / c->sm_count;
+    int64_t rpb = (T + runs - 1) / runs;
     rpb = (rpb + g0 - 1) / g0 * g0;
-    // more than four devices: measured ahead of the copy-ring panel kernel on short inputs only (8 devices,
-    // 2048 x 5120: 22.9 against 24.7 us; level at 4096 tokens, behind from 8192 on)
-    if (N > DR_NREG && rpb > 16 && c->dq_kernel != 1) return false;
+    // 8 devices on rows the tensor-map panel kernel can address: that kernel is ahead from about 1200 rows on
+    // (8192 x 4096: 51 against 62 us; 2048 rows: 16.4 against 18.1; level at 1024); 5 to 7 devices: level or behind
+    if (N == 8 && L8 % 4 == 0 && rpb > 16 && c->dq_kernel != 1) return false;
     int G = 4;
-    if (rpb < 4 || dr_layout(N, E, k, 4, 3).total > (size_t)c->smem_optin) G = 2;
+    // (two blocks per run of rows: a ring of two four-row stages measured ahead of four two-row stages from
+    // 2048 rows on: 8 devices, 8192 x 5120: 70.6 against 75.9 us)
+    const int ring4 = (split && rpb >= 8) ? 2 : 3;
+    if (rpb < 4 || dr_layout(N, E, k, 4, ring4).total > (size_t)c->smem_optin) G = 2;
     if (G < g0) G = g0;
     if (dr_layout(N, E, k, G, 2).total > (size_t)c->smem_optin) return false;
-    const int grid = (int)((T + rpb - 1) / rpb);
+    const int grid = (int)((T + rpb - 1) / rpb) * (split ? 2 : 1);
     const int64_t per_block = (rpb + G - 1) / G;
     int nstage = (int)(per_block < 4 ? per_block : 4);  // deeper rings measured no faster (often slower)
     if (G == 4 && nstage > 3) nstage = 3;
@@ -1616,14 +1690,21 @@ cudaError_t tpq_launch_dequant_tiled(const tpq_ctx *c, const void *const *payloa
             pp.pairs = pp.rows_per_block > 32;
             const size_t smem = dr_layout(c->N, c->E, c->k, pp.G, pp.nstage).total;
             const int L8 = (c->E - c->k) / 8;
-            int consumers = ((L8 + 31) / 32) * 32;
+            pp.half_groups = (L8 + 1) / 2;
+            int consumers = (((c->N > 4 ? pp.half_groups : L8) + 31) / 32) * 32;
             if (consumers < 32) consumers = 32;
             cudaError_t e;
-            if (c->N > DR_NREG)
-                e = launch_rows<8, 640>(pp, fp32_out, grid, consumers, smem, st);
-            else
-                e = consumers <= 640 ? launch_rows<4, 640>(pp, fp32_out, grid, consumers, smem, st)
-                                     : launch_rows<4, 768>(pp, fp32_out, grid, consumers, smem, st);
+            if (c->N > 4) {
+                // (the device count is a compile-time constant there: measured 8 to 25 % ahead of a count read at run time)
+                switch (c->N) {
+                case 5: e = launch_rows<5, 640, 320, 160>(pp, fp32_out, grid, consumers, smem, st); break;
+                case 6: e = launch_rows<6, 640, 320, 160>(pp, fp32_out, grid, consumers, smem, st); break;
+                case 7: e = launch_rows<7, 640, 320, 160>(pp, fp32_out, grid, consumers, smem, st); break;
+                default: e = launch_rows<8, 640, 320, 160>(pp, fp32_out, grid, consumers, smem, st); break;
+                }
+            } else
+                e = L8 <= 640 ? launch_rows<4, 640, 640, DR_AUX>(pp, fp32_out, grid, consumers, smem, st)
+                              : launch_rows<4, 768, 768, DR_AUX>(pp, fp32_out, grid, consumers, smem, st);
             if (e != cudaSuccess) return e;
             ++*launches;
             return cudaGetLastError();

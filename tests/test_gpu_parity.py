@@ -229,6 +229,58 @@ def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
     t2.close()
 
 
+@pytest.mark.parametrize("N,T,E,features", [
+    (8, 1501, 5120, None),                              # the automatic choice: 630 groups, two-row stages, ragged end
+    (6, 4101, 5120, None),                              # four-row stages, ragged end
+    (5, 300, 1016, list(range(4, 1016, 64))),           # an odd number of groups (125): the halves differ by one
+    (7, 41, 1016, list(range(0, 16))),                  # every hole in the first block's half
+    (8, 41, 1016, list(range(992, 1000)) + list(range(1008, 1016))),   # holes in the second half only, selected features among the last k
+    (8, 7, 16, list(range(8, 16))),                     # one group: the second block has none
+    (6, 133, 1024, list(range(1, 1024, 2))[:400]),      # more selected features than auxiliary threads
+    (5, 64, 512, []),                                   # none selected
+])
+def test_row_kernel_with_two_blocks_per_run(N, T, E, features):
+    """5 to 8 devices: two blocks share a run of rows, each decoding half of the groups.  Forced on shapes that
+    reach each of its cases; FP32 and BF16 outputs, with and without a bias, bit-identical to the
+    shape-generic kernel's; the first shapes also against the oracle through the automatic choice."""
+    w = _workload(N, T, E, 29 * E + T, calib=(2, 8))
+    if features is None:
+        _full_pipeline(w, E // 64, binding.PATH_TILED)
+    scale = synth.column_scales(w)
+    t = binding.Tpq(N, E)
+    gu.calibrate_both(t, [synth.calibration_np(w, i, scale=scale) for i in range(N)])
+    if features is None:
+        t.select_features(E // 64)
+    else:
+        t.set_features(features)
+    P = t.payload_bytes(T)
+    pls = []
+    for i in range(N):
+        y = gu.dev_bf16(synth.activations_np(w, i, T, scale=scale))
+        buf = torch.empty(P, dtype=torch.uint8, device="cuda")
+        t.quantize_pack(i, y.data_ptr(), T, buf.data_ptr(), P)
+        pls.append(buf)
+    ptrs = [b.data_ptr() for b in pls]
+    bias = torch.from_numpy(np.random.default_rng(E + T).standard_normal(E).astype(np.float32)).cuda()
+    outs = {}
+    for name, path, kern in [("generic", binding.PATH_GENERIC, binding.DQ_AUTO), ("rows", binding.PATH_TILED, binding.DQ_ROWS)]:
+        t.set_option(binding.TPQ_OPT_KERNEL_PATH, path)
+        t.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, kern)
+        got = []
+        for b in (None, bias.data_ptr()):
+            o32 = torch.full((T, E), float("nan"), dtype=torch.float32, device="cuda")
+            o16 = torch.full((T, E), float("nan"), dtype=torch.bfloat16, device="cuda")
+            t.dequant_reduce(ptrs, T, o32.data_ptr(), binding.TPQ_OUT_FP32, bias_ptr=b)
+            t.dequant_reduce(ptrs, T, o16.data_ptr(), binding.TPQ_OUT_BF16, bias_ptr=b)
+            torch.cuda.synchronize()
+            assert t.device_status() == 0
+            got += [o32.view(torch.int32).cpu().numpy(), o16.view(torch.int16).cpu().numpy()]
+        outs[name] = got
+    for a, b in zip(outs["rows"], outs["generic"]):
+        assert np.array_equal(a, b)
+    t.close()
+
+
 @pytest.mark.parametrize("N,T,E,k", [(4, 301, 1024, 16), (16, 1203, 2048, 32), (9, 100, 1040, 8)])
 def test_back_to_back_launches_and_graph_replay_give_the_eager_result(N, T, E, k):
     """Calls enqueued back to back on one stream (the kernels start before the one ahead has drained and wait
