@@ -570,23 +570,40 @@ struct alignas(64) DTMaps {
 struct DTParams {
     DPParams d;
     int nstage;
+    int g0;  // rows after which the code stream is 16-byte aligned again (1, 2 or 4)
     int *status;
 };
 
-__host__ __device__ inline size_t dt_stage_bytes() { return (size_t)DT_NB * DT_MAIN * DP_R * 4; }  // CG*RC = DT_MAIN*DP_R words per device
-__host__ __device__ inline size_t dt_smem_bytes(int N, int CG, int nstage)
+// Rows whose length is not a multiple of 16 bytes ((E-k)/8 not a multiple of 4): g0 = 2 or 4 adjacent rows
+// are one row of the tensor map, so row class c (row index modulo g0) of a panel starts c*(E-k)/8 words into
+// it, rounded down to a multiple of 4 words (the copy's 16-byte rule); the box is 4 words wider, and a thread
+// reads its word (c*(E-k)/8 mod 4) words further on.  A device's part of a stage holds the g0 classes one
+// after the other, each padded to the 128 bytes the copy's destination must be aligned to.
+__host__ __device__ constexpr uint32_t dt_class_bytes(int CG, int g0)
 {
-    return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes() + (size_t)nstage * 16;  // steps, ring, mbarriers
+    return ((uint32_t)(CG + (g0 > 1 ? 4 : 0)) * (uint32_t)(DT_MAIN / CG * DP_R / g0) * 4u + 127u) & ~127u;
+}
+__host__ __device__ constexpr size_t dt_stage_bytes(int CG, int g0) { return (size_t)DT_NB * g0 * dt_class_bytes(CG, g0); }
+__host__ __device__ inline size_t dt_smem_bytes(int N, int CG, int nstage, int g0)
+{
+    return dp_steps_bytes(N, CG) + (size_t)nstage * dt_stage_bytes(CG, g0) + (size_t)nstage * 16;  // steps, ring, mbarriers
 }
 
 
-template <int CG, bool FP32OUT>
+template <int CG, int G0, int M4, bool FP32OUT>
 __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams tp, const __grid_constant__ DTMaps maps)
 {
     extern __shared__ __align__(128) uint8_t dp_smem[];
     constexpr int RS = DT_MAIN / CG, RC = RS * DP_R;
-    constexpr uint32_t BOX_BYTES = (uint32_t)CG * RC * 4;
+    constexpr int CGW = CG + (G0 > 1 ? 4 : 0);                          // words of a box row
+    constexpr uint32_t CLS_BYTES = dt_class_bytes(CG, G0);              // a row class of a device
+    constexpr uint32_t COPY_BYTES = (uint32_t)CGW * (RC / G0) * 4;      // what one copy brings
+    constexpr uint32_t BOX_BYTES = G0 * CLS_BYTES;                      // a device's part of a stage
     constexpr uint32_t STAGE_BYTES = DT_NB * BOX_BYTES;
+    // word offset of a thread's row r (0 <= r < DP_R) inside a device's part, relative to its row 0 of class 0
+    auto row_off = [](int r) constexpr {
+        return (r % G0) * (int)(CLS_BYTES / 4) + (r / G0) * CGW + ((r % G0) * M4) % 4;
+    };
     const DPParams &pp = tp.d;
     const DQParams &p = pp.q;
     const int N = p.N, E = p.E, k = p.k, L8 = (E - k) >> 3;
@@ -622,7 +639,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
     const int cg = tid & (CG - 1), rs = tid / CG;
     const DecodeConsts dc = decode_consts();
     const float4 *const my_steps = dp_steps + cg;
-    const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R) * CG + cg;
+    const uint32_t *const ring_w = reinterpret_cast<const uint32_t *>(ring) + (rs * DP_R / G0) * CGW + cg;
     // ring state: the producer lane and the main warps walk the same sequence of stages across segments
     int st = 0, it = 0;
     uint32_t parity = (tid >= DT_MAIN) ? 1u : 0u;  // producer: parity of the "empty" phase to wait for
@@ -661,10 +678,13 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                             dead = true;  // nothing more is issued; the loops go on so that every barrier is still met
                         }
                         if (!dead) {
-                            mbar_expect_tx(bar, (uint32_t)nb * BOX_BYTES);
+                            mbar_expect_tx(bar, (uint32_t)nb * G0 * COPY_BYTES);
                             const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
                             for (int i = 0; i < nb; ++i)
-                                tma_load_2d(stage + (uint32_t)i * BOX_BYTES, &maps.m[i0 + i], panel * CG, (int)(ch * RC), bar);
+#pragma unroll
+                                for (int cl = 0; cl < G0; ++cl)
+                                    tma_load_2d(stage + (uint32_t)i * BOX_BYTES + (uint32_t)cl * CLS_BYTES, &maps.m[i0 + i],
+                                                cl * L8 + panel * CG - (cl * M4) % 4, (int)(ch * (RC / G0)), bar);
                         }
                         if (++st == nstage) {
                             st = 0;
@@ -739,7 +759,7 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
 #pragma unroll
                 for (int i = 0; i < DT_NB; ++i)
 #pragma unroll
-                    for (int r = 0; r < DP_R; ++r) w[i][r] = sw[(i * RC + r) * CG];
+                    for (int r = 0; r < DP_R; ++r) w[i][r] = sw[i * (int)(BOX_BYTES / 4) + row_off(r)];
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&empty[st]));  // the stage's words are in registers
                 if (++st == nstage) {
@@ -1505,9 +1525,11 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     // rows above the mean; it walks them four at a time where a ring of three such stages fits, else two
     int64_t rpb = (T + runs - 1) / runs;
     rpb = (rpb + g0 - 1) / g0 * g0;
-    // 8 devices on rows the tensor-map panel kernel can address: that kernel is ahead from about 1200 rows on
-    // (8192 x 4096: 51 against 62 us; 2048 rows: 16.4 against 18.1; level at 1024); 5 to 7 devices: level or behind
-    if (N == 8 && L8 % 4 == 0 && rpb > 16 && c->dq_kernel != 1) return false;
+    // 8 devices: the tensor-map panel kernel (which needs a whole number of g0-row groups) is ahead on longer
+    // inputs: with 256-group panels from about 1200 rows on (8192 x 4096: 51 against 62 us; 2048 rows: 16.4
+    // against 18.1; level at 1024), with the 128-group panels of rows that are not a multiple of 16 bytes long
+    // from about 2400 on (8192 x 5120: 65.7 against 70.6 us; level at 2048); 5 to 7 devices: level or behind
+    if (N == 8 && T % g0 == 0 && rpb > (g0 > 1 ? 32 : 16) && c->dq_kernel != 1) return false;
     int G = 4;
     // (two blocks per run of rows: a ring of two four-row stages measured ahead of four two-row stages from
     // 2048 rows on: 8 devices, 8192 x 5120: 70.6 against 75.9 us)
@@ -1577,7 +1599,7 @@ cudaError_t launch_panels(const tpq_ctx *c, const DPParams &pp, cudaStream_t st)
 struct DTCacheEntry {
     const void *ptr;
     int64_t T;
-    int L8, CG, RC;
+    int L8, CG, RC, g0;
     CUtensorMap map;
 };
 struct DTCache {
@@ -1586,23 +1608,24 @@ struct DTCache {
     DTCacheEntry e[CAP];
 };
 
-bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC, CUtensorMap *out)
+bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC, int g0, CUtensorMap *out)
 {
     if (!c->dq_cache) c->dq_cache = new (std::nothrow) DTCache();
     DTCache *cache = static_cast<DTCache *>(c->dq_cache);
     if (cache)
         for (int j = 0; j < cache->n; ++j) {
             const DTCacheEntry &e = cache->e[j];
-            if (e.ptr == ptr && e.T == T && e.L8 == L8 && e.CG == CG && e.RC == RC) {
+            if (e.ptr == ptr && e.T == T && e.L8 == L8 && e.CG == CG && e.RC == RC && e.g0 == g0) {
                 *out = e.map;
                 return true;
             }
         }
     tpq_encode_tiled_fn fn = tpq_tensor_map_encoder();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)L8, (cuuint64_t)T};
-    const cuuint64_t strides[1] = {(cuuint64_t)L8 * 4};
-    const cuuint32_t box[2] = {(cuuint32_t)CG, (cuuint32_t)RC};
+    // (g0 adjacent rows are one row of the map: see dt_class_bytes)
+    const cuuint64_t dims[2] = {(cuuint64_t)g0 * L8, (cuuint64_t)(T / g0)};
+    const cuuint64_t strides[1] = {(cuuint64_t)g0 * L8 * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)(CG + (g0 > 1 ? 4 : 0)), (cuuint32_t)(RC / g0)};
     const cuuint32_t estr[2] = {1, 1};
     CUtensorMap m;
     if (fn(&m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(ptr), dims, strides, box, estr,
@@ -1611,7 +1634,7 @@ bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC,
         return false;
     if (cache) {
         DTCacheEntry &e = cache->e[cache->next];
-        e.ptr = ptr; e.T = T; e.L8 = L8; e.CG = CG; e.RC = RC; e.map = m;
+        e.ptr = ptr; e.T = T; e.L8 = L8; e.CG = CG; e.RC = RC; e.g0 = g0; e.map = m;
         cache->next = (cache->next + 1) % DTCache::CAP;
         if (cache->n < DTCache::CAP) ++cache->n;
     }
@@ -1623,10 +1646,13 @@ bool payload_map(tpq_ctx *c, const void *ptr, int64_t T, int L8, int CG, int RC,
 bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &tp, DTMaps &maps)
 {
     const int N = c->N, E = c->E, k = c->k, L8 = (E - k) / 8;
-    if (N > DT_MAX_DEV || L8 % 4 != 0 || T > 0x7FFFFFF0LL) return false;
-    int CG = 256;  // (measured at N = 16, E = 8192: panels of 256 groups 4 to 11 % ahead of 128)
-    while (CG >= 32 && dt_smem_bytes(N, CG, 2) > (size_t)c->smem_optin) CG >>= 1;
-    if (CG < 32) return false;
+    const int g0 = g0_of(c);
+    // (rows that are not a multiple of 16 bytes long: whole groups of g0 rows only, and panels of 128 groups:
+    // a box is at most 256 elements wide, and theirs is 4 wider than the panel)
+    if (N > DT_MAX_DEV || T % g0 != 0 || T > 0x7FFFFFF0LL) return false;
+    int CG = g0 > 1 ? 128 : 256;  // (measured at N = 16, E = 8192: panels of 256 groups 4 to 11 % ahead of 128)
+    while (CG >= 32 && dt_smem_bytes(N, CG, 2, g0) > (size_t)c->smem_optin) CG >>= 1;
+    if (CG < (g0 > 1 ? 128 : 32)) return false;
     const int RC = DT_MAIN / CG * DP_R;
     DPParams &pp = tp.d;
     pp.CG = CG;
@@ -1638,34 +1664,39 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     pp.gy = (int)(c->sm_count / pp.panels);
     if (pp.gy < 1) pp.gy = 0;
     int nstage = 6;
-    while (nstage > 2 && dt_smem_bytes(N, CG, nstage) > (size_t)c->smem_optin) --nstage;
+    while (nstage > 2 && dt_smem_bytes(N, CG, nstage, g0) > (size_t)c->smem_optin) --nstage;
     tp.nstage = nstage;
+    tp.g0 = g0;
     tp.status = c->t.status;
     for (int i = 0; i < N; ++i)
-        if (!payload_map(c, payloads[i], T, L8, CG, RC, &maps.m[i])) return false;
+        if (!payload_map(c, payloads[i], T, L8, CG, RC, g0, &maps.m[i])) return false;
     return true;
 }
 
-template <int CG, bool FP32OUT>
+template <int CG, int G0, int M4, bool FP32OUT>
 cudaError_t launch_tpanels_cg(const tpq_ctx *c, const DTParams &tp, const DTMaps &maps, cudaStream_t st)
 {
-    const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage);
-    cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = dt_smem_bytes(c->N, CG, tp.nstage, G0);
+    cudaError_t e = cudaFuncSetAttribute(dequant_tpanels<CG, G0, M4, FP32OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int64_t total = (int64_t)tp.d.panels * tp.d.n_chunks;
     unsigned grid = (unsigned)(total < c->sm_count ? total : c->sm_count);
     if (tp.d.gy > 0) grid = (unsigned)(tp.d.gy * tp.d.panels);
-    return tpq_launch_pdl(dequant_tpanels<CG, FP32OUT>, dim3(grid), dim3(DT_THREADS), smem, st, tp, maps);
+    return tpq_launch_pdl(dequant_tpanels<CG, G0, M4, FP32OUT>, dim3(grid), dim3(DT_THREADS), smem, st, tp, maps);
 }
 
 template <bool FP32OUT>
 cudaError_t launch_tpanels(const tpq_ctx *c, const DTParams &tp, const DTMaps &maps, cudaStream_t st)
 {
+    const int m4 = ((c->E - c->k) / 8) % 4;
+    if (tp.g0 == 2) return launch_tpanels_cg<128, 2, 2, FP32OUT>(c, tp, maps, st);
+    if (tp.g0 == 4)
+        return m4 == 1 ? launch_tpanels_cg<128, 4, 1, FP32OUT>(c, tp, maps, st) : launch_tpanels_cg<128, 4, 3, FP32OUT>(c, tp, maps, st);
     switch (tp.d.CG) {
-    case 256: return launch_tpanels_cg<256, FP32OUT>(c, tp, maps, st);
-    case 128: return launch_tpanels_cg<128, FP32OUT>(c, tp, maps, st);
-    case 64: return launch_tpanels_cg<64, FP32OUT>(c, tp, maps, st);
-    default: return launch_tpanels_cg<32, FP32OUT>(c, tp, maps, st);
+    case 256: return launch_tpanels_cg<256, 1, 0, FP32OUT>(c, tp, maps, st);
+    case 128: return launch_tpanels_cg<128, 1, 0, FP32OUT>(c, tp, maps, st);
+    case 64: return launch_tpanels_cg<64, 1, 0, FP32OUT>(c, tp, maps, st);
+    default: return launch_tpanels_cg<32, 1, 0, FP32OUT>(c, tp, maps, st);
     }
 }
 

@@ -184,7 +184,9 @@ def test_row_kernel_equals_generic_on_clustered_feature_sets():
 
 
 @pytest.mark.parametrize("N,T,E,k", [(4, 37, 512, 32), (2, 301, 1024, 32), (3, 16, 4096, 64), (4, 2, 256, 0), (1, 65, 6144, 96),
-                                     (8, 70, 1056, 32), (5, 33, 4096, 64), (7, 130, 520, 8)])
+                                     (8, 70, 1056, 32), (5, 33, 4096, 64), (7, 130, 520, 8),
+                                     # rows that are not a multiple of 16 bytes long: (E-k)/8 = 630, 129, 131 (mod 4: 2, 1, 3)
+                                     (8, 64, 5120, 80), (8, 36, 1048, 16), (3, 40, 1064, 16)])
 def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
     """The row, tensor-map panel and copy-ring panel kernels forced in turn on shapes that admit all three
     (short inputs included, where the automatic choice would not pick them): FP32 and BF16 outputs are
@@ -225,6 +227,12 @@ def test_every_dequant_kernel_gives_the_same_bits(N, T, E, k):
     t2.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, binding.DQ_ROWS)
     with pytest.raises(binding.TpqError):
         t2.dequant_reduce([pls[0].data_ptr()] * 9, 1, torch.empty((1, 512), dtype=torch.bfloat16, device="cuda").data_ptr())
+    # the tensor-map kernel takes rows that are not a multiple of 16 bytes long only in whole groups of 2 (or 4)
+    if (E - k) // 8 % 4 == 2:
+        t.set_option(binding.TPQ_OPT_KERNEL_PATH, binding.PATH_TILED)
+        t.set_option(binding.TPQ_OPT_DEQUANT_KERNEL, binding.DQ_TENSOR_PANELS)
+        with pytest.raises(binding.TpqError):
+            t.dequant_reduce(ptrs, T - 1, torch.empty((T, E), dtype=torch.bfloat16, device="cuda").data_ptr())
     t.close()
     t2.close()
 
