@@ -256,8 +256,8 @@ __device__ __forceinline__ void cp_async_wait()
 // a thread's DP_R rows of sums -> the output; lane n of a hole's slot holds the sum of the filler feature
 // lp_idx[8g+n] and goes to that feature's column
 template <bool FP32OUT>
-__device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *lp_idx, int64_t t0, int g, uint32_t mask,
-                                              const float2 (&acc_in)[DP_R][4])
+__device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *lp_idx, int64_t t0, int64_t t_lim, int g,
+                                              uint32_t mask, const float2 (&acc_in)[DP_R][4])
 {
     float2 acc[DP_R][4];
 #pragma unroll
@@ -284,14 +284,14 @@ __device__ __forceinline__ void dp_store_rows(const DQParams &p, const int32_t *
     if (mask == 0) {
 #pragma unroll
         for (int r = 0; r < DP_R; ++r)
-            if (t0 + r < p.T) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
+            if (t0 + r < t_lim) store_group<FP32OUT>(p.out, (t0 + r) * p.out_stride + 8 * (int64_t)g, acc[r], 0u);
     } else {
         int col[8];
 #pragma unroll
         for (int n = 0; n < 8; ++n) col[n] = (mask & (1u << n)) ? __ldg(lp_idx + 8 * g + n) : 8 * g + n;
 #pragma unroll
         for (int r = 0; r < DP_R; ++r)
-            if (t0 + r < p.T) {
+            if (t0 + r < t_lim) {
                 const int64_t orow = (t0 + r) * p.out_stride;
                 const float a8[8] = {acc[r][0].x, acc[r][0].y, acc[r][1].x, acc[r][1].y,
                                      acc[r][2].x, acc[r][2].y, acc[r][3].x, acc[r][3].y};
@@ -532,7 +532,7 @@ __global__ void __launch_bounds__(DP_THREADS, 1) dequant_panels(const DPParams p
             for (int i = 0; i < DP_NB; ++i)
                 if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
         }
-        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+        if (live) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, p.T, g, 0u, acc);
         pend = true;
         pend_on = it_on;
         pend_v = hv;
@@ -571,6 +571,7 @@ struct DTParams {
     DPParams d;
     int nstage;
     int g0;  // rows after which the code stream is 16-byte aligned again (1, 2 or 4)
+    int tail_rows;  // T mod g0: rows after the last whole group, which the tensor map does not cover
     int *status;
 };
 
@@ -578,7 +579,9 @@ struct DTParams {
 // are one row of the tensor map, so row class c (row index modulo g0) of a panel starts c*(E-k)/8 words into
 // it, rounded down to a multiple of 4 words (the copy's 16-byte rule); the box is 4 words wider, and a thread
 // reads its word (c*(E-k)/8 mod 4) words further on.  A device's part of a stage holds the g0 classes one
-// after the other, each padded to the 128 bytes the copy's destination must be aligned to.
+// after the other, each padded to the 128 bytes the copy's destination must be aligned to.  The T mod g0 rows
+// after the last whole group are a chunk of their own (the last one), whose words come by one plain bulk copy
+// per device and row, from the same 16-byte aligned places.
 __host__ __device__ constexpr uint32_t dt_class_bytes(int CG, int g0)
 {
     return ((uint32_t)(CG + (g0 > 1 ? 4 : 0)) * (uint32_t)(DT_MAIN / CG * DP_R / g0) * 4u + 127u) & ~127u;
@@ -677,9 +680,29 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                             atomicExch(tp.status, (int)TPQ_ERR_TIMEOUT);
                             dead = true;  // nothing more is issued; the loops go on so that every barrier is still met
                         }
-                        if (!dead) {
+                        const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
+                        if (G0 > 1 && tp.tail_rows > 0 && ch == pp.n_chunks - 1) {
+                            // the rows after the last whole group: row (= class) cl of the chunk, first box row
+                            if (!dead) {
+                                const int64_t row_bytes = (int64_t)L8 * 4, t_tail = p.T - tp.tail_rows;
+                                uint32_t bytes[G0 > 1 ? G0 : 1];
+                                uint32_t sum = 0;
+                                for (int cl = 0; cl < tp.tail_rows; ++cl) {
+                                    // from the class's aligned start to the end of the box row or of the code rows (padded to 16 bytes)
+                                    const int64_t from = (t_tail + cl) * row_bytes + (int64_t)(panel * CG - (cl * M4) % 4) * 4;
+                                    const int64_t end = (p.T * row_bytes + 15) & ~(int64_t)15;
+                                    bytes[cl] = (uint32_t)(end - from < (int64_t)CGW * 4 ? end - from : (int64_t)CGW * 4);
+                                    sum += bytes[cl];
+                                }
+                                mbar_expect_tx(bar, (uint32_t)nb * sum);
+                                for (int i = 0; i < nb; ++i)
+                                    for (int cl = 0; cl < tp.tail_rows; ++cl)
+                                        bulk_g2s(stage + (uint32_t)i * BOX_BYTES + (uint32_t)cl * CLS_BYTES,
+                                                 p.pl[i0 + i] + (t_tail + cl) * row_bytes + (int64_t)(panel * CG - (cl * M4) % 4) * 4,
+                                                 bytes[cl], bar);
+                            }
+                        } else if (!dead) {
                             mbar_expect_tx(bar, (uint32_t)nb * G0 * COPY_BYTES);
-                            const uint32_t stage = smem_u32(ring + (size_t)st * STAGE_BYTES);
                             for (int i = 0; i < nb; ++i)
 #pragma unroll
                                 for (int cl = 0; cl < G0; ++cl)
@@ -727,14 +750,17 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
         };
 
         for (int64_t ch = chb; ch < che; ch += cstep) {
-            const int64_t tc = ch * RC;
+            // (the chunk after the last whole group of g0 rows starts right there)
+            const bool tail = G0 > 1 && tp.tail_rows > 0 && ch == pp.n_chunks - 1;
+            const int64_t tc = tail ? p.T - tp.tail_rows : ch * RC;
+            const int64_t t_lim = tail ? p.T : p.T - (G0 > 1 ? tp.tail_rows : 0);  // (the maps' rows end at the last whole group)
             const int64_t t0 = tc + rs * DP_R;
             float2 acc[DP_R][4];
 #pragma unroll
             for (int r = 0; r < DP_R; ++r)
 #pragma unroll
                 for (int h = 0; h < 4; ++h) acc[r][h] = make_float2(0.0f, 0.0f);
-            const bool it_on = tid < items && tc + my_r < p.T;
+            const bool it_on = tid < items && tc + my_r < t_lim;
             const int64_t it_off = p.lp_bytes + ((tc + my_r) * k + my_h) * 2;
             float hv = 0.0f;
             uint16_t hvv[DT_NB] = {};
@@ -793,14 +819,14 @@ __global__ void __launch_bounds__(DT_THREADS, 1) dequant_tpanels(const DTParams 
                 for (int i = 0; i < DT_NB; ++i)
                     if (i < nl) hv = __fadd_rn(hv, __uint_as_float((uint32_t)hvv[i] << 16));
             }
-            if (live && !dead) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, g, 0u, acc);
+            if (live && !dead) dp_store_rows<FP32OUT>(p, pp.lp_idx, t0, t_lim, g, 0u, acc);
             if (n_it > 0) {
                 asm volatile("bar.sync 1, %0;" ::"n"(DT_MAIN) : "memory");  // the chunk's rows are stored
                 if (it_on && !dead) item_done(tc + my_r, my_col, my_fcol, hv);
                 // panels with more items than threads (many selected features in one panel): the rest, unpipelined
                 for (int a = tid + DT_MAIN; a < items && !dead; a += DT_MAIN) {
                     const int r = a / n_it, h = hs + (a - r * n_it);
-                    if (tc + r >= p.T) break;
+                    if (tc + r >= t_lim) break;
                     const int64_t off = p.lp_bytes + ((tc + r) * k + h) * 2;
                     float v = 0.0f;
                     for (int i = 0; i < N; ++i)
@@ -1525,11 +1551,11 @@ bool rows_plan(const tpq_ctx *c, int64_t T, int *G_out, int *nstage_out, int64_t
     // rows above the mean; it walks them four at a time where a ring of three such stages fits, else two
     int64_t rpb = (T + runs - 1) / runs;
     rpb = (rpb + g0 - 1) / g0 * g0;
-    // 8 devices: the tensor-map panel kernel (which needs a whole number of g0-row groups) is ahead on longer
+    // 8 devices: the tensor-map panel kernel is ahead on longer
     // inputs: with 256-group panels from about 1200 rows on (8192 x 4096: 51 against 62 us; 2048 rows: 16.4
     // against 18.1; level at 1024), with the 128-group panels of rows that are not a multiple of 16 bytes long
     // from about 2400 on (8192 x 5120: 65.7 against 70.6 us; level at 2048); 5 to 7 devices: level or behind
-    if (N == 8 && T % g0 == 0 && rpb > (g0 > 1 ? 32 : 16) && c->dq_kernel != 1) return false;
+    if (N == 8 && rpb > (g0 > 1 ? 32 : 16) && c->dq_kernel != 1) return false;
     int G = 4;
     // (two blocks per run of rows: a ring of two four-row stages measured ahead of four two-row stages from
     // 2048 rows on: 8 devices, 8192 x 5120: 70.6 against 75.9 us)
@@ -1647,9 +1673,10 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
 {
     const int N = c->N, E = c->E, k = c->k, L8 = (E - k) / 8;
     const int g0 = g0_of(c);
-    // (rows that are not a multiple of 16 bytes long: whole groups of g0 rows only, and panels of 128 groups:
-    // a box is at most 256 elements wide, and theirs is 4 wider than the panel)
-    if (N > DT_MAX_DEV || T % g0 != 0 || T > 0x7FFFFFF0LL) return false;
+    const int64_t Tm = T - T % g0;  // rows the tensor maps cover
+    // (rows that are not a multiple of 16 bytes long: panels of 128 groups: a box is at most 256 elements wide,
+    // and theirs is 4 wider than the panel)
+    if (N > DT_MAX_DEV || Tm == 0 || T > 0x7FFFFFF0LL) return false;
     int CG = g0 > 1 ? 128 : 256;  // (measured at N = 16, E = 8192: panels of 256 groups 4 to 11 % ahead of 128)
     while (CG >= 32 && dt_smem_bytes(N, CG, 2, g0) > (size_t)c->smem_optin) CG >>= 1;
     if (CG < (g0 > 1 ? 128 : 32)) return false;
@@ -1657,7 +1684,7 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     DPParams &pp = tp.d;
     pp.CG = CG;
     pp.panels = (L8 + CG - 1) / CG;
-    pp.n_chunks = (T + RC - 1) / RC;
+    pp.n_chunks = (Tm + RC - 1) / RC + (Tm < T ? 1 : 0);
     if (c->dq_kernel != 2 && pp.n_chunks * pp.panels < c->sm_count) return false;  // short inputs: the copy kernel starts faster
     // a block keeps its panel and takes every gy-th chunk (measured 2 to 4 % ahead of equal contiguous runs of
     // (panel, chunk) pairs, which reload the steps when a run crosses into the next panel)
@@ -1667,9 +1694,10 @@ bool tpanels_plan(tpq_ctx *c, const void *const *payloads, int64_t T, DTParams &
     while (nstage > 2 && dt_smem_bytes(N, CG, nstage, g0) > (size_t)c->smem_optin) --nstage;
     tp.nstage = nstage;
     tp.g0 = g0;
+    tp.tail_rows = (int)(T - Tm);
     tp.status = c->t.status;
     for (int i = 0; i < N; ++i)
-        if (!payload_map(c, payloads[i], T, L8, CG, RC, g0, &maps.m[i])) return false;
+        if (!payload_map(c, payloads[i], Tm, L8, CG, RC, g0, &maps.m[i])) return false;
     return true;
 }
 
