@@ -203,8 +203,9 @@ def oracle_leg(w, steps: int, warmup: int):
 
 # ------------------------------------------------------------------ the other configurations (extra.configs)
 def other_configs(args, dev, stream, peak, time_loop, graph_loop):
-    """Config 3 (decode shape: latency, plain launches and graph replay), config 5 at 8192 tokens, and the
-    calibration pass of config 4 on 32 sequences of one shard; the same kernels, timed the same way."""
+    """Config 3 (decode shape: latency, plain launches and graph replay), config 5 at 8192 tokens, config 2's
+    shape with 8 shards, and the calibration pass of config 4 on 32 sequences of one shard; the same kernels,
+    timed the same way."""
     import torch
     from paper_2411_07942_b200 import binding, synth
 
@@ -212,7 +213,7 @@ def other_configs(args, dev, stream, peak, time_loop, graph_loop):
     out = {}
 
     def build(wname, n_sets):
-        w = synth.WORKLOADS[wname]
+        w = wname if isinstance(wname, synth.Workload) else synth.WORKLOADS[wname]
         N, T, E = w.n_shards, w.tokens, w.features
         scale = synth.column_scales(w)
         t = binding.Tpq(N, E)
@@ -280,6 +281,10 @@ def other_configs(args, dev, stream, peak, time_loop, graph_loop):
     out["gemma27b_decode"] = timed("gemma27b_decode", 6, True)
     out["gemma27b_decode"]["note"] = "latency-bound (0.7 MB / 1.8 MB per call): microseconds per call are the figure"
     out["large_8192_tokens"] = timed("large", 2, False)
+    # the paper's tensor-parallel degree (8) on config 2's shape: the row kernel's variant for 5 to 8 devices
+    import dataclasses
+    out["llama13b_prefill_8_devices"] = timed(dataclasses.replace(synth.WORKLOADS["llama13b_prefill"], n_shards=8,
+                                                                  name="llama13b_prefill_8_devices"), 4, False)
     # config 4: the calibration pass, 32 sequences of 2048 tokens of one shard per call (two inputs in turn)
     w = synth.WORKLOADS["calibration"]
     E, S, n_seq = w.features, w.calib_tokens, 32
