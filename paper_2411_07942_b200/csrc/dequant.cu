@@ -1099,17 +1099,20 @@ __global__ void __launch_bounds__(MAXT + DAUX + 32, 1) dequant_rows(const DRPara
         // ---------------- auxiliary warps
         if constexpr (SPLIT) {
             // Two blocks share the rows.  Each adds up only the selected features that its own main threads
-            // overwrite (its holes, ranks [hs, he)) and stores one half of the last k columns, a selected one
+            // overwrite (its holes, ranks [hs, he)) and stores its share of the last k columns, a selected one
             // straight from the devices' BF16 values.  One item (a rank or a column) per thread and row; where
             // the threads outnumber the items, RP rows of a stage are worked on side by side.  What a thread
             // needs from the tables is loaded once.  Short rolled loops: this code runs once per stage, so
             // straight-line code would pay an instruction fetch for every few instructions it executes.
             const int at = tid - 32;
-            const int gfirst = half * pp.half_groups;
-            const int hs = half == 0 ? 0 : (gfirst < L8 ? (int)(__ldg(p.grp + gfirst) >> 8) : x.n_holes);
-            const int he = (half == 0 && pp.half_groups < L8) ? (int)(__ldg(p.grp + pp.half_groups) >> 8) : x.n_holes;
+            const int hmid = pp.half_groups < L8 ? (int)(__ldg(p.grp + pp.half_groups) >> 8) : x.n_holes;  // holes of the first half
+            const int hs = half == 0 ? 0 : hmid, he = half == 0 ? hmid : x.n_holes;
             const int nr = he - hs;
-            const int c0 = half == 0 ? 0 : k / 2, nc = half == 0 ? k / 2 : k - k / 2;
+            // the last k columns are divided so that both blocks have the same number of items (a block with a
+            // few more than DAUX / 2 would work on one row at a time instead of two)
+            int nc0 = (x.n_holes + k + 1) / 2 - hmid;
+            nc0 = nc0 < 0 ? 0 : (nc0 > k ? k : nc0);
+            const int c0 = half == 0 ? 0 : nc0, nc = half == 0 ? nc0 : k - nc0;
             const int W = nr + nc;  // items per row
             const bool fast = W > 0 && W <= DAUX;
             int RP = 1;
