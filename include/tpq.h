@@ -64,7 +64,8 @@ typedef enum {
     TPQ_OPT_KERNEL_PATH = 0,
     /* Which tiled kernel tpq_dequant_reduce uses when the tiled path is taken: 0 = chosen from the
      * shape (default); 1 = row kernel (needs N <= 4 and (E-k)/8 <= 768, or N <= 8 and (E-k)/8 <= 640); 2 = tensor-map panel kernel
-     * (needs N <= 16 and E-k a multiple of 32); 3 = copy-ring panel kernel.  A kernel that the shape
+     * (needs N <= 16 and at least as many rows as it takes for the code stream to be 16-byte aligned again:
+     * 1, 2 or 4); 3 = copy-ring panel kernel.  A kernel that the shape
      * does not admit makes the call return TPQ_ERR_INVALID_ARG.  For tests and measurements: all
      * kernels give identical results. */
     TPQ_OPT_DEQUANT_KERNEL = 1
