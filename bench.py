@@ -326,6 +326,7 @@ def main():
                     help="synthetic workload (default: the configuration the metric is quoted on; the others are "
                          "for profiling captures, e.g. `--workload large --tokens 1024 --sets 2`)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count")
+    ap.add_argument("--shards", type=int, default=0, help="override the workload's number of shards (devices)")
     ap.add_argument("--bits", type=int, default=4, help="code width (4 = the paper's Int4 and the bench's metric; "
                                                         "2..8 run on the shape-generic kernels)")
     args = ap.parse_args()
@@ -338,6 +339,8 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.tokens > 0:
         w = dataclasses.replace(w, tokens=args.tokens)
+    if args.shards > 0:
+        w = dataclasses.replace(w, n_shards=args.shards)
     N, T, E, k = w.n_shards, w.tokens, w.features, w.k
     in_bytes = N * T * E * 2
     config = {"workload": f"{args.workload}: N={N} shards x {T} tokens x {E} features BF16, k={k} BF16 features, "
@@ -629,7 +632,7 @@ def main():
                  "library_gemm_then_quantize_pack_ms": u_ms, "library_gemm_alone_ms": g_ms}
 
     configs_extra = None
-    if rank == 0 and world == 1 and not args.no_extra_configs and args.workload == WORKLOAD and not args.tokens and args.bits == 4:
+    if rank == 0 and world == 1 and not args.no_extra_configs and args.workload == WORKLOAD and not args.tokens and not args.shards and args.bits == 4:
         configs_extra = other_configs(args, dev, stream, peak, time_loop, graph_loop)
 
     # ---- end to end through the C ABI with HOST buffers (pinned), copies inside the timed region
@@ -688,7 +691,7 @@ def main():
     if args.bits != 4:
         config["workload"] += f", {args.bits}-bit codes"
         config["bits"] = args.bits
-    default_workload = args.workload == WORKLOAD and not args.tokens and args.bits == 4
+    default_workload = args.workload == WORKLOAD and not args.tokens and not args.shards and args.bits == 4
 
     def kernel_entry(name, ms_, graph_, nbytes, key):
         """One kernel's roofline entry: algorithmic bytes / measured launch time against the copy bandwidth,
